@@ -1,0 +1,123 @@
+/* S2A 4-bit activation stash for GELU and softmax -- C ABI of libs2a.so (sm_100a).
+ *
+ * The library implements the "Non-Parametric Layers" part (Section 3.2) of
+ * "Structure to Activation" (arXiv 2503.08154): in the forward pass a fused kernel
+ * evaluates the nonlinearity, writes its output, and keeps for the backward pass only
+ * a 4-bit code per element of the one tensor the derivative needs; in the backward
+ * pass a fused kernel unpacks and dequantises the codes and forms grad_in.
+ *
+ * Conventions shared by all four kernels
+ * --------------------------------------
+ * - Every pointer is a DEVICE pointer into memory the caller owns.  The library
+ *   allocates nothing, creates no stream and never synchronises; each call only
+ *   enqueues work on `cuda_stream` (a cudaStream_t passed as void*, NULL = the
+ *   default stream) and returns.
+ * - Tensors are contiguous and row-major: n_elems = n_rows * row_len.  A row is the
+ *   softmax axis, and for GELU the group of row_len consecutive elements that share
+ *   one quantisation range (normally the hidden vector of one token).
+ * - `dt` selects the element type of x / y / grad_out / grad_in: S2A_F32 (binary32)
+ *   or S2A_BF16 (bfloat16).  Arithmetic is binary32 in registers.
+ * - codes: s2a_codes_bytes(n_elems) bytes.  Element e of the flat tensor owns the low
+ *   nibble of byte e/2 when e is even and the high nibble when e is odd; with an odd
+ *   n_elems the last high nibble is written as 0.  (The paper fixes only the bit
+ *   width; the packing is this library's.)
+ * - meta: two floats per row, meta[2r] = min_r and meta[2r+1] = s_r of Eq. 8.
+ * - Quantiser (Eq. 8 with N = 4, per row, in correctly rounded binary32):
+ *     d = max - min; s = d / 15; inv = 15 / d;
+ *     code = round_half_even((v - min) * inv), a value in 0..15;
+ *   a constant row (d == 0) gets codes 0 and s = 0.  Dequantiser (Eq. 9):
+ *   v_hat = code * s + min.
+ * - Alignment: x, y, grad_out, grad_in and codes must be 16-byte aligned, meta 8-byte
+ *   aligned.  In-place use (y == x, grad_in == grad_out) is allowed; codes and meta
+ *   must not overlap any other argument.
+ * - Errors: arguments are checked on the host before anything is enqueued; on an
+ *   error nothing is launched and nothing is written.  n_elems == 0 returns S2A_OK
+ *   without a launch.  Inputs must be finite.
+ * - Supported row_len: 1 .. 2^31-1 (row lengths whose rows fit a shared-memory tile
+ *   take the pipelined path; others a slower row-at-a-time path).
+ */
+#ifndef S2A_H_
+#define S2A_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { S2A_F32 = 0, S2A_BF16 = 1 } s2a_dtype;
+
+typedef enum {
+  S2A_OK = 0,
+  S2A_ERR_NULL = 1,   /* a required pointer is NULL                              */
+  S2A_ERR_SHAPE = 2,  /* row_len == 0, or n_elems not a multiple of row_len      */
+  S2A_ERR_ALIGN = 3,  /* a pointer is not aligned as stated above                */
+  S2A_ERR_DTYPE = 4,  /* dt is neither S2A_F32 nor S2A_BF16                      */
+  S2A_ERR_CUDA = 5,   /* the CUDA runtime refused the launch                     */
+  S2A_ERR_DEVICE = 6  /* a kernel gave up on a bounded wait (see s2a_device_error) */
+} s2a_status;
+
+/* Bytes of packed codes for n_elems elements: (n_elems + 1) / 2. */
+size_t s2a_codes_bytes(size_t n_elems);
+
+/* Bytes of per-row metadata: (n_elems / row_len) * 2 * sizeof(float); 0 if row_len is 0. */
+size_t s2a_meta_bytes(size_t n_elems, size_t row_len);
+
+/* Static, human-readable name of a status code. */
+const char* s2a_status_string(int status);
+
+/* GELU forward with stash.  Eq. 10: y = x * sigmoid(1.702 x).  The stash is Eq. 8
+ * applied per row to the INPUT clipped into [-2, 2] (Section 3.2, "GeLU layer").
+ *   x      in   n_elems elements of type dt
+ *   y      out  n_elems elements of type dt (may alias x)
+ *   codes  out  s2a_codes_bytes(n_elems) bytes
+ *   meta   out  s2a_meta_bytes(n_elems, row_len) bytes
+ */
+int s2a_gelu_fwd(const void* x, void* y, uint8_t* codes, float* meta, size_t n_elems,
+                 size_t row_len, int dt, void* cuda_stream);
+
+/* GELU backward from the stash.  Eq. 9 gives x_hat; Eq. 12 gives the derivative
+ * sigmoid(1.702 x_hat) + 0.22 sin(1.5 x_hat); grad_in = grad_out * derivative.  The 16
+ * derivative values a row can take are evaluated in binary64 and rounded to binary32.
+ *   grad_out in   n_elems elements of type dt
+ *   codes    in   as written by s2a_gelu_fwd
+ *   meta     in   as written by s2a_gelu_fwd
+ *   grad_in  out  n_elems elements of type dt (may alias grad_out)
+ */
+int s2a_gelu_bwd(const void* grad_out, const uint8_t* codes, const float* meta, void* grad_in,
+                 size_t n_elems, size_t row_len, int dt, void* cuda_stream);
+
+/* Softmax forward with stash.  Eq. 7 over each row (the row maximum is subtracted
+ * first); y is rounded to dt and the values AS WRITTEN are quantised with Eq. 8 over
+ * the row, so codes == Q(y) exactly.  Arguments as for s2a_gelu_fwd.
+ */
+int s2a_softmax_fwd(const void* x, void* y, uint8_t* codes, float* meta, size_t n_elems,
+                    size_t row_len, int dt, void* cuda_stream);
+
+/* Softmax backward from the stash.  Eq. 9 gives y_hat; the Jacobian of Eq. 7 at y_hat
+ * applied to grad_out gives grad_in_i = y_hat_i * (grad_out_i - sum_j grad_out_j y_hat_j).
+ * Arguments as for s2a_gelu_bwd.
+ */
+int s2a_softmax_bwd(const void* grad_out, const uint8_t* codes, const float* meta, void* grad_in,
+                    size_t n_elems, size_t row_len, int dt, void* cuda_stream);
+
+/* The pipelined kernels wait on shared-memory barriers with an iteration limit; a
+ * wait that runs out records a bit in a per-device word and the kernel returns early.
+ * This call copies that word of the CURRENT device into *flags (0 = no kernel ever gave
+ * up) and clears it when `clear` is non-zero.  It synchronises the device.  Returns
+ * S2A_OK, S2A_ERR_NULL or S2A_ERR_CUDA.
+ */
+int s2a_device_error(unsigned int* flags, int clear);
+
+/* How a call would be run: writes into `out` (capacity `cap` bytes, always
+ * NUL-terminated) a one-line description of the kernel variant and launch shape chosen
+ * for (kernel, row_len, dt, n_elems).  kernel: 0 gelu_fwd, 1 gelu_bwd, 2 softmax_fwd,
+ * 3 softmax_bwd.  Host-only; launches nothing.  Returns S2A_OK or an argument error.
+ */
+int s2a_describe_plan(int kernel, size_t n_elems, size_t row_len, int dt, char* out, size_t cap);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* S2A_H_ */

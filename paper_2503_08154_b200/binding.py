@@ -1,0 +1,157 @@
+"""Thin ctypes binding of libs2a.so: argument marshalling only.
+
+Each function takes torch CUDA tensors (PyTorch is used for device memory and streams,
+nothing else), passes their raw pointers, the element count, the row length and the
+current stream to the C-ABI call of the same name, and raises on a non-zero status.
+There is no CPU path: a missing or unloadable library is an error.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libs2a.so")
+
+F32 = 0
+BF16 = 1
+GELU_FWD, GELU_BWD, SOFTMAX_FWD, SOFTMAX_BWD = 0, 1, 2, 3
+
+EXPORTS = (
+    "s2a_codes_bytes", "s2a_meta_bytes", "s2a_status_string", "s2a_gelu_fwd", "s2a_gelu_bwd",
+    "s2a_softmax_fwd", "s2a_softmax_bwd", "s2a_device_error", "s2a_describe_plan",
+)
+
+_lib = None
+
+
+class S2AError(RuntimeError):
+    pass
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libs2a.so (built in-tree by ``build.py``); raises if it is absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise S2AError("libs2a.so is not built: run `python -m paper_2503_08154_b200.build` "
+                           "(there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        c = ctypes
+        L.s2a_codes_bytes.argtypes = [c.c_size_t]
+        L.s2a_codes_bytes.restype = c.c_size_t
+        L.s2a_meta_bytes.argtypes = [c.c_size_t, c.c_size_t]
+        L.s2a_meta_bytes.restype = c.c_size_t
+        L.s2a_status_string.argtypes = [c.c_int]
+        L.s2a_status_string.restype = c.c_char_p
+        for name in ("s2a_gelu_fwd", "s2a_softmax_fwd", "s2a_gelu_bwd", "s2a_softmax_bwd"):
+            f = getattr(L, name)
+            f.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_size_t, c.c_size_t,
+                          c.c_int, c.c_void_p]
+            f.restype = c.c_int
+        L.s2a_device_error.argtypes = [c.POINTER(c.c_uint), c.c_int]
+        L.s2a_device_error.restype = c.c_int
+        L.s2a_describe_plan.argtypes = [c.c_int, c.c_size_t, c.c_size_t, c.c_int, c.c_char_p, c.c_size_t]
+        L.s2a_describe_plan.restype = c.c_int
+        _lib = L
+    return _lib
+
+
+def dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise S2AError("unsupported dtype %s (float32 or bfloat16)" % t.dtype)
+
+
+def codes_bytes(n_elems: int) -> int:
+    return int(lib().s2a_codes_bytes(n_elems))
+
+
+def meta_bytes(n_elems: int, row_len: int) -> int:
+    return int(lib().s2a_meta_bytes(n_elems, row_len))
+
+
+def status_string(status: int) -> str:
+    return lib().s2a_status_string(int(status)).decode()
+
+
+def check(status: int) -> None:
+    if status != 0:
+        raise S2AError(status_string(status))
+
+
+def _stream_ptr() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _dev(t: torch.Tensor, what: str) -> torch.Tensor:
+    if not t.is_cuda:
+        raise S2AError("%s must be a CUDA tensor" % what)
+    if not t.is_contiguous():
+        raise S2AError("%s must be contiguous" % what)
+    return t
+
+
+def alloc_stash(n_elems: int, row_len: int, device) -> tuple[torch.Tensor, torch.Tensor]:
+    """Device buffers for the packed codes (uint8) and the per-row (min, s) metadata."""
+    codes = torch.empty(codes_bytes(n_elems), dtype=torch.uint8, device=device)
+    meta = torch.empty(meta_bytes(n_elems, row_len) // 4, dtype=torch.float32, device=device)
+    return codes, meta
+
+
+def _fwd(fn, x, y, codes, meta, row_len):
+    _dev(x, "x"), _dev(y, "y"), _dev(codes, "codes"), _dev(meta, "meta")
+    n = x.numel()
+    if y.numel() != n or y.dtype != x.dtype:
+        raise S2AError("y must match x in size and dtype")
+    if codes.dtype != torch.uint8 or meta.dtype != torch.float32:
+        raise S2AError("codes must be uint8 and meta float32")
+    if row_len > 0 and (codes.numel() < codes_bytes(n) or meta.numel() * 4 < meta_bytes(n, row_len)):
+        raise S2AError("codes/meta buffers are too small")
+    check(fn(x.data_ptr(), y.data_ptr(), codes.data_ptr(), meta.data_ptr(), n, row_len,
+             dtype_code(x), _stream_ptr()))
+
+
+def _bwd(fn, grad_out, codes, meta, grad_in, row_len):
+    _dev(grad_out, "grad_out"), _dev(grad_in, "grad_in"), _dev(codes, "codes"), _dev(meta, "meta")
+    n = grad_out.numel()
+    if grad_in.numel() != n or grad_in.dtype != grad_out.dtype:
+        raise S2AError("grad_in must match grad_out in size and dtype")
+    if codes.dtype != torch.uint8 or meta.dtype != torch.float32:
+        raise S2AError("codes must be uint8 and meta float32")
+    if row_len > 0 and (codes.numel() < codes_bytes(n) or meta.numel() * 4 < meta_bytes(n, row_len)):
+        raise S2AError("codes/meta buffers are too small")
+    check(fn(grad_out.data_ptr(), codes.data_ptr(), meta.data_ptr(), grad_in.data_ptr(), n,
+             row_len, dtype_code(grad_out), _stream_ptr()))
+
+
+def s2a_gelu_fwd(x, y, codes, meta, row_len: int) -> None:
+    _fwd(lib().s2a_gelu_fwd, x, y, codes, meta, row_len)
+
+
+def s2a_gelu_bwd(grad_out, codes, meta, grad_in, row_len: int) -> None:
+    _bwd(lib().s2a_gelu_bwd, grad_out, codes, meta, grad_in, row_len)
+
+
+def s2a_softmax_fwd(x, y, codes, meta, row_len: int) -> None:
+    _fwd(lib().s2a_softmax_fwd, x, y, codes, meta, row_len)
+
+
+def s2a_softmax_bwd(grad_out, codes, meta, grad_in, row_len: int) -> None:
+    _bwd(lib().s2a_softmax_bwd, grad_out, codes, meta, grad_in, row_len)
+
+
+def s2a_device_error(clear: bool = False) -> int:
+    flags = ctypes.c_uint(0)
+    check(lib().s2a_device_error(ctypes.byref(flags), int(clear)))
+    return int(flags.value)
+
+
+def s2a_describe_plan(kernel: int, n_elems: int, row_len: int, dt: int) -> str:
+    buf = ctypes.create_string_buffer(256)
+    check(lib().s2a_describe_plan(kernel, n_elems, row_len, dt, buf, 256))
+    return buf.value.decode()

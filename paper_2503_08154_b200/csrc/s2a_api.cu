@@ -1,0 +1,118 @@
+// extern "C" entry points of libs2a.so: argument checks, choice of kernel path, launch.
+#include <stdio.h>
+#include <string.h>
+
+#include "../../include/s2a.h"
+#include "s2a_common.cuh"
+#include "s2a_launch.h"
+
+namespace {
+
+using namespace s2a;
+
+bool misaligned(const void* p, size_t a) { return ((uintptr_t)p & (a - 1)) != 0; }
+
+int check_args(const void* a, const void* b, const void* codes, const void* meta, size_t n,
+               size_t row_len, int dt) {
+  if (dt != S2A_F32 && dt != S2A_BF16) return S2A_ERR_DTYPE;
+  if (row_len == 0 || row_len > 0x7fffffffull || n % row_len != 0) return S2A_ERR_SHAPE;
+  if (n == 0) return S2A_OK;
+  if (!a || !b || !codes || !meta) return S2A_ERR_NULL;
+  if (misaligned(a, 16) || misaligned(b, 16) || misaligned(codes, 16) || misaligned(meta, 8))
+    return S2A_ERR_ALIGN;
+  return S2A_OK;
+}
+
+// Full tiles go to the pipelined kernel, whatever rows remain to the row-at-a-time one.
+int run(int kernel, const void* in, void* out, uint8_t* codes, float* meta, size_t n,
+        size_t row_len, int dt, void* stream) {
+  int rc = check_args(in, out, codes, meta, n, row_len, dt);
+  if (rc != S2A_OK || n == 0) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  const uint64_t n_rows = n / row_len;
+  TilePlan p = plan_tile(kernel, dt, n_rows, (uint32_t)row_len);
+  uint64_t done_rows = 0;
+  if (p.tile_rows != 0 && p.n_tiles != 0) {
+    TileArgs ta{in, out, codes, meta, (uint32_t)row_len, p.n_tiles};
+    if (launch_tile(kernel, dt, p, ta, st) != cudaSuccess) return S2A_ERR_CUDA;
+    done_rows = p.n_tiles * p.tile_rows;
+  }
+  if (done_rows < n_rows) {
+    RowwiseArgs ra{in, out, codes, meta, done_rows, n_rows - done_rows, (uint32_t)row_len};
+    if (launch_rowwise(kernel, dt, ra, st) != cudaSuccess) return S2A_ERR_CUDA;
+  }
+  return S2A_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t s2a_codes_bytes(size_t n_elems) { return (n_elems + 1) / 2; }
+
+size_t s2a_meta_bytes(size_t n_elems, size_t row_len) {
+  return row_len == 0 ? 0 : (n_elems / row_len) * 2 * sizeof(float);
+}
+
+const char* s2a_status_string(int status) {
+  switch (status) {
+    case S2A_OK: return "S2A_OK";
+    case S2A_ERR_NULL: return "S2A_ERR_NULL: a required pointer is NULL";
+    case S2A_ERR_SHAPE: return "S2A_ERR_SHAPE: row_len is 0 or does not divide n_elems";
+    case S2A_ERR_ALIGN: return "S2A_ERR_ALIGN: data/codes need 16-byte, meta 8-byte alignment";
+    case S2A_ERR_DTYPE: return "S2A_ERR_DTYPE: dt must be S2A_F32 or S2A_BF16";
+    case S2A_ERR_CUDA: return "S2A_ERR_CUDA: the CUDA runtime refused the launch";
+    case S2A_ERR_DEVICE: return "S2A_ERR_DEVICE: a kernel gave up on a bounded wait";
+    default: return "unknown s2a status";
+  }
+}
+
+int s2a_gelu_fwd(const void* x, void* y, uint8_t* codes, float* meta, size_t n_elems,
+                 size_t row_len, int dt, void* cuda_stream) {
+  return run(kGeluFwd, x, y, codes, meta, n_elems, row_len, dt, cuda_stream);
+}
+
+int s2a_gelu_bwd(const void* grad_out, const uint8_t* codes, const float* meta, void* grad_in,
+                 size_t n_elems, size_t row_len, int dt, void* cuda_stream) {
+  return run(kGeluBwd, grad_out, grad_in, const_cast<uint8_t*>(codes), const_cast<float*>(meta),
+             n_elems, row_len, dt, cuda_stream);
+}
+
+int s2a_softmax_fwd(const void* x, void* y, uint8_t* codes, float* meta, size_t n_elems,
+                    size_t row_len, int dt, void* cuda_stream) {
+  return run(kSoftmaxFwd, x, y, codes, meta, n_elems, row_len, dt, cuda_stream);
+}
+
+int s2a_softmax_bwd(const void* grad_out, const uint8_t* codes, const float* meta, void* grad_in,
+                    size_t n_elems, size_t row_len, int dt, void* cuda_stream) {
+  return run(kSoftmaxBwd, grad_out, grad_in, const_cast<uint8_t*>(codes),
+             const_cast<float*>(meta), n_elems, row_len, dt, cuda_stream);
+}
+
+int s2a_device_error(unsigned int* flags, int clear) {
+  if (!flags) return S2A_ERR_NULL;
+  return read_error_word(flags, clear != 0) == cudaSuccess ? S2A_OK : S2A_ERR_CUDA;
+}
+
+int s2a_describe_plan(int kernel, size_t n_elems, size_t row_len, int dt, char* out, size_t cap) {
+  if (!out || cap == 0) return S2A_ERR_NULL;
+  out[0] = 0;
+  if (kernel < 0 || kernel > 3) return S2A_ERR_SHAPE;
+  if (dt != S2A_F32 && dt != S2A_BF16) return S2A_ERR_DTYPE;
+  if (row_len == 0 || row_len > 0x7fffffffull || n_elems % row_len != 0) return S2A_ERR_SHAPE;
+  const uint64_t n_rows = n_elems / row_len;
+  TilePlan p = plan_tile(kernel, dt, n_rows, (uint32_t)row_len);
+  if (p.tile_rows == 0 || p.n_tiles == 0) {
+    snprintf(out, cap, "rowwise rows=%llu", (unsigned long long)n_rows);
+  } else {
+    snprintf(out, cap,
+             "tile rows/tile=%u unit=%u vec=%u iters=%u warps=%u stages=%u smem=%u grid=%u "
+             "tiles=%llu tail_rows=%llu",
+             p.tile_rows, p.unit_lanes, p.vec_elems, p.iters, p.warps, p.stages, p.smem_bytes,
+             p.grid, (unsigned long long)p.n_tiles,
+             (unsigned long long)(n_rows - p.n_tiles * p.tile_rows));
+  }
+  return S2A_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,108 @@
+// Device-side building blocks shared by the S2A kernels: I/O type traits, the Eq. 8
+// quantiser in pinned binary32 operations, Eq. 10 / Eq. 12 arithmetic, reductions.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace s2a {
+
+constexpr int kF32 = 0;
+constexpr int kBF16 = 1;
+
+constexpr float kSlope = 1.702f;   // Eq. 10 / Eq. 12: sigmoid(1.702 x)
+constexpr float kSineAmp = 0.22f;  // Eq. 12: 0.22 sin(1.5 x)
+constexpr float kSineFreq = 1.5f;
+constexpr float kClip = 2.0f;      // Section 3.2: GELU input clipped into [-2, 2]
+constexpr float kLevels = 15.0f;   // 2^N - 1 with N = 4 (Eq. 8)
+
+// Bits of the per-device error word (see s2a_device_error).
+constexpr unsigned kErrLoadWait = 1u;   // a consumer gave up waiting for a tile to arrive
+constexpr unsigned kErrDrainWait = 2u;  // the producer gave up waiting for the consumers
+
+// ---------------------------------------------------------------- I/O element types
+template <int DT> struct Io;
+template <> struct Io<kF32> {
+  using T = float;
+  static constexpr int kBytes = 4;
+  static __device__ __forceinline__ float widen(float v) { return v; }
+  static __device__ __forceinline__ float narrow(float v) { return v; }
+};
+template <> struct Io<kBF16> {
+  using T = __nv_bfloat16;
+  static constexpr int kBytes = 2;
+  static __device__ __forceinline__ float widen(__nv_bfloat16 v) { return __bfloat162float(v); }
+  static __device__ __forceinline__ __nv_bfloat16 narrow(float v) { return __float2bfloat16_rn(v); }
+};
+
+// ---------------------------------------------------------------- Eq. 8 quantiser
+// Specified as correctly rounded binary32 steps; the intrinsics keep the compiler from
+// contracting the subtract and the multiply into one fused operation.
+struct QRange {
+  float mn;   // min of the row
+  float inv;  // 15 / (max - min), 0 for a constant row
+  float s;    // (max - min) / 15, 0 for a constant row
+};
+
+__device__ __forceinline__ QRange make_qrange(float mn, float mx) {
+  QRange q;
+  q.mn = mn;
+  float d = __fsub_rn(mx, mn);
+  if (d == 0.0f) {
+    q.inv = 0.0f;
+    q.s = 0.0f;
+  } else {
+    q.inv = __fdiv_rn(kLevels, d);
+    q.s = __fdiv_rn(d, kLevels);
+  }
+  return q;
+}
+
+// For v inside [min, max] the scaled value lies in [0, 15 + 2^-20], so adding
+// 1.5 * 2^23 rounds it half-to-even into the low mantissa bits without a clamp.
+__device__ __forceinline__ uint32_t quant_code(float v, const QRange& q) {
+  float t = __fmul_rn(__fsub_rn(v, q.mn), q.inv);
+  return __float_as_uint(__fadd_rn(t, 12582912.0f)) & 0xFu;
+}
+
+// Eq. 9 in binary32: one rounding of the exact code * s + min.
+__device__ __forceinline__ float dequant(uint32_t code, float mn, float s) {
+  return __fmaf_rn((float)code, s, mn);
+}
+
+// ---------------------------------------------------------------- Eq. 10 and Eq. 12
+// y = x / (1 + exp(-1.702 x)).  The product 1.702 x is carried as hi + lo so that its
+// rounding does not scale the error of exp with |x|.
+__device__ __forceinline__ float gelu_value(float x) {
+  float z = __fmul_rn(kSlope, x);
+  float zlo = __fmaf_rn(kSlope, x, -z);
+  float e = expf(-z) * (1.0f - zlo);  // exp(-(z + zlo)); stays inf when exp overflows
+  return __fdiv_rn(x, 1.0f + e);
+}
+
+// Eq. 12 at a dequantised x_hat = code * s + min, in binary64.
+__device__ __forceinline__ double gelu_sine_derivative(uint32_t code, float mn, float s) {
+  double xh = (double)code * (double)s + (double)mn;
+  double sig = 1.0 / (1.0 + exp(-(double)kSlope * xh));
+  return sig + (double)kSineAmp * sin((double)kSineFreq * xh);
+}
+
+// ---------------------------------------------------------------- warp reductions
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_min(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fminf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+}  // namespace s2a

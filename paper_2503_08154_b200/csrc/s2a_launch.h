@@ -1,0 +1,59 @@
+// Host-side launch interfaces between the C-ABI entry points and the kernel files.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace s2a {
+
+enum { kGeluFwd = 0, kGeluBwd = 1, kSoftmaxFwd = 2, kSoftmaxBwd = 3 };
+
+// One launch of a row-at-a-time kernel over rows [row0, row0 + n_rows) of a tensor.
+// row0 * row_len must be even (whole code bytes).  `in` is x or grad_out, `out` is y or
+// grad_in, both pointing at element 0 of the whole tensor; codes and meta likewise.
+struct RowwiseArgs {
+  const void* in;
+  void* out;
+  uint8_t* codes;  // written by the forward kernels, read by the backward kernels
+  float* meta;     // likewise
+  uint64_t row0;
+  uint64_t n_rows;
+  uint32_t row_len;
+};
+
+cudaError_t launch_rowwise(int kernel, int dt, const RowwiseArgs& a, cudaStream_t st);
+
+// ---------------------------------------------------------------- pipelined tiles
+// A tile is `tile_rows` consecutive rows whose flat element span starts and ends on a
+// multiple of 32 elements, so that its data and its code bytes can move with 16-byte
+// bulk copies.  A plan with tile_rows == 0 means "no pipelined path for this shape".
+struct TilePlan {
+  uint32_t tile_rows;   // rows per tile (0: not applicable)
+  uint32_t unit_lanes;  // lanes that cooperate on one row: 8, 16 or 32
+  uint32_t vec_elems;   // elements per shared-memory access: 2 (pair mode) or 16 bytes' worth
+  uint32_t iters;       // compile-time bound on accesses per lane per row
+  uint32_t warps;       // consumer warps per CTA (one more warp drives the copies)
+  uint32_t stages;      // tiles resident in shared memory per CTA
+  uint32_t smem_bytes;  // dynamic shared memory per CTA
+  uint32_t grid;        // CTAs launched
+  uint64_t n_tiles;     // full tiles covered; remaining rows go to the row-at-a-time path
+};
+
+struct TileArgs {
+  const void* in;
+  void* out;
+  uint8_t* codes;
+  float* meta;
+  uint32_t row_len;
+  uint64_t n_tiles;
+};
+
+// Chooses the launch shape for (kernel, dt, row_len, n_rows) on the current device.
+TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t row_len);
+cudaError_t launch_tile(int kernel, int dt, const TilePlan& p, const TileArgs& a, cudaStream_t st);
+
+// Reads (and optionally clears) the per-device error word the pipelined kernels set
+// when a bounded wait runs out.  Synchronises the device.
+cudaError_t read_error_word(unsigned int* flags, bool clear);
+
+}  // namespace s2a

@@ -1,0 +1,168 @@
+"""Helpers of the GPU parity tests: moving seeded host arrays through the C-ABI calls
+(with guard bands around every output), and the tolerance checks.
+
+Tolerances (all written out here, used by every parity test):
+
+* 4-bit codes and (min, s) metadata: bit-exact.  GELU codes depend on x only, so they
+  must equal the oracle's everywhere.  Softmax codes are Q(y as written): they must
+  equal an independent numpy binary32 evaluation of Eq. 8 on the GPU's own y with zero
+  tolerance, and may differ from the oracle's codes only where the GPU's y (or the
+  row's min/max) differs from the oracle's by its allowed rounding -- such elements sit
+  within one ulp of a bin edge; they are counted and the count is bounded.
+* binary32 outputs: |a - b| <= rtol * (|b| + M) + 2^-126 with rtol = 1e-6.  M is 0
+  except for the softmax VJP, where it is y_hat_i * sum_j |g_j| y_hat_j (the size of the
+  terms that cancel in g_i - dot), and for softmax y, where rtol is widened by
+  2^-24 * |x_i - max_j x_j| (the rounding of the exponent's argument).
+* bfloat16 outputs: within 1 bfloat16 ulp of max(|b|, M).
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from paper_2503_08154_b200 import binding, synth
+
+F32, BF16 = 0, 1
+GUARD = 512  # bytes of canary on each side of every output buffer
+CANARY = 0xA5
+
+
+def torch_dtype(dt):
+    return torch.float32 if dt == F32 else torch.bfloat16
+
+
+def to_device(a: np.ndarray, dt: int) -> torch.Tensor:
+    if dt == F32:
+        return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).cuda()
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.uint16).view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def to_host(t: torch.Tensor, dt: int) -> np.ndarray:
+    if dt == F32:
+        return t.detach().cpu().numpy()
+    return t.detach().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+class Guarded:
+    """A device buffer of `nbytes` with canary bytes on both sides."""
+
+    def __init__(self, nbytes: int):
+        self.nbytes = nbytes
+        self.raw = torch.full((nbytes + 2 * GUARD,), CANARY, dtype=torch.uint8, device="cuda")
+        self.body = self.raw[GUARD:GUARD + nbytes]
+
+    def view(self, dtype):
+        return self.body.view(dtype) if self.nbytes else torch.empty(0, dtype=dtype, device="cuda")
+
+    def check(self, what: str):
+        raw = self.raw.cpu().numpy()
+        assert (raw[:GUARD] == CANARY).all(), "%s: bytes before the buffer were overwritten" % what
+        assert (raw[GUARD + self.nbytes:] == CANARY).all(), "%s: bytes after the buffer were overwritten" % what
+
+
+def _round16(n):
+    return (n + 15) // 16 * 16
+
+
+def gpu_fwd(kind: str, x: np.ndarray, L: int, dt: int, inplace: bool = False):
+    """Runs s2a_{gelu,softmax}_fwd on a host array; returns (y, codes, meta) as numpy."""
+    n = x.size
+    item = synth.io_itemsize(dt)
+    xd = to_device(x, dt)
+    yg = Guarded(n * item)
+    cg = Guarded(binding.codes_bytes(n))
+    mg = Guarded(binding.meta_bytes(n, L))
+    if inplace:
+        yg.view(torch_dtype(dt)).copy_(xd)
+        xin = yg.view(torch_dtype(dt))
+    else:
+        xin = xd
+    fn = binding.s2a_gelu_fwd if kind == "gelu" else binding.s2a_softmax_fwd
+    fn(xin, yg.view(torch_dtype(dt)), cg.view(torch.uint8), mg.view(torch.float32), L)
+    torch.cuda.synchronize()
+    assert binding.s2a_device_error() == 0
+    for g, w in ((yg, "y"), (cg, "codes"), (mg, "meta")):
+        g.check(kind + "_fwd " + w)
+    if not inplace:
+        assert np.array_equal(to_host(xd, dt), x), "the input tensor was modified"
+    return to_host(yg.view(torch_dtype(dt)), dt), cg.view(torch.uint8).cpu().numpy(), mg.view(torch.float32).cpu().numpy()
+
+
+def gpu_bwd(kind: str, g: np.ndarray, codes: np.ndarray, meta: np.ndarray, L: int, dt: int,
+            inplace: bool = False):
+    n = g.size
+    item = synth.io_itemsize(dt)
+    gd = to_device(g, dt)
+    cd = torch.from_numpy(np.ascontiguousarray(codes)).cuda()
+    md = torch.from_numpy(np.ascontiguousarray(meta)).cuda()
+    og = Guarded(n * item)
+    if inplace:
+        og.view(torch_dtype(dt)).copy_(gd)
+        gin = og.view(torch_dtype(dt))
+    else:
+        gin = gd
+    fn = binding.s2a_gelu_bwd if kind == "gelu" else binding.s2a_softmax_bwd
+    fn(gin, cd, md, og.view(torch_dtype(dt)), L)
+    torch.cuda.synchronize()
+    assert binding.s2a_device_error() == 0
+    og.check(kind + "_bwd grad_in")
+    assert np.array_equal(cd.cpu().numpy(), codes) and np.array_equal(md.cpu().numpy(), meta)
+    return to_host(og.view(torch_dtype(dt)), dt)
+
+
+# ------------------------------------------------------------------ host-side checks
+def widen(a: np.ndarray, dt: int) -> np.ndarray:
+    return synth.io_to_f32(a, dt).astype(np.float64)
+
+
+def numpy_quantize(v32: np.ndarray, L: int):
+    """Eq. 8 as the header specifies it, in numpy binary32 (independent of the oracle and
+    of the kernels).  Returns (unpacked codes uint8 [rows, L], meta float32 [2*rows])."""
+    v = np.ascontiguousarray(v32, dtype=np.float32).reshape(-1, L)
+    mn = v.min(axis=1, keepdims=True)
+    mx = v.max(axis=1, keepdims=True)
+    d = (mx - mn).astype(np.float32)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        inv = np.where(d == 0, np.float32(0), np.float32(15) / d).astype(np.float32)
+        s = np.where(d == 0, np.float32(0), d / np.float32(15)).astype(np.float32)
+    t = ((v - mn).astype(np.float32) * inv).astype(np.float32)
+    q = np.clip(np.rint(t), 0, 15).astype(np.uint8)
+    meta = np.empty(2 * v.shape[0], dtype=np.float32)
+    meta[0::2] = mn[:, 0]
+    meta[1::2] = s[:, 0]
+    return q, meta
+
+
+def unpack_np(codes: np.ndarray, n: int) -> np.ndarray:
+    out = np.empty(2 * codes.size, dtype=np.uint8)
+    out[0::2] = codes & 0xF
+    out[1::2] = codes >> 4
+    return out[:n]
+
+
+def bf16_ulp(mag: np.ndarray) -> np.ndarray:
+    """Spacing of bfloat16 numbers at magnitude `mag` (>= the subnormal spacing)."""
+    mag = np.maximum(np.abs(mag), 2.0 ** -126)
+    return np.exp2(np.floor(np.log2(mag)) - 7)
+
+
+def assert_close(got, want, dt, what, extra_mag=None, extra_rtol=None):
+    """got/want: float64 arrays of widened outputs.  See the module docstring."""
+    got = np.asarray(got, dtype=np.float64).reshape(-1)
+    want = np.asarray(want, dtype=np.float64).reshape(-1)
+    mag = np.abs(want) if extra_mag is None else np.abs(want) + np.asarray(extra_mag).reshape(-1)
+    if dt == F32:
+        rtol = 1e-6 if extra_rtol is None else 1e-6 + np.asarray(extra_rtol).reshape(-1)
+        tol = rtol * mag + 2.0 ** -126
+    else:
+        ref = np.abs(want) if extra_mag is None else np.maximum(np.abs(want), np.asarray(extra_mag).reshape(-1))
+        tol = bf16_ulp(ref)
+        if extra_rtol is not None:
+            tol = tol + np.asarray(extra_rtol).reshape(-1) * mag
+    err = np.abs(got - want)
+    bad = err > tol
+    if bad.any():
+        i = int(np.argmax(err / tol))
+        raise AssertionError("%s: %d of %d outside tolerance; worst at %d: got %r want %r tol %r"
+                             % (what, int(bad.sum()), got.size, i, got[i], want[i], tol[i]))
+    return float(np.max(err / np.maximum(mag, 1e-300)))

@@ -1,0 +1,208 @@
+"""GPU parity: the CUDA kernels, called through the C ABI, against the CPU oracle on the
+same seeded inputs, element by element.  Tolerances are in parity_util's docstring."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import s2a_oracle as o
+from paper_2503_08154_b200 import binding, synth
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+F32, BF16 = 0, 1
+THREADS = max(1, os.cpu_count() or 1)
+
+
+# ------------------------------------------------------------------ the two checks
+def check_gelu(x, g, L, dt, inplace=False):
+    n = x.size
+    y_o, codes_o, meta_o = o.gelu_fwd(x, L, dt, threads=THREADS)
+    y_g, codes_g, meta_g = pu.gpu_fwd("gelu", x, L, dt, inplace=inplace)
+    assert np.array_equal(codes_g, codes_o), "GELU codes differ from the oracle's"
+    assert np.array_equal(meta_g.view(np.uint32), meta_o.view(np.uint32)), "GELU (min, s) differ"
+    pu.assert_close(pu.widen(y_g, dt), pu.widen(y_o, dt), dt, "gelu y")
+    gin_o = o.gelu_bwd(g, codes_o, meta_o, L, dt, threads=THREADS)
+    gin_g = pu.gpu_bwd("gelu", g, codes_o, meta_o, L, dt, inplace=inplace)
+    pu.assert_close(pu.widen(gin_g, dt), pu.widen(gin_o, dt), dt, "gelu grad_in")
+    return n
+
+
+def check_softmax(x, g, L, dt, inplace=False, max_flip_frac=2e-3):
+    n = x.size
+    rows = n // L
+    y_o, codes_o, meta_o = o.softmax_fwd(x, L, dt, threads=THREADS)
+    y_g, codes_g, meta_g = pu.gpu_fwd("softmax", x, L, dt, inplace=inplace)
+    xw = pu.widen(x, dt).reshape(rows, L)
+    arg_gap = (xw.max(axis=1, keepdims=True) - xw) * 2.0 ** -24
+    pu.assert_close(pu.widen(y_g, dt), pu.widen(y_o, dt), dt, "softmax y", extra_rtol=arg_gap)
+    # the stash is exactly Q(y as written), checked without the oracle and without tolerance
+    q_np, meta_np = pu.numpy_quantize(synth.io_to_f32(y_g, dt), L)
+    q_g = pu.unpack_np(codes_g, n).reshape(rows, L)
+    assert np.array_equal(q_g, q_np), "softmax codes are not Q(y as written)"
+    assert np.array_equal(meta_g.view(np.uint32), meta_np.view(np.uint32))
+    if n % 2 == 1:
+        assert codes_g[-1] >> 4 == 0, "unpaired last nibble must be zero"
+    # against the oracle's codes: differences only where y or the row range moved by rounding
+    q_o = pu.unpack_np(codes_o, n).reshape(rows, L)
+    diff = q_g != q_o
+    if diff.any():
+        y_same = (y_g.reshape(rows, L) == y_o.reshape(rows, L))
+        meta_same = (meta_g.reshape(rows, 2).view(np.uint32) == meta_o.reshape(rows, 2).view(np.uint32)).all(axis=1)
+        unexplained = diff & y_same & meta_same[:, None]
+        assert not unexplained.any(), "codes differ where y and the row range agree"
+        assert np.abs(q_g.astype(int) - q_o.astype(int)).max() <= 1
+        assert diff.mean() <= max_flip_frac, "too many edge flips: %g" % diff.mean()
+    # backward from the ORACLE's stash, so that both sides see identical inputs
+    gin_o = o.softmax_bwd(g, codes_o, meta_o, L, dt, threads=THREADS)
+    gin_g = pu.gpu_bwd("softmax", g, codes_o, meta_o, L, dt, inplace=inplace)
+    yh = q_o.astype(np.float64) * meta_o[1::2, None].astype(np.float64) + meta_o[0::2, None].astype(np.float64)
+    gw = pu.widen(g, dt).reshape(rows, L)
+    M = yh * (np.abs(gw) * yh).sum(axis=1, keepdims=True)
+    pu.assert_close(pu.widen(gin_g, dt), pu.widen(gin_o, dt), dt, "softmax grad_in", extra_mag=M)
+    return int(diff.sum())
+
+
+def _gelu_inputs(rows, L, dt, seed=0, scale=1.3):
+    n = rows * L
+    x = synth.to_io(synth.gelu_preact(seed, ("pg", rows, L, dt), n) * np.float32(scale), dt)
+    g = synth.to_io(synth.normal(seed, ("pgg", rows, L, dt), n), dt)
+    return x, g
+
+
+def _softmax_inputs(rows, L, dt, seed=0):
+    x = synth.to_io(synth.softmax_logits(seed, ("ps", rows, L, dt), rows, L), dt)
+    g = synth.to_io(synth.normal(seed, ("psg", rows, L, dt), rows * L), dt)
+    return x, g
+
+
+# ------------------------------------------------------------------ small shapes, tails
+GELU_SHAPES = [(5, 1), (3, 2), (7, 3), (9, 63), (64, 64), (33, 65), (41, 197), (12, 257), (37, 1024),
+               (40, 3072), (13, 3072), (11, 4096), (6, 5120), (3, 8191), (2, 8192), (1, 16384), (2, 40000)]
+SOFTMAX_SHAPES = [(7, 1), (4, 2), (5, 3), (33, 63), (77, 64), (1000, 64), (33, 65), (300, 197), (1, 197),
+                  (130, 257), (257, 257), (40, 1024), (9, 4096), (5, 8191), (3, 8192), (2, 40000)]
+
+
+@pytest.mark.parametrize("dt", [F32, BF16])
+@pytest.mark.parametrize("rows,L", GELU_SHAPES)
+def test_gelu_small(rows, L, dt):
+    check_gelu(*_gelu_inputs(rows, L, dt), L, dt)
+
+
+@pytest.mark.parametrize("dt", [F32, BF16])
+@pytest.mark.parametrize("rows,L", SOFTMAX_SHAPES)
+def test_softmax_small(rows, L, dt):
+    check_softmax(*_softmax_inputs(rows, L, dt), L, dt)
+
+
+@pytest.mark.parametrize("dt", [F32, BF16])
+def test_in_place(dt):
+    check_gelu(*_gelu_inputs(70, 3072, dt, seed=3), 3072, dt, inplace=True)
+    check_gelu(*_gelu_inputs(70, 197, dt, seed=3), 197, dt, inplace=True)
+    check_softmax(*_softmax_inputs(700, 197, dt, seed=3), 197, dt, inplace=True)
+    check_softmax(*_softmax_inputs(20, 4096, dt, seed=3), 4096, dt, inplace=True)
+
+
+# ------------------------------------------------------------------ degenerate inputs
+@pytest.mark.parametrize("dt", [F32, BF16])
+def test_degenerate_rows(dt):
+    L, rows = 197, 66
+    x = np.zeros((rows, L), dtype=np.float32)
+    x[1] = 0.37          # constant rows: max == min
+    x[2] = -5.0
+    x[3] = 7.0           # constant beyond the clip
+    x[4, ::2] = 1e4      # extreme magnitudes
+    x[4, 1::2] = -1e4
+    x[5] = np.linspace(-3, 3, L)
+    x[6, 0] = 2.0        # exactly on the clip
+    x[6, 1] = -2.0
+    x[7:] = synth.normal(1, "deg", (rows - 7) * L).reshape(rows - 7, L) * 0.05  # unsaturated rows
+    g = synth.normal(1, "degg", rows * L)
+    check_gelu(synth.to_io(x.reshape(-1), dt), synth.to_io(g, dt), L, dt)
+    xs = x.copy()
+    xs[4, ::2] = 80.0    # softmax: differences of 160 underflow to zero
+    xs[4, 1::2] = -80.0
+    xs[8] = 0.0
+    xs[8, 5] = 30.0      # one-hot row
+    check_softmax(synth.to_io(xs.reshape(-1), dt), synth.to_io(g, dt), L, dt)
+
+
+def test_gelu_saturated_row_hand_codes():
+    # bin edges of a [-2, 2] row; 0 is the exact tie 7.5 and must round to 8
+    row = np.array([-3, -2, -1, -0.1333333, 0, 0.1333334, 0.5, 1, 2, 2.5], dtype=np.float32)
+    y, codes, meta = pu.gpu_fwd("gelu", row, 10, F32)
+    assert pu.unpack_np(codes, 10).tolist() == [0, 0, 4, 7, 8, 8, 9, 11, 15, 15]
+    assert meta[0] == -2.0 and meta[1] == np.float32(np.float32(4) / np.float32(15))
+
+
+def test_softmax_worked_row():
+    x = np.array([0, 1, 2, 3], dtype=np.float32)
+    y, codes, meta = pu.gpu_fwd("softmax", x, 4, F32)
+    e = np.exp(np.arange(4.0))
+    assert np.allclose(y, e / e.sum(), rtol=1e-6)
+    assert codes.tolist() == [0x10, 0xF5]
+    gin = pu.gpu_bwd("softmax", np.array([1, -1, 0.5, 2], dtype=np.float32), codes, meta, 4, F32)
+    yh = np.array([0, 1, 5, 15]) * float(meta[1]) + float(meta[0])
+    dot = float(np.array([1, -1, 0.5, 2]) @ yh)
+    assert np.allclose(gin, yh * (np.array([1, -1, 0.5, 2]) - dot), rtol=2e-6)
+
+
+def test_empty_and_argument_errors():
+    L = binding.lib()
+    dev = torch.device("cuda")
+    x = torch.zeros(64, device=dev)
+    codes, meta = binding.alloc_stash(64, 8, dev)
+    s = torch.cuda.current_stream().cuda_stream
+    before = (x.clone(), codes.clone().fill_(7), meta.clone().fill_(3))
+    codes.fill_(7), meta.fill_(3)
+    args = lambda xp, yp, cp, mp, n, rl, dt: L.s2a_gelu_fwd(xp, yp, cp, mp, n, rl, dt, s)
+    assert args(x.data_ptr(), x.data_ptr(), codes.data_ptr(), meta.data_ptr(), 0, 8, 0) == 0      # empty
+    assert args(None, x.data_ptr(), codes.data_ptr(), meta.data_ptr(), 64, 8, 0) == 1               # NULL
+    assert args(x.data_ptr(), x.data_ptr(), codes.data_ptr(), meta.data_ptr(), 64, 0, 0) == 2       # row_len 0
+    assert args(x.data_ptr(), x.data_ptr(), codes.data_ptr(), meta.data_ptr(), 63, 8, 0) == 2       # ragged
+    assert args(x.data_ptr() + 4, x.data_ptr(), codes.data_ptr(), meta.data_ptr(), 32, 8, 0) == 3   # alignment
+    assert args(x.data_ptr(), x.data_ptr(), codes.data_ptr(), meta.data_ptr() + 4, 32, 8, 0) == 3
+    assert args(x.data_ptr(), x.data_ptr(), codes.data_ptr(), meta.data_ptr(), 64, 8, 7) == 4       # dtype
+    for f in (L.s2a_gelu_bwd, L.s2a_softmax_fwd, L.s2a_softmax_bwd):
+        assert f(x.data_ptr(), None, meta.data_ptr(), x.data_ptr(), 64, 8, 0, s) == 1
+    torch.cuda.synchronize()
+    assert torch.equal(x, before[0]) and torch.equal(codes, before[1]) and torch.equal(meta, before[2])
+    with pytest.raises(binding.S2AError):
+        binding.s2a_gelu_fwd(x.cpu(), x, codes, meta, 8)
+
+
+# ------------------------------------------------------------------ the named workloads
+def test_config1_single_gelu_layer_f32_full():
+    sh = synth.VIT_B16_B8_F32
+    x, g = synth.vit_gelu_inputs(sh, 0, 0)
+    assert x.size == 8 * 197 * 3072
+    check_gelu(x, g, sh.hidden, sh.dtype)
+
+
+@pytest.mark.parametrize("shape", [synth.VIT_B16_B64, synth.VIT_L16_B64, synth.VIT_H14_B32],
+                         ids=lambda s: s.name)
+def test_vit_block_full_size(shape):
+    """One block of each ViT workload at its full size, every element compared."""
+    x, g = synth.vit_gelu_inputs(shape, 0, 0)
+    assert x.size == shape.gelu_elems
+    check_gelu(x, g, shape.hidden, shape.dtype)
+    # every row of the bulk+tail input saturates the clip: per-row == per-tensor range
+    del x, g
+    x, g = synth.vit_softmax_inputs(shape, 0, 0)
+    assert x.size == shape.softmax_elems
+    flips = check_softmax(x, g, shape.tokens, shape.dtype)
+    print("%s: softmax edge flips vs oracle: %d of %d" % (shape.name, flips, x.size))
+
+
+def test_stash_bytes_are_half_a_byte_per_element_plus_row_metadata():
+    for sh in (synth.VIT_B16_B64, synth.VIT_L16_B64, synth.VIT_H14_B32):
+        total = 0
+        for n, L in ((sh.gelu_elems, sh.hidden), (sh.softmax_elems, sh.tokens)):
+            assert binding.codes_bytes(n) == (n + 1) // 2
+            assert binding.meta_bytes(n, L) == 8 * (n // L)
+            total += sh.blocks * (binding.codes_bytes(n) + binding.meta_bytes(n, L))
+        bf16_stash = sh.blocks * 2 * (sh.gelu_elems + sh.softmax_elems)
+        assert 3.8 < bf16_stash / total < 4.0
+        free, _ = torch.cuda.mem_get_info()
+        assert total < 0.02 * 180e9 and total < free
