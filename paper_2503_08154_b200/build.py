@@ -4,33 +4,52 @@ from __future__ import annotations
 import os
 import subprocess
 import sys
+from concurrent.futures import ThreadPoolExecutor
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
+OBJ = os.path.join(HERE, "_build")
 OUT = os.path.join(HERE, "libs2a.so")
-SOURCES = ["s2a_api.cu", "s2a_rowwise.cu", "s2a_tile.cu"]
-HEADERS = ["s2a_common.cuh", "s2a_launch.h", os.path.join("..", "..", "include", "s2a.h")]
+SOURCES = ["s2a_api.cu", "s2a_rowwise.cu", "s2a_tile.cu", "s2a_tile_gelu_fwd.cu",
+           "s2a_tile_gelu_bwd.cu", "s2a_tile_softmax_fwd.cu", "s2a_tile_softmax_bwd.cu"]
+HEADERS = ["s2a_common.cuh", "s2a_launch.h", "s2a_tile.cuh", os.path.join("..", "..", "include", "s2a.h")]
 
-NVCC_FLAGS = [
-    "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "-Xcompiler", "-fPIC", "-shared", "--threads", "4",
-]
+ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
+NVCC_FLAGS = [*ARCH, "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC"]
 
 
-def stale() -> bool:
-    if not os.path.exists(OUT):
+def _newer(deps, target) -> bool:
+    if not os.path.exists(target):
         return True
-    t = os.path.getmtime(OUT)
-    deps = [os.path.join(CSRC, f) for f in SOURCES + HEADERS] + [os.path.abspath(__file__)]
+    t = os.path.getmtime(target)
     return any(os.path.getmtime(d) > t for d in deps)
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
-    if force or stale():
-        nvcc = os.environ.get("NVCC", "nvcc")
-        cmd = [nvcc, *NVCC_FLAGS, *(["-Xptxas", "-v"] if verbose else []),
-               *[os.path.join(CSRC, f) for f in SOURCES], "-o", OUT + ".tmp"]
-        subprocess.run(cmd, check=True)
+    nvcc = os.environ.get("NVCC", "nvcc")
+    hdrs = [os.path.join(CSRC, h) for h in HEADERS] + [os.path.abspath(__file__)]
+    os.makedirs(OBJ, exist_ok=True)
+    jobs = []
+    for src in SOURCES:
+        path = os.path.join(CSRC, src)
+        obj = os.path.join(OBJ, src[:-3] + ".o")
+        if force or _newer([path, *hdrs], obj):
+            jobs.append([nvcc, *NVCC_FLAGS, *(["-Xptxas", "-v"] if verbose else []), "-c", path, "-o", obj])
+
+    def run(cmd):
+        r = subprocess.run(cmd, capture_output=True, text=True)
+        return cmd, r
+
+    if jobs:
+        with ThreadPoolExecutor(max_workers=min(len(jobs), os.cpu_count() or 1)) as pool:
+            for cmd, r in pool.map(run, jobs):
+                if verbose or r.returncode != 0:
+                    sys.stderr.write(r.stdout + r.stderr)
+                if r.returncode != 0:
+                    raise RuntimeError("nvcc failed: " + " ".join(cmd))
+    objs = [os.path.join(OBJ, s[:-3] + ".o") for s in SOURCES]
+    if jobs or _newer(objs, OUT):
+        subprocess.run([nvcc, *ARCH, "-shared", *objs, "-o", OUT + ".tmp"], check=True)
         os.replace(OUT + ".tmp", OUT)
     return OUT
 

@@ -32,7 +32,8 @@ int run(int kernel, const void* in, void* out, uint8_t* codes, float* meta, size
   const uint64_t n_rows = n / row_len;
   TilePlan p = plan_tile(kernel, dt, n_rows, (uint32_t)row_len);
   uint64_t done_rows = 0;
-  if (p.tile_rows != 0 && p.n_tiles != 0) {
+  // the pipelined path moves metadata with 16-byte bulk copies
+  if (p.tile_rows != 0 && p.n_tiles != 0 && !misaligned(meta, 16)) {
     TileArgs ta{in, out, codes, meta, (uint32_t)row_len, p.n_tiles};
     if (launch_tile(kernel, dt, p, ta, st) != cudaSuccess) return S2A_ERR_CUDA;
     done_rows = p.n_tiles * p.tile_rows;

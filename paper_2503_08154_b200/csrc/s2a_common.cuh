@@ -72,13 +72,15 @@ __device__ __forceinline__ float dequant(uint32_t code, float mn, float s) {
 }
 
 // ---------------------------------------------------------------- Eq. 10 and Eq. 12
-// y = x / (1 + exp(-1.702 x)).  The product 1.702 x is carried as hi + lo so that its
-// rounding does not scale the error of exp with |x|.
+// y = x * sigmoid(1.702 x), evaluated through t = exp(-|1.702 x|) so that neither tail
+// overflows: sigmoid(z) = 1 / (1 + t) for z >= 0 and t / (1 + t) for z < 0.  The
+// product 1.702 x is carried as hi + lo so that its rounding does not scale the error
+// of exp with |x|.
 __device__ __forceinline__ float gelu_value(float x) {
   float z = __fmul_rn(kSlope, x);
   float zlo = __fmaf_rn(kSlope, x, -z);
-  float e = expf(-z) * (1.0f - zlo);  // exp(-(z + zlo)); stays inf when exp overflows
-  return __fdiv_rn(x, 1.0f + e);
+  float t = expf(-fabsf(z)) * (1.0f - (z >= 0.0f ? zlo : -zlo));
+  return __fdiv_rn(z >= 0.0f ? x : x * t, 1.0f + t);
 }
 
 // Eq. 12 at a dequantised x_hat = code * s + min, in binary64.

@@ -1,14 +1,181 @@
-// Pipelined tile kernels (placeholder: no shape is planned onto this path yet).
-#include "s2a_common.cuh"
-#include "s2a_launch.h"
+// Host side of the pipelined tile path: launch-shape policy, argument packing, the
+// per-device error word.
+#include "s2a_tile.cuh"
+
+#include <stdlib.h>
 
 namespace s2a {
 
 __device__ unsigned int g_error_word = 0;
 
-TilePlan plan_tile(int, int, uint64_t, uint32_t) { return TilePlan{}; }
+cudaError_t launch_tile_gelu_fwd(int dt, const TilePlan& p, const void* kernel_args, cudaStream_t st);
+cudaError_t launch_tile_gelu_bwd(int dt, const TilePlan& p, const void* kernel_args, cudaStream_t st);
+cudaError_t launch_tile_softmax_fwd(int dt, const TilePlan& p, const void* kernel_args, cudaStream_t st);
+cudaError_t launch_tile_softmax_bwd(int dt, const TilePlan& p, const void* kernel_args, cudaStream_t st);
 
-cudaError_t launch_tile(int, int, const TilePlan&, const TileArgs&, cudaStream_t) {
+namespace {
+
+constexpr uint32_t kMaxStageBytes = 56 * 1024;
+
+int env_int(const char* name, int dflt) {
+  const char* v = getenv(name);
+  return (v && *v) ? atoi(v) : dflt;
+}
+
+uint32_t gcd_u32(uint32_t a, uint32_t b) {
+  while (b) { uint32_t t = a % b; a = b; b = t; }
+  return a;
+}
+
+uint32_t align_up(uint32_t v, uint32_t a) { return (v + a - 1) / a * a; }
+
+int sm_count() {
+  static int cached = 0;
+  if (cached == 0) {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
+      cached = n;
+    else
+      return 148;  // no device visible (planning on a build host): assume a B200
+  }
+  return cached;
+}
+
+
+unsigned int* error_word_address() {
+  // one address per device; looked up on first use with that device current
+  static unsigned int* addr[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  if (!addr[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_error_word) != cudaSuccess) return nullptr;
+    addr[dev] = (unsigned int*)p;
+  }
+  return addr[dev];
+}
+
+}  // namespace
+
+// Launch-shape policy.  Environment overrides (for tuning sweeps): S2A_PATH=rowwise
+// disables this path; S2A_UNIT, S2A_TILE_ROWS, S2A_WARPS, S2A_STAGES, S2A_CTAS_PER_SM.
+TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L) {
+  TilePlan p{};
+  const char* path = getenv("S2A_PATH");
+  if (path && path[0] == 'r') return p;
+  const uint32_t esize = dt == kF32 ? 4u : 2u;
+  const uint32_t vec = 16u / esize;                 // elements per 16-byte access
+  const bool vec16 = (L % vec) == 0;
+  const uint32_t epa = vec16 ? vec : 2u;
+  const uint32_t n_acc = vec16 ? L / vec : (L + 1) / 2;  // accesses covering one row
+  // rows per tile: the tile's element count must be a multiple of 32, its row count even
+  uint32_t r_min = 32u / gcd_u32(L, 32u);
+  if (r_min < 2) r_min = 2;
+  const uint64_t min_tile_bytes = (uint64_t)r_min * L * esize;
+  if (min_tile_bytes > kMaxStageBytes) return p;
+
+  // lanes per row: the smallest unit that keeps a lane at or under ~32 elements, else
+  // the largest unit with up to 16 accesses per lane
+  const uint32_t cap_iters = 32u / epa > 16u ? 16u : 32u / epa;  // vec16 bf16: 4, f32: 8, pair: 16
+  const uint32_t max_iters = (dt == kBF16 && vec16) ? 8u : 16u;  // what is instantiated
+  const uint32_t units[4] = {8, 16, 32, 128};
+  uint32_t unit = 0, need = 0;
+  for (int k = 0; k < 4 && unit == 0; ++k) {
+    need = (n_acc + units[k] - 1) / units[k];
+    if (need <= cap_iters) unit = units[k];
+  }
+  if (unit == 0) {
+    need = (n_acc + 127) / 128;
+    if (need > max_iters) return p;
+    unit = 128;
+  }
+  unit = (uint32_t)env_int("S2A_UNIT", (int)unit);
+  if (unit != 8 && unit != 16 && unit != 32 && unit != 128) return p;
+  need = (n_acc + unit - 1) / unit;
+  if (need > max_iters) return p;
+  uint32_t iters = 1;
+  while (iters < need) iters *= 2;
+
+  uint32_t warps = unit == 128 ? 8u : 4u;
+  warps = (uint32_t)env_int("S2A_WARPS", (int)warps);
+  if (warps < 1 || warps > 8 || (warps * 32) % unit != 0) return p;
+  const uint32_t n_units = warps * 32 / unit;
+  const uint32_t G = (!vec16 && (L & 1u)) ? 2u : 1u;
+
+  // tile rows: a multiple of r_min that gives every unit a row (pair) per round, within
+  // the stage budget; prefer ~16 KiB of data per tile
+  uint32_t rows = r_min;
+  const uint32_t want_rows = n_units * G;
+  while (rows % want_rows != 0 && (uint64_t)(rows + r_min) * L * esize <= kMaxStageBytes) rows += r_min;
+  while ((uint64_t)rows * L * esize < 16 * 1024 && (uint64_t)rows * 2 * L * esize <= kMaxStageBytes) rows *= 2;
+  rows = (uint32_t)env_int("S2A_TILE_ROWS", (int)rows);
+  if (rows == 0 || rows % r_min != 0 || (uint64_t)rows * L * esize > kMaxStageBytes) return p;
+
+  const uint32_t data_bytes = rows * L * esize;
+  const uint32_t code_bytes = rows * L / 2;
+  const uint32_t meta_bytes = rows * 8;
+  const uint32_t code_off = align_up(data_bytes, 128);
+  const uint32_t meta_off = code_off + align_up(code_bytes, 128);
+  const uint32_t stage_bytes = meta_off + align_up(meta_bytes, 128);
+
+  int ctas_per_sm = env_int("S2A_CTAS_PER_SM", 2);
+  if (ctas_per_sm < 1) ctas_per_sm = 1;
+  uint32_t budget = kMaxSmem / (uint32_t)ctas_per_sm - 1024;
+  uint32_t stages = (budget - kHeaderBytes) / stage_bytes;
+  if (stages > 4) stages = 4;
+  stages = (uint32_t)env_int("S2A_STAGES", (int)stages);
+  if (stages > (uint32_t)kMaxStages) stages = kMaxStages;
+  if (stages < 2) {
+    ctas_per_sm = 1;
+    stages = (kMaxSmem - kHeaderBytes) / stage_bytes;
+    if (stages > 4) stages = 4;
+    if (stages < 2) return p;
+  }
+  const uint32_t smem = kHeaderBytes + stages * stage_bytes;
+  if (smem > kMaxSmem) return p;
+
+  p.n_tiles = n_rows / rows;
+  if (p.n_tiles == 0) return TilePlan{};
+  p.tile_rows = rows;
+  p.unit_lanes = unit;
+  p.vec_elems = epa;
+  p.iters = iters;
+  p.warps = warps;
+  p.stages = stages;
+  p.smem_bytes = smem;
+  uint64_t grid = (uint64_t)sm_count() * (uint32_t)ctas_per_sm;
+  if (grid > p.n_tiles) grid = p.n_tiles;
+  p.grid = (uint32_t)grid;
+  (void)kernel;
+  return p;
+}
+
+cudaError_t launch_tile(int kernel, int dt, const TilePlan& p, const TileArgs& a, cudaStream_t st) {
+  TileKernelArgs ka;
+  ka.in = (const unsigned char*)a.in;
+  ka.out = (unsigned char*)a.out;
+  ka.codes = a.codes;
+  ka.meta = (unsigned char*)a.meta;
+  ka.n_tiles = a.n_tiles;
+  ka.row_len = a.row_len;
+  ka.tile_rows = p.tile_rows;
+  const uint32_t esize = dt == kF32 ? 4u : 2u;
+  ka.data_bytes = p.tile_rows * a.row_len * esize;
+  ka.code_bytes = p.tile_rows * a.row_len / 2;
+  ka.meta_bytes = p.tile_rows * 8;
+  ka.code_off = align_up(ka.data_bytes, 128);
+  ka.meta_off = ka.code_off + align_up(ka.code_bytes, 128);
+  ka.stage_bytes = ka.meta_off + align_up(ka.meta_bytes, 128);
+  ka.stages = p.stages;
+  ka.error_word = error_word_address();
+  if (!ka.error_word) return cudaErrorInvalidDevice;
+  switch (kernel) {
+    case kGeluFwd: return launch_tile_gelu_fwd(dt, p, &ka, st);
+    case kGeluBwd: return launch_tile_gelu_bwd(dt, p, &ka, st);
+    case kSoftmaxFwd: return launch_tile_softmax_fwd(dt, p, &ka, st);
+    case kSoftmaxBwd: return launch_tile_softmax_bwd(dt, p, &ka, st);
+  }
   return cudaErrorInvalidValue;
 }
 

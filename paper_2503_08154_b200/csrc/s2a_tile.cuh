@@ -1,0 +1,705 @@
+// Pipelined tile kernels: the bandwidth path of all four S2A entry points.
+//
+// A persistent CTA walks tiles of `tile_rows` consecutive rows.  One extra warp moves
+// whole tiles between HBM and shared memory with bulk asynchronous copies (the TMA
+// engine, no multicast): loads complete on a "full" mbarrier per stage, the consumer
+// warps rewrite the tile in place in shared memory (x -> y, grad_out -> grad_in) and
+// produce or consume the packed codes and the per-row (min, s), signal a "done"
+// mbarrier, and the copy warp streams the results back out and refills the stage.
+// Memory-level parallelism therefore comes from the copy engine, not from registers or
+// occupancy, and rows of any alignment are handled because a tile always starts and
+// ends on a multiple of 32 elements (16-byte aligned data AND code bytes).
+//
+// Inside a tile a "unit" of 8, 16, 32 or 128 lanes owns one row at a time and keeps it
+// in registers; row reductions are warp shuffles (plus one shared-memory hop for
+// 128-lane units).  Rows are read as 16-byte vectors when row_len allows it and
+// otherwise as 2-element words on the tile's even-element grid, where a row of odd
+// length shares its first or last word (and code byte) with its neighbour: the two rows
+// of such a pair are handled back to back by the same unit.
+//
+// Every wait on an mbarrier is bounded; a wait that runs out sets a bit in the
+// per-device error word and the CTA winds down.
+#pragma once
+#include "s2a_common.cuh"
+#include "s2a_launch.h"
+
+namespace s2a {
+namespace {
+
+constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr int kMaxStages = 8;
+constexpr int kHeaderBytes = 4096;  // barriers, reduction scratch, derivative tables
+constexpr int kRedOffset = 256;     // float[2 slots][4 units][4 warps]  (multi-warp units)
+constexpr int kFlagOffset = 768;    // int[4]: abort flag per multi-warp unit
+constexpr int kTabOffset = 1024;    // float[units][16]: Eq. 12 table per unit (<= 32 units)
+
+enum { kVec16 = 0, kPair = 1 };
+
+struct TileKernelArgs {
+  const unsigned char* in;
+  unsigned char* out;
+  unsigned char* codes;
+  unsigned char* meta;
+  uint64_t n_tiles;
+  uint32_t row_len;
+  uint32_t tile_rows;
+  uint32_t data_bytes;   // per tile
+  uint32_t code_bytes;   // per tile
+  uint32_t meta_bytes;   // per tile
+  uint32_t code_off;     // offsets inside a stage
+  uint32_t meta_off;
+  uint32_t stage_bytes;
+  uint32_t stages;
+  unsigned int* error_word;  // device address of the per-device error word
+};
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)),
+               "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait for the phase with the given parity to complete.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned int* err, unsigned err_bit) {
+  for (uint32_t i = 0; i < kSpinLimit; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  atomicOr(err, err_bit);
+  return false;
+}
+__device__ __forceinline__ void fence_barrier_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+// global -> shared bulk copy; completion is counted in bytes on `bar`.
+__device__ __forceinline__ void bulk_load(void* dst_smem, const void* src, uint32_t bytes,
+                                          uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::
+          "r"(smem_u32(dst_smem)),
+      "l"(src), "r"(bytes), "r"(smem_u32(bar))
+      : "memory");
+}
+// shared -> global bulk copy, tracked by the thread's bulk-group.
+__device__ __forceinline__ void bulk_store(void* dst, const void* src_smem, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst),
+               "r"(smem_u32(src_smem)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() {
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() {
+  asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+__device__ __forceinline__ void named_bar_sync(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
+// ---------------------------------------------------------------- shared-memory access
+// One "access" is what a lane reads or writes at a time: EPA elements and the code
+// bytes that belong to them.
+template <int DT, int VMODE> struct Acc;
+
+template <> struct Acc<kBF16, kVec16> {
+  static constexpr int EPA = 8;
+  using Raw = uint4;
+  static __device__ __forceinline__ Raw load(const unsigned char* d, uint32_t a) {
+    return *(const uint4*)(d + (size_t)a * 16);
+  }
+  static __device__ __forceinline__ void widen(const Raw& r, float* v) {
+    const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      v[2 * k] = __uint_as_float(w[k] << 16);
+      v[2 * k + 1] = __uint_as_float(w[k] & 0xffff0000u);
+    }
+  }
+  // Rounds to the I/O type, stores, and leaves in v the values as written.
+  static __device__ __forceinline__ void narrow_store(unsigned char* d, uint32_t a, float* v, int) {
+    uint32_t w[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      __nv_bfloat162 b = __floats2bfloat162_rn(v[2 * k], v[2 * k + 1]);
+      w[k] = *(uint32_t*)&b;
+      v[2 * k] = __uint_as_float(w[k] << 16);
+      v[2 * k + 1] = __uint_as_float(w[k] & 0xffff0000u);
+    }
+    *(uint4*)(d + (size_t)a * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+  static __device__ __forceinline__ uint32_t load_codes(const unsigned char* c, uint32_t a) {
+    return *(const uint32_t*)(c + (size_t)a * 4);
+  }
+  static __device__ __forceinline__ void store_codes(unsigned char* c, uint32_t a, uint32_t bits) {
+    *(uint32_t*)(c + (size_t)a * 4) = bits;
+  }
+};
+
+template <> struct Acc<kF32, kVec16> {
+  static constexpr int EPA = 4;
+  using Raw = float4;
+  static __device__ __forceinline__ Raw load(const unsigned char* d, uint32_t a) {
+    return *(const float4*)(d + (size_t)a * 16);
+  }
+  static __device__ __forceinline__ void widen(const Raw& r, float* v) {
+    v[0] = r.x; v[1] = r.y; v[2] = r.z; v[3] = r.w;
+  }
+  static __device__ __forceinline__ void narrow_store(unsigned char* d, uint32_t a, float* v, int) {
+    *(float4*)(d + (size_t)a * 16) = make_float4(v[0], v[1], v[2], v[3]);
+  }
+  static __device__ __forceinline__ uint32_t load_codes(const unsigned char* c, uint32_t a) {
+    return *(const uint16_t*)(c + (size_t)a * 2);
+  }
+  static __device__ __forceinline__ void store_codes(unsigned char* c, uint32_t a, uint32_t bits) {
+    *(uint16_t*)(c + (size_t)a * 2) = (uint16_t)bits;
+  }
+};
+
+// Pair mode: `keep` says which of the two elements belong to the row (bit 0: low,
+// bit 1: high); the other half of a shared word is left untouched.
+template <> struct Acc<kBF16, kPair> {
+  static constexpr int EPA = 2;
+  using Raw = uint32_t;
+  static __device__ __forceinline__ Raw load(const unsigned char* d, uint32_t a) {
+    return *(const uint32_t*)(d + (size_t)a * 4);
+  }
+  static __device__ __forceinline__ void widen(const Raw& r, float* v) {
+    v[0] = __uint_as_float(r << 16);
+    v[1] = __uint_as_float(r & 0xffff0000u);
+  }
+  static __device__ __forceinline__ void narrow_store(unsigned char* d, uint32_t a, float* v, int keep) {
+    __nv_bfloat162 b = __floats2bfloat162_rn(v[0], v[1]);
+    uint32_t w = *(uint32_t*)&b;
+    v[0] = __uint_as_float(w << 16);
+    v[1] = __uint_as_float(w & 0xffff0000u);
+    if (keep == 3) *(uint32_t*)(d + (size_t)a * 4) = w;
+    else if (keep == 1) *(uint16_t*)(d + (size_t)a * 4) = (uint16_t)w;
+    else if (keep == 2) *(uint16_t*)(d + (size_t)a * 4 + 2) = (uint16_t)(w >> 16);
+  }
+  static __device__ __forceinline__ uint32_t load_codes(const unsigned char* c, uint32_t a) {
+    return c[a];
+  }
+  static __device__ __forceinline__ void store_codes(unsigned char* c, uint32_t a, uint32_t bits) {
+    c[a] = (unsigned char)bits;
+  }
+};
+
+template <> struct Acc<kF32, kPair> {
+  static constexpr int EPA = 2;
+  using Raw = float2;
+  static __device__ __forceinline__ Raw load(const unsigned char* d, uint32_t a) {
+    return *(const float2*)(d + (size_t)a * 8);
+  }
+  static __device__ __forceinline__ void widen(const Raw& r, float* v) {
+    v[0] = r.x; v[1] = r.y;
+  }
+  static __device__ __forceinline__ void narrow_store(unsigned char* d, uint32_t a, float* v, int keep) {
+    if (keep == 3) *(float2*)(d + (size_t)a * 8) = make_float2(v[0], v[1]);
+    else if (keep == 1) *(float*)(d + (size_t)a * 8) = v[0];
+    else if (keep == 2) *(float*)(d + (size_t)a * 8 + 4) = v[1];
+  }
+  static __device__ __forceinline__ uint32_t load_codes(const unsigned char* c, uint32_t a) {
+    return c[a];
+  }
+  static __device__ __forceinline__ void store_codes(unsigned char* c, uint32_t a, uint32_t bits) {
+    c[a] = (unsigned char)bits;
+  }
+};
+
+// ---------------------------------------------------------------- units
+enum { kOpMax = 0, kOpMin = 1, kOpSum = 2 };
+
+template <int OP>
+__device__ __forceinline__ float op2(float a, float b) {
+  return OP == kOpMax ? fmaxf(a, b) : (OP == kOpMin ? fminf(a, b) : a + b);
+}
+
+template <int UNIT>
+struct Unit {
+  int ul;       // lane within the unit
+  int uid;      // unit within the CTA
+  float* red;   // reduction scratch of this unit (multi-warp units only)
+  int phase;
+
+  template <int OP>
+  __device__ __forceinline__ float reduce(float v) {
+    constexpr int W = UNIT < 32 ? UNIT : 32;
+#pragma unroll
+    for (int o = W / 2; o > 0; o >>= 1) v = op2<OP>(v, __shfl_xor_sync(0xffffffffu, v, o));
+    if (UNIT > 32) {
+      constexpr int NW = UNIT / 32;
+      float* slot = red + (phase & 1) * 16;
+      if ((ul & 31) == 0) slot[ul >> 5] = v;
+      named_bar_sync(1 + uid, UNIT);
+      v = slot[0];
+#pragma unroll
+      for (int k = 1; k < NW; ++k) v = op2<OP>(v, slot[k]);
+      ++phase;
+    }
+    return v;
+  }
+  // Orders shared-memory accesses of the unit's lanes (and keeps them in step).
+  __device__ __forceinline__ void sync() {
+    if (UNIT > 32) named_bar_sync(1 + uid, UNIT);
+    else __syncwarp();
+  }
+};
+
+// Geometry of one row inside a tile, in accesses.
+struct RowGeom {
+  uint32_t a0;    // first access (tile-relative)
+  uint32_t n_acc; // accesses covering the row
+  bool head;      // pair mode: low element of the first access belongs to the previous row
+  bool tail;      // pair mode: high element of the last access belongs to the next row
+};
+
+template <int DT, int VMODE>
+__device__ __forceinline__ RowGeom row_geom(uint32_t r, uint32_t L) {
+  RowGeom g;
+  if (VMODE == kVec16) {
+    constexpr int EPA = Acc<DT, VMODE>::EPA;
+    g.n_acc = L / EPA;
+    g.a0 = r * g.n_acc;
+    g.head = false;
+    g.tail = false;
+  } else {
+    uint32_t e0 = r * L;
+    g.a0 = e0 >> 1;
+    g.n_acc = ((e0 + L - 1) >> 1) - g.a0 + 1;
+    g.head = (e0 & 1u) != 0;
+    g.tail = ((e0 + L) & 1u) != 0;
+  }
+  return g;
+}
+
+// Fast sigmoid-GELU pieces for the bfloat16 path (result is rounded to 8 bits).
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float rcp_approx(float x) {
+  float y;
+  asm("rcp.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+template <int DT>
+__device__ __forceinline__ float gelu_eval(float x) {
+  if (DT == kF32) return gelu_value(x);
+  // t = exp(-|1.702 x|); y = (z >= 0 ? x : x t) / (1 + t)
+  const float z = kSlope * x;
+  const float t = ex2_approx(-1.4426950408889634f * fabsf(z));
+  const float num = z >= 0.0f ? x : x * t;
+  return num * rcp_approx(1.0f + t);
+}
+
+template <int DT>
+__device__ __forceinline__ float exp_eval(float d) {  // d <= 0
+  if (DT == kF32) return expf(d);
+  return ex2_approx(1.4426950408889634f * d);
+}
+
+// ---------------------------------------------------------------- per-row work
+// All lanes of a unit call these together.  `active` is false for a unit that has no
+// row in this round; it still takes part in the reductions.
+template <int KERNEL, int DT, int VMODE, int UNIT, int ITERS>
+struct RowWork {
+  using A = Acc<DT, VMODE>;
+  static constexpr int EPA = A::EPA;
+
+  // Which elements of access i belong to the row (bit k = element k); 0 if none.
+  static __device__ __forceinline__ uint32_t keep_mask(const RowGeom& g, uint32_t idx, bool active) {
+    if (!active || idx >= g.n_acc) return 0u;
+    uint32_t m = (1u << EPA) - 1u;
+    if (VMODE == kPair) {
+      if (g.head && idx == 0) m &= ~1u;
+      if (g.tail && idx == g.n_acc - 1) m &= ~2u;
+    }
+    return m;
+  }
+
+  static __device__ __forceinline__ void gelu_fwd(Unit<UNIT>& u, unsigned char* data, unsigned char* codes,
+                                                  float* meta_s, uint32_t r, uint32_t L, bool active) {
+    const RowGeom g = row_geom<DT, VMODE>(r, L);
+    typename A::Raw raw[ITERS];
+    float mn = INFINITY, mx = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < ITERS; ++i) {
+      const uint32_t idx = u.ul + UNIT * i;
+      const uint32_t keep = keep_mask(g, idx, active);
+      if (keep) {
+        raw[i] = A::load(data, g.a0 + idx);
+        float v[EPA];
+        A::widen(raw[i], v);
+#pragma unroll
+        for (int k = 0; k < EPA; ++k)
+          if (keep >> k & 1) { mn = fminf(mn, v[k]); mx = fmaxf(mx, v[k]); }
+      }
+    }
+    mn = u.template reduce<kOpMin>(mn);
+    mx = u.template reduce<kOpMax>(mx);
+    const QRange q = make_qrange(fminf(fmaxf(mn, -kClip), kClip), fminf(fmaxf(mx, -kClip), kClip));
+    if (active && u.ul == 0) { meta_s[2 * r] = q.mn; meta_s[2 * r + 1] = q.s; }
+#pragma unroll
+    for (int i = 0; i < ITERS; ++i) {
+      const uint32_t idx = u.ul + UNIT * i;
+      const uint32_t keep = keep_mask(g, idx, active);
+      if (keep) {
+        float v[EPA];
+        A::widen(raw[i], v);
+        uint32_t bits = 0;
+#pragma unroll
+        for (int k = 0; k < EPA; ++k) {
+          if (keep >> k & 1) bits |= quant_code(fminf(fmaxf(v[k], -kClip), kClip), q) << (4 * k);
+          v[k] = gelu_eval<DT>(v[k]);
+        }
+        if (VMODE == kPair && !(keep & 1)) bits |= A::load_codes(codes, g.a0 + idx) & 0xFu;
+        A::narrow_store(data, g.a0 + idx, v, (int)keep);
+        A::store_codes(codes, g.a0 + idx, bits);
+      }
+    }
+  }
+
+  static __device__ __forceinline__ void softmax_fwd(Unit<UNIT>& u, unsigned char* data, unsigned char* codes,
+                                                     float* meta_s, uint32_t r, uint32_t L, bool active) {
+    const RowGeom g = row_geom<DT, VMODE>(r, L);
+    float e[ITERS][EPA];
+    float m = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < ITERS; ++i) {
+      const uint32_t idx = u.ul + UNIT * i;
+      const uint32_t keep = keep_mask(g, idx, active);
+#pragma unroll
+      for (int k = 0; k < EPA; ++k) e[i][k] = -INFINITY;
+      if (keep) {
+        float v[EPA];
+        A::widen(A::load(data, g.a0 + idx), v);
+#pragma unroll
+        for (int k = 0; k < EPA; ++k)
+          if (keep >> k & 1) { e[i][k] = v[k]; m = fmaxf(m, v[k]); }
+      }
+    }
+    m = u.template reduce<kOpMax>(m);
+    if (!active) m = 0.0f;
+    float z = 0.0f;
+#pragma unroll
+    for (int i = 0; i < ITERS; ++i)
+#pragma unroll
+      for (int k = 0; k < EPA; ++k) {
+        e[i][k] = exp_eval<DT>(e[i][k] - m);  // elements outside the row: exp(-inf) = 0
+        z += e[i][k];
+      }
+    z = u.template reduce<kOpSum>(z);
+    const float rz = __fdiv_rn(1.0f, active ? z : 1.0f);
+    float mn = INFINITY, mx = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < ITERS; ++i) {
+      const uint32_t idx = u.ul + UNIT * i;
+      const uint32_t keep = keep_mask(g, idx, active);
+      if (keep) {
+#pragma unroll
+        for (int k = 0; k < EPA; ++k) e[i][k] *= rz;
+        A::narrow_store(data, g.a0 + idx, e[i], (int)keep);  // e now holds y as written
+#pragma unroll
+        for (int k = 0; k < EPA; ++k)
+          if (keep >> k & 1) { mn = fminf(mn, e[i][k]); mx = fmaxf(mx, e[i][k]); }
+      }
+    }
+    mn = u.template reduce<kOpMin>(mn);
+    mx = u.template reduce<kOpMax>(mx);
+    const QRange q = make_qrange(mn, mx);
+    if (active && u.ul == 0) { meta_s[2 * r] = q.mn; meta_s[2 * r + 1] = q.s; }
+#pragma unroll
+    for (int i = 0; i < ITERS; ++i) {
+      const uint32_t idx = u.ul + UNIT * i;
+      const uint32_t keep = keep_mask(g, idx, active);
+      if (keep) {
+        uint32_t bits = 0;
+#pragma unroll
+        for (int k = 0; k < EPA; ++k)
+          if (keep >> k & 1) bits |= quant_code(e[i][k], q) << (4 * k);
+        if (VMODE == kPair && !(keep & 1)) bits |= A::load_codes(codes, g.a0 + idx) & 0xFu;
+        A::store_codes(codes, g.a0 + idx, bits);
+      }
+    }
+  }
+
+  static __device__ __forceinline__ void gelu_bwd(Unit<UNIT>& u, unsigned char* data, const unsigned char* codes,
+                                                  const float* meta_s, float* tab, float& tab_mn, float& tab_s,
+                                                  uint32_t r, uint32_t L, bool active) {
+    const RowGeom g = row_geom<DT, VMODE>(r, L);
+    const float mn = active ? meta_s[2 * r] : tab_mn;
+    const float s = active ? meta_s[2 * r + 1] : tab_s;
+    // The 16 values of Eq. 12 this row can take, in binary64; kept while (min, s) repeat.
+    if (mn != tab_mn || s != tab_s) {
+#pragma unroll
+      for (int c = 0; c < 16; c += (UNIT < 16 ? UNIT : 16)) {
+        const int code = c + u.ul;
+        if (u.ul < 16 && code < 16) tab[code] = (float)gelu_sine_derivative((uint32_t)code, mn, s);
+      }
+      tab_mn = mn;
+      tab_s = s;
+    }
+    u.sync();
+#pragma unroll
+    for (int i = 0; i < ITERS; ++i) {
+      const uint32_t idx = u.ul + UNIT * i;
+      const uint32_t keep = keep_mask(g, idx, active);
+      if (keep) {
+        float v[EPA];
+        A::widen(A::load(data, g.a0 + idx), v);
+        const uint32_t bits = A::load_codes(codes, g.a0 + idx);
+#pragma unroll
+        for (int k = 0; k < EPA; ++k) v[k] *= tab[(bits >> (4 * k)) & 0xFu];
+        A::narrow_store(data, g.a0 + idx, v, (int)keep);
+      }
+    }
+  }
+
+  static __device__ __forceinline__ void softmax_bwd(Unit<UNIT>& u, unsigned char* data, const unsigned char* codes,
+                                                     const float* meta_s, uint32_t r, uint32_t L, bool active) {
+    const RowGeom g = row_geom<DT, VMODE>(r, L);
+    const float mn = active ? meta_s[2 * r] : 0.0f;
+    const float s = active ? meta_s[2 * r + 1] : 0.0f;
+    float gv[ITERS][EPA], yh[ITERS][EPA];
+    float dot = 0.0f;
+#pragma unroll
+    for (int i = 0; i < ITERS; ++i) {
+      const uint32_t idx = u.ul + UNIT * i;
+      const uint32_t keep = keep_mask(g, idx, active);
+      if (keep) {
+        A::widen(A::load(data, g.a0 + idx), gv[i]);
+        const uint32_t bits = A::load_codes(codes, g.a0 + idx);
+#pragma unroll
+        for (int k = 0; k < EPA; ++k) {
+          yh[i][k] = dequant((bits >> (4 * k)) & 0xFu, mn, s);
+          if (keep >> k & 1) dot = fmaf(gv[i][k], yh[i][k], dot);
+        }
+      }
+    }
+    dot = u.template reduce<kOpSum>(dot);
+#pragma unroll
+    for (int i = 0; i < ITERS; ++i) {
+      const uint32_t idx = u.ul + UNIT * i;
+      const uint32_t keep = keep_mask(g, idx, active);
+      if (keep) {
+        float v[EPA];
+#pragma unroll
+        for (int k = 0; k < EPA; ++k) v[k] = yh[i][k] * (gv[i][k] - dot);
+        A::narrow_store(data, g.a0 + idx, v, (int)keep);
+      }
+    }
+  }
+};
+
+// ---------------------------------------------------------------- the kernel
+template <int KERNEL, int DT, int VMODE, int UNIT, int ITERS>
+__global__ void __launch_bounds__(288) tile_kernel(TileKernelArgs a) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  constexpr bool kFwd = (KERNEL == kGeluFwd || KERNEL == kSoftmaxFwd);
+
+  uint64_t* full = (uint64_t*)smem;                 // [stages]
+  uint64_t* done = (uint64_t*)smem + kMaxStages;    // [stages]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_cwarps = (blockDim.x >> 5) - 1;
+  const uint32_t S = a.stages;
+  const uint64_t my_tiles =
+      a.n_tiles > blockIdx.x ? (a.n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+
+  if (threadIdx.x == 0) {
+    for (uint32_t s = 0; s < S; ++s) {
+      mbar_init(&full[s], 1);
+      mbar_init(&done[s], (uint32_t)n_cwarps);
+    }
+    int* flags = (int*)(smem + kFlagOffset);
+    for (int k = 0; k < 4; ++k) flags[k] = 0;
+    fence_barrier_init();
+  }
+  __syncthreads();
+
+  if (warp == n_cwarps) {
+    // ------------------------------------------------------------ copy warp
+    if (lane != 0) return;
+    auto stage_ptr = [&](uint64_t it) { return smem + kHeaderBytes + (size_t)(it % S) * a.stage_bytes; };
+    auto issue_load = [&](uint64_t it) {
+      const uint64_t t = blockIdx.x + it * gridDim.x;
+      unsigned char* st = stage_ptr(it);
+      uint64_t* bar = &full[it % S];
+      const uint32_t bytes = kFwd ? a.data_bytes : a.data_bytes + a.code_bytes + a.meta_bytes;
+      mbar_arrive_expect_tx(bar, bytes);
+      bulk_load(st, a.in + t * a.data_bytes, a.data_bytes, bar);
+      if (!kFwd) {
+        bulk_load(st + a.code_off, a.codes + t * a.code_bytes, a.code_bytes, bar);
+        bulk_load(st + a.meta_off, a.meta + t * a.meta_bytes, a.meta_bytes, bar);
+      }
+    };
+    const uint64_t pre = my_tiles < S ? my_tiles : S;
+    for (uint64_t it = 0; it < pre; ++it) issue_load(it);
+    uint64_t issued = pre;
+    uint64_t it = 0;
+    bool ok = true;
+    for (; it < my_tiles; ++it) {
+      if (!mbar_wait(&done[it % S], (uint32_t)((it / S) & 1), a.error_word, kErrDrainWait)) { ok = false; break; }
+      const uint64_t t = blockIdx.x + it * gridDim.x;
+      unsigned char* st = stage_ptr(it);
+      bulk_store(a.out + t * a.data_bytes, st, a.data_bytes);
+      if (kFwd) {
+        bulk_store(a.codes + t * a.code_bytes, st + a.code_off, a.code_bytes);
+        bulk_store(a.meta + t * a.meta_bytes, st + a.meta_off, a.meta_bytes);
+      }
+      bulk_commit();
+      if (it >= 1 && issued < my_tiles) {
+        bulk_wait_read<1>();  // the stores of tile it-1 have left shared memory
+        issue_load(issued);   // == it - 1 + S: refills the stage of tile it-1
+        ++issued;
+      }
+    }
+    bulk_wait_all();
+    if (!ok) {
+      // wind down: let every load already issued land before shared memory is released
+      for (uint64_t j = it; j < issued; ++j)
+        mbar_wait(&full[j % S], (uint32_t)((j / S) & 1), a.error_word, kErrLoadWait);
+    }
+    return;
+  }
+
+  // -------------------------------------------------------------- consumer warps
+  using W = RowWork<KERNEL, DT, VMODE, UNIT, ITERS>;
+  const int ctid = threadIdx.x;  // consumer warps come first
+  Unit<UNIT> u;
+  u.ul = ctid % UNIT;
+  u.uid = ctid / UNIT;
+  u.red = (float*)(smem + kRedOffset) + u.uid * 4;
+  u.phase = 0;
+  // red layout: [slot(2)][16 floats]; unit k uses floats 4k..4k+3 of each slot
+  const uint32_t n_units = (uint32_t)(n_cwarps * 32 / UNIT);
+  int* abort_flag = (int*)(smem + kFlagOffset) + (UNIT > 32 ? u.uid : 0);
+  float* tab = (float*)(smem + kTabOffset) + u.uid * 16;
+  float tab_mn = __int_as_float(0x7fc00000), tab_s = tab_mn;  // NaN: nothing cached yet
+
+  const uint32_t L = a.row_len;
+  const uint32_t G = (VMODE == kPair && (L & 1u)) ? 2u : 1u;  // rows handled back to back
+  const uint32_t n_groups = a.tile_rows / G;
+  const uint32_t rounds = (n_groups + n_units - 1) / n_units;
+
+  for (uint64_t it = 0; it < my_tiles; ++it) {
+    const uint32_t s = (uint32_t)(it % S);
+    bool ok = mbar_wait(&full[s], (uint32_t)((it / S) & 1), a.error_word, kErrLoadWait);
+    ok = __all_sync(0xffffffffu, ok);
+    if (UNIT > 32) {
+      if (!ok && lane == 0) *(volatile int*)abort_flag = 1;
+      named_bar_sync(1 + u.uid, UNIT);
+      ok = *(volatile int*)abort_flag == 0;
+    }
+    if (!ok) break;
+    unsigned char* st = smem + kHeaderBytes + (size_t)s * a.stage_bytes;
+    unsigned char* data = st;
+    unsigned char* codes = st + a.code_off;
+    float* meta_s = (float*)(st + a.meta_off);
+    for (uint32_t rd = 0; rd < rounds; ++rd) {
+      const uint32_t grp = rd * n_units + u.uid;
+      const bool active = grp < n_groups;
+      for (uint32_t h = 0; h < G; ++h) {
+        const uint32_t r = active ? grp * G + h : 0;
+        if (KERNEL == kGeluFwd) W::gelu_fwd(u, data, codes, meta_s, r, L, active);
+        if (KERNEL == kSoftmaxFwd) W::softmax_fwd(u, data, codes, meta_s, r, L, active);
+        if (KERNEL == kGeluBwd) W::gelu_bwd(u, data, codes, meta_s, tab, tab_mn, tab_s, r, L, active);
+        if (KERNEL == kSoftmaxBwd) W::softmax_bwd(u, data, codes, meta_s, r, L, active);
+        u.sync();  // the next row may share a word / code byte with this one
+      }
+    }
+    fence_proxy_async();  // this thread's shared-memory writes -> visible to the copy engine
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&done[s]);
+  }
+}
+
+constexpr uint32_t kMaxSmem = 227 * 1024;
+
+// Largest per-lane access count instantiated for an access kind.
+template <int DT, int VMODE>
+constexpr int kMaxIters() { return (DT == kBF16 && VMODE == kVec16) ? 8 : 16; }
+
+template <int KERNEL, int DT, int VMODE, int UNIT, int ITERS>
+cudaError_t launch_inst(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
+  auto kfn = tile_kernel<KERNEL, DT, VMODE, UNIT, ITERS>;
+  static bool configured = false;  // per instantiation; the attribute is per device context
+  static int configured_dev = -1;
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (!configured || configured_dev != dev) {
+    cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem);
+    if (e != cudaSuccess) return e;
+    configured = true;
+    configured_dev = dev;
+  }
+  kfn<<<p.grid, (p.warps + 1) * 32, p.smem_bytes, st>>>(ka);
+  return cudaGetLastError();
+}
+
+template <int KERNEL, int DT, int VMODE, int UNIT>
+cudaError_t launch_iters(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
+  switch (p.iters) {
+    case 1: return launch_inst<KERNEL, DT, VMODE, UNIT, 1>(p, ka, st);
+    case 2: return launch_inst<KERNEL, DT, VMODE, UNIT, 2>(p, ka, st);
+    case 4: return launch_inst<KERNEL, DT, VMODE, UNIT, 4>(p, ka, st);
+    case 8: return launch_inst<KERNEL, DT, VMODE, UNIT, 8>(p, ka, st);
+    case 16:
+      // 16 accesses of 8 bfloat16 would be 128 elements per lane: not instantiated
+      if (kMaxIters<DT, VMODE>() >= 16) return launch_inst<KERNEL, DT, VMODE, UNIT, kMaxIters<DT, VMODE>() >= 16 ? 16 : 8>(p, ka, st);
+  }
+  return cudaErrorInvalidValue;
+}
+
+template <int KERNEL, int DT, int VMODE>
+cudaError_t launch_unit(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
+  switch (p.unit_lanes) {
+    case 8: return launch_iters<KERNEL, DT, VMODE, 8>(p, ka, st);
+    case 16: return launch_iters<KERNEL, DT, VMODE, 16>(p, ka, st);
+    case 32: return launch_iters<KERNEL, DT, VMODE, 32>(p, ka, st);
+    case 128: return launch_iters<KERNEL, DT, VMODE, 128>(p, ka, st);
+  }
+  return cudaErrorInvalidValue;
+}
+
+template <int KERNEL, int DT>
+cudaError_t launch_vmode(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
+  return p.vec_elems == 2 ? launch_unit<KERNEL, DT, kPair>(p, ka, st)
+                          : launch_unit<KERNEL, DT, kVec16>(p, ka, st);
+}
+
+
+// One translation unit per entry point instantiates this.
+template <int KERNEL>
+cudaError_t launch_tile_kernel(int dt, const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
+  return dt == kF32 ? launch_vmode<KERNEL, kF32>(p, ka, st) : launch_vmode<KERNEL, kBF16>(p, ka, st);
+}
+
+}  // namespace
+}  // namespace s2a

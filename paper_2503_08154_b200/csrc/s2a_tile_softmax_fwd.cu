@@ -1,0 +1,10 @@
+// Instantiations of the pipelined tile kernel for s2a_softmax_fwd.
+#include "s2a_tile.cuh"
+
+namespace s2a {
+
+cudaError_t launch_tile_softmax_fwd(int dt, const TilePlan& p, const void* kernel_args, cudaStream_t st) {
+  return launch_tile_kernel<kSoftmaxFwd>(dt, p, *(const TileKernelArgs*)kernel_args, st);
+}
+
+}  // namespace s2a

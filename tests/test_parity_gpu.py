@@ -78,10 +78,14 @@ def _softmax_inputs(rows, L, dt, seed=0):
 
 
 # ------------------------------------------------------------------ small shapes, tails
-GELU_SHAPES = [(5, 1), (3, 2), (7, 3), (9, 63), (64, 64), (33, 65), (41, 197), (12, 257), (37, 1024),
-               (40, 3072), (13, 3072), (11, 4096), (6, 5120), (3, 8191), (2, 8192), (1, 16384), (2, 40000)]
-SOFTMAX_SHAPES = [(7, 1), (4, 2), (5, 3), (33, 63), (77, 64), (1000, 64), (33, 65), (300, 197), (1, 197),
-                  (130, 257), (257, 257), (40, 1024), (9, 4096), (5, 8191), (3, 8192), (2, 40000)]
+# Row counts are chosen so that the pipelined path runs several tiles AND leaves a ragged
+# remainder for the row-at-a-time path; the very long and the tiny cases take the latter only.
+GELU_SHAPES = [(5, 1), (3, 2), (7, 3), (9, 63), (701, 63), (64, 64), (1001, 64), (33, 65), (531, 65),
+               (41, 197), (451, 197), (301, 257), (137, 1024), (300, 66), (203, 1000),
+               (40, 3072), (13, 3072), (11, 4096), (9, 5120), (3, 8191), (5, 8192), (1, 16384), (2, 40000)]
+SOFTMAX_SHAPES = [(7, 1), (4, 2), (5, 3), (33, 63), (701, 63), (77, 64), (1001, 64), (531, 65), (300, 197),
+                  (1, 197), (1283, 197), (130, 257), (257, 257), (323, 257), (137, 1024), (300, 66),
+                  (203, 1000), (9, 4096), (21, 3072), (7, 5120), (5, 8191), (5, 8192), (2, 40000)]
 
 
 @pytest.mark.parametrize("dt", [F32, BF16])
@@ -102,6 +106,14 @@ def test_in_place(dt):
     check_gelu(*_gelu_inputs(70, 197, dt, seed=3), 197, dt, inplace=True)
     check_softmax(*_softmax_inputs(700, 197, dt, seed=3), 197, dt, inplace=True)
     check_softmax(*_softmax_inputs(20, 4096, dt, seed=3), 4096, dt, inplace=True)
+
+
+def test_benchmark_shapes_take_the_pipelined_path():
+    for sh in (synth.VIT_B16_B8_F32, synth.VIT_B16_B64, synth.VIT_L16_B64, synth.VIT_H14_B32):
+        for kernel in range(4):
+            n, L = (sh.gelu_elems, sh.hidden) if kernel < 2 else (sh.softmax_elems, sh.tokens)
+            plan = binding.s2a_describe_plan(kernel, n, L, sh.dtype)
+            assert plan.startswith("tile") and plan.endswith("tail_rows=0"), plan
 
 
 # ------------------------------------------------------------------ degenerate inputs
