@@ -1,0 +1,456 @@
+#!/usr/bin/env python
+"""Benchmark of the S2A 4-bit stash hot path on synthetic ViT-shaped activations.
+
+One step = one pass of the whole path over one batch: for every transformer block the
+softmax and GELU forward kernels (keeping each block's 4-bit stash resident), then for
+every block in reverse the GELU and softmax backward kernels.  The default workload is
+ViT-B/16 at 224 px, batch 64, bfloat16, 12 blocks.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line.  With N > 1 (launched by torchrun, one rank per GPU) every rank
+runs an independent replica -- rows are independent, the path has no exchange step --
+and the line reports the aggregate over ranks against the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import ctypes
+import hashlib
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2503_08154_b200 import synth  # noqa: E402
+
+KERNELS = ("softmax_fwd", "gelu_fwd", "gelu_bwd", "softmax_bwd")
+L2_BYTES = 126 * 1024 * 1024
+NOMINAL_HBM_GBS = 8000.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=synth.VIT_B16_B64.name, choices=sorted(synth.SHAPES))
+    ap.add_argument("--blocks", type=int, default=0, help="override the number of blocks (0: the workload's)")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--skip-e2e", action="store_true")
+    ap.add_argument("--skip-cpu-baseline", action="store_true")
+    ap.add_argument("--seed", type=int, default=0)
+    return ap.parse_args()
+
+
+# ------------------------------------------------------------------ bytes the method must move
+def algorithmic_bytes(n_elems: int, row_len: int, itemsize: int) -> int:
+    """Per kernel launch: tensor in + tensor out + packed codes + per-row (min, s)."""
+    return 2 * n_elems * itemsize + (n_elems + 1) // 2 + 8 * (n_elems // row_len)
+
+
+def workload_tables(shape, blocks):
+    item = synth.io_itemsize(shape.dtype)
+    has_softmax = shape.name != synth.VIT_B16_B8_F32.name
+    per_launch = {}
+    elems = {}
+    for k in KERNELS:
+        if k.startswith("softmax"):
+            if not has_softmax:
+                continue
+            elems[k] = shape.softmax_elems
+            per_launch[k] = algorithmic_bytes(shape.softmax_elems, shape.tokens, item)
+        else:
+            elems[k] = shape.gelu_elems
+            per_launch[k] = algorithmic_bytes(shape.gelu_elems, shape.hidden, item)
+    step_bytes = blocks * sum(per_launch.values())
+    # each nonlinearity's elements are counted once per step (forward+backward is one unit)
+    step_elems = blocks * (shape.gelu_elems + (shape.softmax_elems if has_softmax else 0))
+    stash = blocks * sum((elems[k] + 1) // 2 + 8 * (elems[k] // (shape.tokens if k.startswith("softmax") else shape.hidden))
+                         for k in per_launch if k.endswith("fwd"))
+    return has_softmax, per_launch, elems, step_bytes, step_elems, stash
+
+
+# ------------------------------------------------------------------ host inputs
+def host_inputs(shape, blocks, seed, rows_gelu=None, rows_softmax=None, with_softmax=True):
+    """Per block: (gelu_x, gelu_g, softmax_x, softmax_g) as numpy arrays in I/O representation."""
+    def one(b):
+        gx, gg = synth.vit_gelu_inputs(shape, seed, b, rows_gelu)
+        if with_softmax:
+            sx, sg = synth.vit_softmax_inputs(shape, seed, b, rows_softmax)
+        else:
+            sx = sg = None
+        return gx, gg, sx, sg
+
+    with ThreadPoolExecutor(max_workers=max(1, min(blocks, os.cpu_count() or 1))) as pool:
+        return list(pool.map(one, range(blocks)))
+
+
+# ------------------------------------------------------------------ clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    REASONS = {
+        0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+        0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+        0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting",
+    }
+
+    def __init__(self, uuid, index):
+        self.samples = []
+        self.stop = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            self.nv = pynvml
+            pynvml.nvmlInit()
+            try:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + str(uuid)).encode())
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.max_mhz = None
+        self.thread = threading.Thread(target=self._run, daemon=True)
+
+    def _run(self):
+        nv = self.nv
+        while not self.stop.is_set():
+            try:
+                mhz = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)
+                try:
+                    reasons = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    reasons = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                self.samples.append((time.perf_counter(), mhz, reasons))
+            except Exception:
+                pass
+            self.stop.wait(0.01)
+
+    def start(self):
+        if self.ok:
+            self.thread.start()
+
+    def finish(self, t0, t1):
+        if not self.ok:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "note": "NVML unavailable"}
+        self.stop.set()
+        self.thread.join()
+        inside = [s for s in self.samples if t0 <= s[0] <= t1]
+        note = "sampled during the timed region"
+        if not inside:
+            inside = self.samples[-3:]
+            note = "timed region shorter than the sampling period: last samples under load"
+        bits = 0
+        for s in inside:
+            bits |= s[2]
+        reasons = [name for bit, name in self.REASONS.items() if bits & bit and name != "gpu_idle"]
+        return {"sm_mhz": statistics.median(s[1] for s in inside) if inside else None,
+                "sm_max_mhz": self.max_mhz, "reasons": reasons, "samples": len(inside), "note": note}
+
+
+# ------------------------------------------------------------------ peaks and stored traffic
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        return float(json.load(open(path))["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def kernel_source_digest():
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_2503_08154_b200", "csrc")
+    for name in sorted(os.listdir(csrc)):
+        h.update(open(os.path.join(csrc, name), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def stored_traffic(kernel, workload):
+    """DRAM bytes per launch from the committed ncu capture, if the kernels are unchanged since."""
+    try:
+        t = json.load(open(os.path.join(ROOT, "profiles", "traffic.json")))
+        e = t[workload][kernel]
+        return e["dram_bytes_per_launch"] if e["source_digest"] == kernel_source_digest() else None
+    except Exception:
+        return None
+
+
+# ------------------------------------------------------------------ the CPU oracle legs
+def oracle_sample_rate(shape, seed, threads):
+    """Times the oracle, as it stands, on one block's worth of rows (bounded sample)."""
+    from oracle import s2a_oracle as o
+    has_softmax = shape.name != synth.VIT_B16_B8_F32.name
+    item = synth.io_itemsize(shape.dtype)
+    rows_g = min(shape.gelu_rows, max(1, 12_000_000 // shape.hidden))
+    rows_s = min(shape.softmax_rows, max(1, 12_000_000 // shape.tokens))
+    gx, gg, sx, sg = host_inputs(shape, 1, seed, rows_g, rows_s, has_softmax)[0]
+    o.lib()
+    t0 = time.perf_counter()
+    y, c, m = o.gelu_fwd(gx, shape.hidden, shape.dtype, threads)
+    o.gelu_bwd(gg, c, m, shape.hidden, shape.dtype, threads)
+    nbytes = 2 * algorithmic_bytes(gx.size, shape.hidden, item)
+    nelem = gx.size
+    if has_softmax:
+        y, c, m = o.softmax_fwd(sx, shape.tokens, shape.dtype, threads)
+        o.softmax_bwd(sg, c, m, shape.tokens, shape.dtype, threads)
+        nbytes += 2 * algorithmic_bytes(sx.size, shape.tokens, item)
+        nelem += sx.size
+    dt = time.perf_counter() - t0
+    sample = "fwd+bwd on the first %d GELU rows%s of block 0" % (
+        rows_g, (" and %d softmax rows" % rows_s) if has_softmax else "")
+    return nbytes / dt / 1e9, nelem / dt / 1e9, dt, sample
+
+
+def run_reference(args, shape, blocks):
+    """--impl reference: the oracle on the host cores, each step a bounded sample."""
+    from oracle import s2a_oracle as o
+    threads = o.hardware_threads()
+    rates = []
+    t_all = time.perf_counter()
+    sample = ""
+    for i in range(args.warmup + args.steps):
+        gbs, gel, dt, sample = oracle_sample_rate(shape, args.seed, threads)
+        if i >= args.warmup:
+            rates.append((gbs, gel, dt))
+        if time.perf_counter() - t_all > 150 and len(rates) >= 1:
+            break
+    gbs = statistics.mean(r[0] for r in rates)
+    line = {
+        "impl": "reference", "metric": "s2a_fwd_bwd_algorithmic_bandwidth", "value": gbs, "unit": "GB/s",
+        "n_gpus": args.gpus, "steps": len(rates), "warmup": args.warmup,
+        "ms_per_step": 1e3 * statistics.mean(r[2] for r in rates), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": shape.name, "blocks": blocks, "sample_per_step": sample},
+        "gelem_per_s": statistics.mean(r[1] for r in rates),
+        "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------ the CUDA path
+def run_ours(args, shape, blocks, rank, world):
+    import torch
+    from paper_2503_08154_b200 import binding
+
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    lib = binding.lib()  # raises if the CUDA library is missing: there is no other path
+    has_softmax, per_launch, elems, step_bytes, step_elems, stash = workload_tables(shape, blocks)
+    item = synth.io_itemsize(shape.dtype)
+    tdt = torch.float32 if shape.dtype == synth.F32 else torch.bfloat16
+
+    def pin(a):
+        t = torch.from_numpy(a.view(np.int16) if a.dtype == np.uint16 else a)
+        return t.pin_memory()
+
+    def dview(t):
+        return t.view(tdt) if tdt == torch.bfloat16 else t
+
+    host = [tuple(pin(a) if a is not None else None for a in blk) for blk in host_inputs(
+        shape, blocks, args.seed + 1000 * rank, with_softmax=has_softmax)]
+
+    class Block:
+        pass
+
+    blks = []
+    for b in range(blocks):
+        B = Block()
+        gx, gg, sx, sg = host[b]
+        B.gx, B.gg = dview(gx.to(dev)), dview(gg.to(dev))
+        B.gy, B.gin = torch.empty_like(B.gx), torch.empty_like(B.gg)
+        B.gcodes, B.gmeta = binding.alloc_stash(shape.gelu_elems, shape.hidden, dev)
+        if has_softmax:
+            B.sx, B.sg = dview(sx.to(dev)), dview(sg.to(dev))
+            B.sy, B.sin = torch.empty_like(B.sx), torch.empty_like(B.sg)
+            B.scodes, B.smeta = binding.alloc_stash(shape.softmax_elems, shape.tokens, dev)
+        blks.append(B)
+
+    stream = torch.cuda.current_stream()
+    sp = ctypes.c_void_p(stream.cuda_stream)
+    dtc = shape.dtype
+    ng, Lg = shape.gelu_elems, shape.hidden
+    ns, Ls = shape.softmax_elems, shape.tokens
+
+    # the sequence of C-ABI calls of one step, with pre-marshalled arguments
+    calls = []
+    for B in blks:
+        if has_softmax:
+            calls.append(("softmax_fwd", lib.s2a_softmax_fwd, (B.sx.data_ptr(), B.sy.data_ptr(), B.scodes.data_ptr(), B.smeta.data_ptr(), ns, Ls, dtc, sp)))
+        calls.append(("gelu_fwd", lib.s2a_gelu_fwd, (B.gx.data_ptr(), B.gy.data_ptr(), B.gcodes.data_ptr(), B.gmeta.data_ptr(), ng, Lg, dtc, sp)))
+    for B in reversed(blks):
+        calls.append(("gelu_bwd", lib.s2a_gelu_bwd, (B.gg.data_ptr(), B.gcodes.data_ptr(), B.gmeta.data_ptr(), B.gin.data_ptr(), ng, Lg, dtc, sp)))
+        if has_softmax:
+            calls.append(("softmax_bwd", lib.s2a_softmax_bwd, (B.sg.data_ptr(), B.scodes.data_ptr(), B.smeta.data_ptr(), B.sin.data_ptr(), ns, Ls, dtc, sp)))
+
+    def step():
+        for _, fn, a in calls:
+            rc = fn(*a)
+            if rc:
+                raise RuntimeError(binding.status_string(rc))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    if binding.s2a_device_error() != 0:
+        raise RuntimeError("a kernel gave up on a bounded wait during warm-up")
+
+    # ---- timed region: K steps, an event before every launch and one at the end
+    n_calls = len(calls)
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(n_calls + 1)] for _ in range(args.steps)]
+    sampler = ClockSampler(getattr(torch.cuda.get_device_properties(local), "uuid", ""), local)
+    sampler.start()
+    barrier()
+    t0 = time.perf_counter()
+    for k in range(args.steps):
+        ev = events[k]
+        for i, (_, fn, a) in enumerate(calls):
+            ev[i].record(stream)
+            rc = fn(*a)
+            if rc:
+                raise RuntimeError(binding.status_string(rc))
+        ev[n_calls].record(stream)
+    barrier()
+    t1 = time.perf_counter()
+    clocks = sampler.finish(t0, t1)
+    total_ms = events[0][0].elapsed_time(events[-1][n_calls])
+    if binding.s2a_device_error() != 0:
+        raise RuntimeError("a kernel gave up on a bounded wait during the timed region")
+
+    per_kernel_ms = {k: [] for k in per_launch}
+    for ev in events:
+        for i, (name, _, _) in enumerate(calls):
+            per_kernel_ms[name].append(ev[i].elapsed_time(ev[i + 1]))
+
+    if world > 1:
+        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+
+    # ---- end to end: pinned host inputs in, results out, every step
+    e2e = None
+    if not args.skip_e2e:
+        hy_g = torch.empty(shape.gelu_elems * item, dtype=torch.uint8).pin_memory()
+        hy_s = torch.empty(shape.softmax_elems * item, dtype=torch.uint8).pin_memory() if has_softmax else None
+
+        def e2e_step():
+            for B, (gx, gg, sx, sg) in zip(blks, host):
+                if has_softmax:
+                    B.sx.copy_(dview(sx), non_blocking=True)
+                    binding.s2a_softmax_fwd(B.sx, B.sy, B.scodes, B.smeta, Ls)
+                    hy_s.copy_(B.sy.view(torch.uint8), non_blocking=True)
+                B.gx.copy_(dview(gx), non_blocking=True)
+                binding.s2a_gelu_fwd(B.gx, B.gy, B.gcodes, B.gmeta, Lg)
+                hy_g.copy_(B.gy.view(torch.uint8), non_blocking=True)
+            for B, (gx, gg, sx, sg) in zip(reversed(blks), reversed(host)):
+                B.gg.copy_(dview(gg), non_blocking=True)
+                binding.s2a_gelu_bwd(B.gg, B.gcodes, B.gmeta, B.gin, Lg)
+                hy_g.copy_(B.gin.view(torch.uint8), non_blocking=True)
+                if has_softmax:
+                    B.sg.copy_(dview(sg), non_blocking=True)
+                    binding.s2a_softmax_bwd(B.sg, B.scodes, B.smeta, B.sin, Ls)
+                    hy_s.copy_(B.sin.view(torch.uint8), non_blocking=True)
+
+        e2e_step()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        e1.record(stream)
+        barrier()
+        e2e_ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        io_bytes = blocks * 2 * item * (shape.gelu_elems + (shape.softmax_elems if has_softmax else 0))
+        e2e = {"value": world * step_bytes * args.e2e_steps / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s",
+               "h2d_bytes_per_step": io_bytes, "d2h_bytes_per_step": io_bytes, "steps": args.e2e_steps,
+               "ms_per_step": e2e_ms / args.e2e_steps}
+
+    if rank != 0:
+        return
+
+    peak, peak_kind = measured_peak()
+    per_kernel = {}
+    for k, ms in per_kernel_ms.items():
+        avg = statistics.mean(ms)
+        gbs = per_launch[k] / (avg * 1e-3) / 1e9
+        per_kernel[k] = {"avg_ms": avg, "launches": len(ms), "algorithmic_bytes": per_launch[k], "GBps": gbs,
+                         "gelem_per_s": elems[k] / (avg * 1e-3) / 1e9, "frac_of_%s_peak" % peak_kind: gbs / peak,
+                         "frac_of_8TBps": gbs / NOMINAL_HBM_GBS, "share_of_step": sum(ms) / (total_ms)}
+    dominant = max(per_kernel, key=lambda k: per_kernel[k]["share_of_step"])
+    roofline = {"bound": "hbm", "kernel": "s2a_" + dominant, "achieved": per_kernel[dominant]["GBps"], "peak": peak,
+                "peak_source": "%s copy bandwidth" % peak_kind, "unit": "GB/s",
+                "frac": per_kernel[dominant]["GBps"] / peak, "traffic": stored_traffic(dominant, shape.name)}
+
+    value = world * step_bytes * args.steps / (total_ms * 1e-3) / 1e9
+    cpu_baseline = None
+    if not args.skip_cpu_baseline:
+        from oracle import s2a_oracle as o
+        threads = o.hardware_threads()
+        gbs, gel, dtc_s, sample = oracle_sample_rate(shape, args.seed, threads)
+        cpu_baseline = {"value": gbs, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": sample,
+                        "gelem_per_s": gel, "seconds": dtc_s}
+
+    bf16_stash = blocks * 2 * (shape.gelu_elems + (shape.softmax_elems if has_softmax else 0))
+    line = {
+        "metric": "s2a_fwd_bwd_algorithmic_bandwidth", "value": value, "unit": "GB/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": shape.name, "blocks": blocks, "io_dtype": "bf16" if shape.dtype else "f32",
+                   "gelu": [shape.gelu_rows, shape.hidden], "softmax": [shape.softmax_rows, shape.tokens] if has_softmax else None,
+                   "l2": "inputs larger than L2: %.2f GB touched per step, distinct buffers per block" % (step_bytes / 1e9),
+                   "multi_gpu": "independent replicas, no collective"},
+        "gelem_per_s": world * step_elems * args.steps / (total_ms * 1e-3) / 1e9,
+        "frac_of_8TBps": value / world / NOMINAL_HBM_GBS,
+        "frac_of_%s_peak" % peak_kind: value / world / peak,
+        "saved_activation_bytes": {"stash": stash, "bf16_stash": bf16_stash, "fp32_stash": 2 * bf16_stash,
+                                   "reduction_vs_bf16": bf16_stash / stash},
+        "per_kernel": per_kernel, "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e,
+        "gpu_launches": n_calls * args.steps, "clocks": clocks,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    args = parse_args()
+    shape = synth.SHAPES[args.workload]
+    blocks = args.blocks if args.blocks > 0 else shape.blocks
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        if rank == 0:
+            run_reference(args, shape, blocks)
+        return
+    if world != args.gpus and world == 1 and args.gpus > 1:
+        sys.exit("--gpus %d needs a torchrun launch with one rank per GPU" % args.gpus)
+    run_ours(args, shape, blocks, rank, world)
+
+
+if __name__ == "__main__":
+    main()
