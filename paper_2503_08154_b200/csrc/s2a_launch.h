@@ -27,11 +27,14 @@ cudaError_t launch_rowwise(int kernel, int dt, const RowwiseArgs& a, cudaStream_
 // A tile is `tile_rows` consecutive rows whose flat element span starts and ends on a
 // multiple of 32 elements, so that its data and its code bytes can move with 16-byte
 // bulk copies.  A plan with tile_rows == 0 means "no pipelined path for this shape".
+enum { kVariantGeneric = 0, kVariantStream = 1, kVariantPairFixed = 2 };
+
 struct TilePlan {
   uint32_t tile_rows;   // rows per tile (0: not applicable)
-  uint32_t unit_lanes;  // lanes that cooperate on one row: 8, 16 or 32
+  uint32_t variant;     // kVariantGeneric / kVariantStream / kVariantPairFixed
+  uint32_t unit_lanes;  // lanes that cooperate on one row: 8, 16, 32 or 128
   uint32_t vec_elems;   // elements per shared-memory access: 2 (pair mode) or 16 bytes' worth
-  uint32_t iters;       // compile-time bound on accesses per lane per row
+  uint32_t iters;       // accesses per lane per row kept in registers (0: streamed)
   uint32_t warps;       // consumer warps per CTA (one more warp drives the copies)
   uint32_t stages;      // tiles resident in shared memory per CTA
   uint32_t smem_bytes;  // dynamic shared memory per CTA

@@ -59,43 +59,68 @@ unsigned int* error_word_address() {
 }  // namespace
 
 // Launch-shape policy.  Environment overrides (for tuning sweeps): S2A_PATH=rowwise
-// disables this path; S2A_UNIT, S2A_TILE_ROWS, S2A_WARPS, S2A_STAGES, S2A_CTAS_PER_SM.
+// disables this path; S2A_UNIT, S2A_TILE_ROWS, S2A_WARPS, S2A_STAGES, S2A_CTAS_PER_SM,
+// S2A_VARIANT=generic.
 TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L) {
   TilePlan p{};
   const char* path = getenv("S2A_PATH");
   if (path && path[0] == 'r') return p;
+  const char* var = getenv("S2A_VARIANT");
+  const bool force_generic = var && var[0] == 'g';
+  const bool is_gelu = kernel == kGeluFwd || kernel == kGeluBwd;
   const uint32_t esize = dt == kF32 ? 4u : 2u;
-  const uint32_t vec = 16u / esize;                 // elements per 16-byte access
+  const uint32_t vec = 16u / esize;  // elements per 16-byte access
   const bool vec16 = (L % vec) == 0;
   const uint32_t epa = vec16 ? vec : 2u;
   const uint32_t n_acc = vec16 ? L / vec : (L + 1) / 2;  // accesses covering one row
   // rows per tile: the tile's element count must be a multiple of 32, its row count even
   uint32_t r_min = 32u / gcd_u32(L, 32u);
   if (r_min < 2) r_min = 2;
-  const uint64_t min_tile_bytes = (uint64_t)r_min * L * esize;
-  if (min_tile_bytes > kMaxStageBytes) return p;
+  if ((uint64_t)r_min * L * esize > kMaxStageBytes) return p;
 
-  // lanes per row: the smallest unit that keeps a lane at or under ~32 elements, else
-  // the largest unit with up to 16 accesses per lane
-  const uint32_t cap_iters = 32u / epa > 16u ? 16u : 32u / epa;  // vec16 bf16: 4, f32: 8, pair: 16
-  const uint32_t max_iters = (dt == kBF16 && vec16) ? 8u : 16u;  // what is instantiated
-  const uint32_t units[4] = {8, 16, 32, 128};
-  uint32_t unit = 0, need = 0;
-  for (int k = 0; k < 4 && unit == 0; ++k) {
-    need = (n_acc + units[k] - 1) / units[k];
-    if (need <= cap_iters) unit = units[k];
+  uint32_t variant = kVariantGeneric, unit = 0, iters = 0;
+  const int env_unit = env_int("S2A_UNIT", 0);
+  if (vec16 && !force_generic && is_gelu) {
+    // streamed: nothing held in registers; a warp per row unless the row is short
+    variant = kVariantStream;
+    unit = n_acc >= 32 ? 32u : (n_acc >= 16 ? 16u : 8u);
+    if (env_unit == 8 || env_unit == 16 || env_unit == 32) unit = (uint32_t)env_unit;
+  } else if (vec16 && !force_generic) {
+    // softmax on 16-byte vectors: up to 32 (at most 64) elements per lane in registers
+    const uint32_t cap = 32u / epa, cap2 = 64u / epa;
+    const uint32_t units[3] = {8, 16, 32};
+    for (int k = 0; k < 3 && unit == 0; ++k)
+      if ((n_acc + units[k] - 1) / units[k] <= cap) unit = units[k];
+    if (unit == 0 && (n_acc + 31) / 32 <= cap2) unit = 32;
+    if (env_unit == 8 || env_unit == 16 || env_unit == 32) unit = (uint32_t)env_unit;
+    if (unit != 0 && (n_acc + unit - 1) / unit <= cap2) {
+      variant = kVariantStream;
+      iters = 1;
+      while (iters < (n_acc + unit - 1) / unit) iters *= 2;
+    } else {
+      unit = 0;
+    }
+  } else if (!vec16 && !force_generic && !is_gelu && (L == 197 || L == 257)) {
+    variant = kVariantPairFixed;
+    unit = 8;
+    iters = (n_acc + 7) / 8;
   }
-  if (unit == 0) {
-    need = (n_acc + 127) / 128;
+  if (variant == kVariantGeneric) {
+    // general register-resident form: pair accesses with 8 or 32 lanes per row, or 16-byte
+    // accesses with 128 lanes per row (long softmax rows)
+    const uint32_t max_iters = (dt == kBF16 && vec16) ? 8u : 16u;
+    if (vec16) {
+      if (is_gelu) return p;
+      unit = 128;
+    } else {
+      unit = (n_acc + 7) / 8 <= 16 ? 8u : 32u;
+      if (env_unit == 8 || env_unit == 32) unit = (uint32_t)env_unit;
+    }
+    const uint32_t need = (n_acc + unit - 1) / unit;
     if (need > max_iters) return p;
-    unit = 128;
+    iters = 1;
+    while (iters < need) iters *= 2;
   }
-  unit = (uint32_t)env_int("S2A_UNIT", (int)unit);
-  if (unit != 8 && unit != 16 && unit != 32 && unit != 128) return p;
-  need = (n_acc + unit - 1) / unit;
-  if (need > max_iters) return p;
-  uint32_t iters = 1;
-  while (iters < need) iters *= 2;
 
   uint32_t warps = unit == 128 ? 8u : 4u;
   warps = (uint32_t)env_int("S2A_WARPS", (int)warps);
@@ -109,6 +134,7 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L) {
   const uint32_t want_rows = n_units * G;
   while (rows % want_rows != 0 && (uint64_t)(rows + r_min) * L * esize <= kMaxStageBytes) rows += r_min;
   while ((uint64_t)rows * L * esize < 16 * 1024 && (uint64_t)rows * 2 * L * esize <= kMaxStageBytes) rows *= 2;
+  if (variant == kVariantPairFixed && rows < 64 && (uint64_t)64 * L * esize <= kMaxStageBytes) rows = 64;
   rows = (uint32_t)env_int("S2A_TILE_ROWS", (int)rows);
   if (rows == 0 || rows % r_min != 0 || (uint64_t)rows * L * esize > kMaxStageBytes) return p;
 
@@ -138,6 +164,7 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L) {
   p.n_tiles = n_rows / rows;
   if (p.n_tiles == 0) return TilePlan{};
   p.tile_rows = rows;
+  p.variant = variant;
   p.unit_lanes = unit;
   p.vec_elems = epa;
   p.iters = iters;
@@ -147,7 +174,6 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L) {
   uint64_t grid = (uint64_t)sm_count() * (uint32_t)ctas_per_sm;
   if (grid > p.n_tiles) grid = p.n_tiles;
   p.grid = (uint32_t)grid;
-  (void)kernel;
   return p;
 }
 
@@ -168,6 +194,13 @@ cudaError_t launch_tile(int kernel, int dt, const TilePlan& p, const TileArgs& a
   ka.meta_off = ka.code_off + align_up(ka.code_bytes, 128);
   ka.stage_bytes = ka.meta_off + align_up(ka.meta_bytes, 128);
   ka.stages = p.stages;
+  {
+    // spreading needs every warp's units to find a group in every round
+    const uint32_t upw = p.unit_lanes < 32 ? 32 / p.unit_lanes : 1;
+    const uint32_t G = (p.vec_elems == 2 && (a.row_len & 1u)) ? 2u : 1u;
+    const uint32_t n_groups = p.tile_rows / G;
+    ka.spread_units = (upw > 1 && n_groups % upw == 0 && env_int("S2A_SPREAD", 1) != 0) ? 1u : 0u;
+  }
   ka.error_word = error_word_address();
   if (!ka.error_word) return cudaErrorInvalidDevice;
   switch (kernel) {

@@ -50,6 +50,7 @@ struct TileKernelArgs {
   uint32_t meta_off;
   uint32_t stage_bytes;
   uint32_t stages;
+  uint32_t spread_units;     // 1: sub-warp units of a warp take groups a fixed stride apart
   unsigned int* error_word;  // device address of the per-device error word
 };
 
@@ -518,10 +519,568 @@ struct RowWork {
   }
 };
 
+// ---------------------------------------------------------------- work policies
+// A policy tells the pipeline skeleton how the consumer lanes of a CTA turn one tile
+// in shared memory into its results.  `group` is called by all lanes of a unit for one
+// group of consecutive rows (one row, or the two rows of an odd-length pair).
+struct StagePtrs {
+  unsigned char* data;
+  unsigned char* codes;
+  float* meta;
+};
+
+// Policy 0: the general register-resident form (any row length that fits ITERS).
+template <int KERNEL, int DT, int VMODE, int UNIT_, int ITERS>
+struct GenericWork {
+  static constexpr int kKernel = KERNEL;
+  static constexpr int UNIT = UNIT_;
+  using W = RowWork<KERNEL, DT, VMODE, UNIT_, ITERS>;
+  struct State {
+    float tab_mn, tab_s;
+  };
+  static __device__ __forceinline__ void init(State& st) {
+    st.tab_mn = __int_as_float(0x7fc00000);  // NaN: nothing cached yet
+    st.tab_s = st.tab_mn;
+  }
+  static __device__ __forceinline__ uint32_t rows_per_group(uint32_t L) {
+    return (VMODE == kPair && (L & 1u)) ? 2u : 1u;
+  }
+  static __device__ __forceinline__ void group(Unit<UNIT_>& u, State& st, const StagePtrs& p, float* tab,
+                                               uint32_t grp, bool active, uint32_t L) {
+    const uint32_t G = rows_per_group(L);
+    for (uint32_t h = 0; h < G; ++h) {
+      const uint32_t r = active ? grp * G + h : 0;
+      if (KERNEL == kGeluFwd) W::gelu_fwd(u, p.data, p.codes, p.meta, r, L, active);
+      if (KERNEL == kSoftmaxFwd) W::softmax_fwd(u, p.data, p.codes, p.meta, r, L, active);
+      if (KERNEL == kGeluBwd) W::gelu_bwd(u, p.data, p.codes, p.meta, tab, st.tab_mn, st.tab_s, r, L, active);
+      if (KERNEL == kSoftmaxBwd) W::softmax_bwd(u, p.data, p.codes, p.meta, r, L, active);
+      u.sync();  // the next row may share a word / code byte with this one
+    }
+  }
+};
+
+// ---------------------------------------------------------------- 16-byte streaming
+// Rows whose length is a multiple of the 16-byte vector.  A unit streams the row out of
+// shared memory as many times as the arithmetic needs (shared memory has several times
+// the bandwidth of an SM's share of HBM), so the GELU kernels keep nothing in registers
+// and accept any row length; the softmax kernels keep NV vectors per lane.
+constexpr uint32_t kMagicBits = 0x4B400000u;  // bit pattern of 1.5 * 2^23
+
+template <int DT> struct V16;
+template <> struct V16<kBF16> {
+  static constexpr int EPA = 8;
+  using Raw = uint4;
+  struct MinMax {  // packed bfloat16x2 running min / max
+    uint32_t mn, mx;
+    __device__ __forceinline__ void init() { mn = 0x7F807F80u; mx = 0xFF80FF80u; }
+    __device__ __forceinline__ void add(const Raw& r) {
+      const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        __nv_bfloat162 v = *(const __nv_bfloat162*)&w[k];
+        __nv_bfloat162 a = __hmin2(*(__nv_bfloat162*)&mn, v), b = __hmax2(*(__nv_bfloat162*)&mx, v);
+        mn = *(uint32_t*)&a;
+        mx = *(uint32_t*)&b;
+      }
+    }
+    __device__ __forceinline__ float lo() const {
+      return fminf(__uint_as_float(mn << 16), __uint_as_float(mn & 0xffff0000u));
+    }
+    __device__ __forceinline__ float hi() const {
+      return fmaxf(__uint_as_float(mx << 16), __uint_as_float(mx & 0xffff0000u));
+    }
+  };
+  static __device__ __forceinline__ void widen(const Raw& r, float* v) {
+    const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      v[2 * k] = __uint_as_float(w[k] << 16);
+      v[2 * k + 1] = __uint_as_float(w[k] & 0xffff0000u);
+    }
+  }
+  // Rounds to bfloat16; leaves the values as written in v.
+  static __device__ __forceinline__ Raw narrow(float* v) {
+    uint32_t w[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      __nv_bfloat162 b = __floats2bfloat162_rn(v[2 * k], v[2 * k + 1]);
+      w[k] = *(uint32_t*)&b;
+      v[2 * k] = __uint_as_float(w[k] << 16);
+      v[2 * k + 1] = __uint_as_float(w[k] & 0xffff0000u);
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+  }
+  static __device__ __forceinline__ uint32_t load_codes(const unsigned char* c, uint32_t j) {
+    return *(const uint32_t*)(c + j * 4u);
+  }
+  static __device__ __forceinline__ void store_codes(unsigned char* c, uint32_t j, uint32_t bits) {
+    *(uint32_t*)(c + j * 4u) = bits;
+  }
+};
+template <> struct V16<kF32> {
+  static constexpr int EPA = 4;
+  using Raw = float4;
+  struct MinMax {
+    float mn, mx;
+    __device__ __forceinline__ void init() { mn = INFINITY; mx = -INFINITY; }
+    __device__ __forceinline__ void add(const Raw& r) {
+      mn = fminf(fminf(mn, r.x), fminf(r.y, fminf(r.z, r.w)));
+      mx = fmaxf(fmaxf(mx, r.x), fmaxf(r.y, fmaxf(r.z, r.w)));
+    }
+    __device__ __forceinline__ float lo() const { return mn; }
+    __device__ __forceinline__ float hi() const { return mx; }
+  };
+  static __device__ __forceinline__ void widen(const Raw& r, float* v) {
+    v[0] = r.x; v[1] = r.y; v[2] = r.z; v[3] = r.w;
+  }
+  static __device__ __forceinline__ Raw narrow(float* v) { return make_float4(v[0], v[1], v[2], v[3]); }
+  static __device__ __forceinline__ uint32_t load_codes(const unsigned char* c, uint32_t j) {
+    return *(const uint16_t*)(c + j * 2u);
+  }
+  static __device__ __forceinline__ void store_codes(unsigned char* c, uint32_t j, uint32_t bits) {
+    *(uint16_t*)(c + j * 2u) = (uint16_t)bits;
+  }
+};
+
+// Codes of N elements packed with one shift-add each: the rounded value sits in the low
+// mantissa bits of (t + 1.5 * 2^23), whose other bits are a known constant.  Only the
+// low 4N bits of `acc` are meaningful.
+template <int N>
+struct CodePacker {
+  static constexpr uint32_t kOnes = N == 8 ? 0x11111111u : (N == 4 ? 0x1111u : 0x11u);
+  uint32_t acc;
+  __device__ __forceinline__ void init() { acc = 0u - kMagicBits * kOnes; }
+  __device__ __forceinline__ void add(int k, float v, const QRange& q) {
+    const float t = __fmul_rn(__fsub_rn(v, q.mn), q.inv);
+    acc += __float_as_uint(__fadd_rn(t, 12582912.0f)) << (4 * k);
+  }
+};
+
+template <int DT, int UNIT_>
+struct StreamGeluFwd {
+  static constexpr int kKernel = kGeluFwd;
+  static constexpr int UNIT = UNIT_;
+  using V = V16<DT>;
+  struct State {};
+  static __device__ __forceinline__ void init(State&) {}
+  static __device__ __forceinline__ uint32_t rows_per_group(uint32_t) { return 1u; }
+
+  static __device__ __forceinline__ void group(Unit<UNIT_>& u, State&, const StagePtrs& p, float*, uint32_t r,
+                                               bool active, uint32_t L) {
+    const uint32_t nv = active ? L / V::EPA : 0u;
+    unsigned char* row = p.data + (size_t)r * L * Io<DT>::kBytes;
+    unsigned char* crow = p.codes + (size_t)r * (L / 2);
+    typename V::MinMax mm;
+    mm.init();
+#pragma unroll 4
+    for (uint32_t j = u.ul; j < nv; j += UNIT_) mm.add(*(const typename V::Raw*)(row + j * 16u));
+    const float mn = u.template reduce<kOpMin>(mm.lo());
+    const float mx = u.template reduce<kOpMax>(mm.hi());
+    // min / max of the clipped row = clipped min / max of the row (the clip is monotone)
+    const QRange q = make_qrange(fminf(fmaxf(mn, -kClip), kClip), fminf(fmaxf(mx, -kClip), kClip));
+    if (active && u.ul == 0) { p.meta[2 * r] = q.mn; p.meta[2 * r + 1] = q.s; }
+#pragma unroll 2
+    for (uint32_t j = u.ul; j < nv; j += UNIT_) {
+      float v[V::EPA];
+      V::widen(*(const typename V::Raw*)(row + j * 16u), v);
+      CodePacker<V::EPA> pk;
+      pk.init();
+#pragma unroll
+      for (int k = 0; k < V::EPA; ++k) {
+        pk.add(k, fminf(fmaxf(v[k], -kClip), kClip), q);
+        v[k] = gelu_eval<DT>(v[k]);
+      }
+      *(typename V::Raw*)(row + j * 16u) = V::narrow(v);
+      V::store_codes(crow, j, pk.acc);
+    }
+  }
+};
+
+// GELU backward.  With a whole warp on one row the 16 derivative values live one per
+// lane (twice over) and are fetched with a shuffle indexed by the code; smaller units
+// read them from a shared-memory table.
+template <int DT, int UNIT_>
+struct StreamGeluBwd {
+  static constexpr int kKernel = kGeluBwd;
+  static constexpr int UNIT = UNIT_;
+  using V = V16<DT>;
+  struct State {
+    float tab_mn, tab_s, d;  // cached (min, s) and this lane's table entry
+  };
+  static __device__ __forceinline__ void init(State& st) {
+    st.tab_mn = __int_as_float(0x7fc00000);
+    st.tab_s = st.tab_mn;
+    st.d = 0.0f;
+  }
+  static __device__ __forceinline__ uint32_t rows_per_group(uint32_t) { return 1u; }
+
+  static __device__ __forceinline__ void group(Unit<UNIT_>& u, State& st, const StagePtrs& p, float* tab,
+                                               uint32_t r, bool active, uint32_t L) {
+    const float mn = active ? p.meta[2 * r] : st.tab_mn;
+    const float s = active ? p.meta[2 * r + 1] : st.tab_s;
+    // The 16 values of Eq. 12 this row can take, in binary64; kept while (min, s) repeat.
+    if (mn != st.tab_mn || s != st.tab_s) {
+      if (UNIT_ == 32) {
+        st.d = (float)gelu_sine_derivative((uint32_t)(u.ul & 15), mn, s);
+      } else {
+#pragma unroll
+        for (int c = 0; c < 16; c += (UNIT_ < 16 ? UNIT_ : 16)) {
+          const int code = c + u.ul;
+          if (u.ul < 16 && code < 16) tab[code] = (float)gelu_sine_derivative((uint32_t)code, mn, s);
+        }
+      }
+      st.tab_mn = mn;
+      st.tab_s = s;
+    }
+    if (UNIT_ != 32) u.sync();
+    const uint32_t nv = active ? L / V::EPA : 0u;
+    unsigned char* row = p.data + (size_t)r * L * Io<DT>::kBytes;
+    const unsigned char* crow = p.codes + (size_t)r * (L / 2);
+    // every lane runs the same number of rounds so that the shuffles stay warp-wide
+    const uint32_t rounds = (nv + UNIT_ - 1) / UNIT_;
+#pragma unroll 2
+    for (uint32_t it = 0; it < rounds; ++it) {
+      const uint32_t j = it * UNIT_ + u.ul;
+      const bool ok = j < nv;
+      float v[V::EPA];
+      uint32_t bits = 0;
+      if (ok) {
+        V::widen(*(const typename V::Raw*)(row + j * 16u), v);
+        bits = V::load_codes(crow, j);
+      }
+#pragma unroll
+      for (int k = 0; k < V::EPA; ++k) {
+        float d;
+        if (UNIT_ == 32) d = __shfl_sync(0xffffffffu, st.d, (int)(bits >> (4 * k)));  // lane = code mod 16 (+16)
+        else d = tab[(bits >> (4 * k)) & 0xFu];
+        v[k] *= d;
+      }
+      if (ok) *(typename V::Raw*)(row + j * 16u) = V::narrow(v);
+    }
+  }
+};
+
+// Softmax forward on 16-byte vectors, NV vectors per lane kept in registers.
+template <int DT, int UNIT_, int NV>
+struct StreamSoftmaxFwd {
+  static constexpr int kKernel = kSoftmaxFwd;
+  static constexpr int UNIT = UNIT_;
+  using V = V16<DT>;
+  static constexpr int EPA = V::EPA;
+  struct State {};
+  static __device__ __forceinline__ void init(State&) {}
+  static __device__ __forceinline__ uint32_t rows_per_group(uint32_t) { return 1u; }
+
+  static __device__ __forceinline__ void group(Unit<UNIT_>& u, State&, const StagePtrs& p, float*, uint32_t r,
+                                               bool active, uint32_t L) {
+    const uint32_t nv = active ? L / EPA : 0u;
+    unsigned char* row = p.data + (size_t)r * L * Io<DT>::kBytes;
+    unsigned char* crow = p.codes + (size_t)r * (L / 2);
+    float e[NV][EPA];
+    float m = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+      const uint32_t j = u.ul + UNIT_ * i;
+      if (j < nv) {
+        V::widen(*(const typename V::Raw*)(row + j * 16u), e[i]);
+#pragma unroll
+        for (int k = 0; k < EPA; ++k) m = fmaxf(m, e[i][k]);
+      } else {
+#pragma unroll
+        for (int k = 0; k < EPA; ++k) e[i][k] = -INFINITY;
+      }
+    }
+    m = u.template reduce<kOpMax>(m);
+    if (!active) m = 0.0f;
+    float z = 0.0f;
+#pragma unroll
+    for (int i = 0; i < NV; ++i)
+#pragma unroll
+      for (int k = 0; k < EPA; ++k) {
+        e[i][k] = exp_eval<DT>(e[i][k] - m);
+        z += e[i][k];
+      }
+    z = u.template reduce<kOpSum>(z);
+    const float rz = __fdiv_rn(1.0f, active ? z : 1.0f);
+    float mn = INFINITY, mx = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+      const uint32_t j = u.ul + UNIT_ * i;
+      if (j < nv) {
+#pragma unroll
+        for (int k = 0; k < EPA; ++k) e[i][k] *= rz;
+        *(typename V::Raw*)(row + j * 16u) = V::narrow(e[i]);  // e now holds y as written
+#pragma unroll
+        for (int k = 0; k < EPA; ++k) { mn = fminf(mn, e[i][k]); mx = fmaxf(mx, e[i][k]); }
+      }
+    }
+    mn = u.template reduce<kOpMin>(mn);
+    mx = u.template reduce<kOpMax>(mx);
+    const QRange q = make_qrange(mn, mx);
+    if (active && u.ul == 0) { p.meta[2 * r] = q.mn; p.meta[2 * r + 1] = q.s; }
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+      const uint32_t j = u.ul + UNIT_ * i;
+      if (j < nv) {
+        CodePacker<EPA> pk;
+        pk.init();
+#pragma unroll
+        for (int k = 0; k < EPA; ++k) pk.add(k, e[i][k], q);
+        V::store_codes(crow, j, pk.acc);
+      }
+    }
+  }
+};
+
+template <int DT, int UNIT_, int NV>
+struct StreamSoftmaxBwd {
+  static constexpr int kKernel = kSoftmaxBwd;
+  static constexpr int UNIT = UNIT_;
+  using V = V16<DT>;
+  static constexpr int EPA = V::EPA;
+  struct State {};
+  static __device__ __forceinline__ void init(State&) {}
+  static __device__ __forceinline__ uint32_t rows_per_group(uint32_t) { return 1u; }
+
+  static __device__ __forceinline__ void group(Unit<UNIT_>& u, State&, const StagePtrs& p, float*, uint32_t r,
+                                               bool active, uint32_t L) {
+    const uint32_t nv = active ? L / EPA : 0u;
+    unsigned char* row = p.data + (size_t)r * L * Io<DT>::kBytes;
+    const unsigned char* crow = p.codes + (size_t)r * (L / 2);
+    const float mn = active ? p.meta[2 * r] : 0.0f;
+    const float s = active ? p.meta[2 * r + 1] : 0.0f;
+    float g[NV][EPA], yh[NV][EPA];
+    float dot = 0.0f;
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+      const uint32_t j = u.ul + UNIT_ * i;
+      if (j < nv) {
+        V::widen(*(const typename V::Raw*)(row + j * 16u), g[i]);
+        const uint32_t bits = V::load_codes(crow, j);
+#pragma unroll
+        for (int k = 0; k < EPA; ++k) {
+          yh[i][k] = dequant((bits >> (4 * k)) & 0xFu, mn, s);
+          dot = fmaf(g[i][k], yh[i][k], dot);
+        }
+      }
+    }
+    dot = u.template reduce<kOpSum>(dot);
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+      const uint32_t j = u.ul + UNIT_ * i;
+      if (j < nv) {
+        float v[EPA];
+#pragma unroll
+        for (int k = 0; k < EPA; ++k) v[k] = yh[i][k] * (g[i][k] - dot);
+        *(typename V::Raw*)(row + j * 16u) = V::narrow(v);
+      }
+    }
+  }
+};
+
+// ---------------------------------------------------------------- odd rows, fixed length
+// Softmax rows of a compile-time odd length (the attention widths 197 and 257).  Rows
+// are read as 2-element words on the tile's even-element grid: a row that starts on an
+// even element shares its LAST word (and code byte) with the next row, a row that starts
+// on an odd element shares its FIRST word with the previous one; a unit handles such a
+// pair back to back.  With the length fixed every mask is resolved at compile time
+// except on the one or two words that are actually shared or ragged.
+template <int DT> struct P2;
+template <> struct P2<kBF16> {
+  using Raw = uint32_t;
+  static constexpr int kWordBytes = 4;
+  static __device__ __forceinline__ Raw load(const unsigned char* d, uint32_t a) { return *(const uint32_t*)(d + a * 4u); }
+  static __device__ __forceinline__ float lo(Raw w) { return __uint_as_float(w << 16); }
+  static __device__ __forceinline__ float hi(Raw w) { return __uint_as_float(w & 0xffff0000u); }
+  static __device__ __forceinline__ Raw pack(float a, float b) {
+    __nv_bfloat162 t = __floats2bfloat162_rn(a, b);
+    return *(uint32_t*)&t;
+  }
+  static __device__ __forceinline__ void store(unsigned char* d, uint32_t a, Raw w) { *(uint32_t*)(d + a * 4u) = w; }
+  static __device__ __forceinline__ void store_lo(unsigned char* d, uint32_t a, Raw w) { *(uint16_t*)(d + a * 4u) = (uint16_t)w; }
+  static __device__ __forceinline__ void store_hi(unsigned char* d, uint32_t a, Raw w) { *(uint16_t*)(d + a * 4u + 2) = (uint16_t)(w >> 16); }
+};
+template <> struct P2<kF32> {
+  using Raw = float2;
+  static constexpr int kWordBytes = 8;
+  static __device__ __forceinline__ Raw load(const unsigned char* d, uint32_t a) { return *(const float2*)(d + a * 8u); }
+  static __device__ __forceinline__ float lo(Raw w) { return w.x; }
+  static __device__ __forceinline__ float hi(Raw w) { return w.y; }
+  static __device__ __forceinline__ Raw pack(float a, float b) { return make_float2(a, b); }
+  static __device__ __forceinline__ void store(unsigned char* d, uint32_t a, Raw w) { *(float2*)(d + a * 8u) = w; }
+  static __device__ __forceinline__ void store_lo(unsigned char* d, uint32_t a, Raw w) { *(float*)(d + a * 8u) = w.x; }
+  static __device__ __forceinline__ void store_hi(unsigned char* d, uint32_t a, Raw w) { *(float*)(d + a * 8u + 4) = w.y; }
+};
+
+template <int UNIT_, int LCT>
+struct PairGeom {
+  static_assert(LCT % 2 == 1, "odd row lengths only");
+  static constexpr int NACC = (LCT + 1) / 2;               // words covering one row
+  static constexpr int ITERS = (NACC + UNIT_ - 1) / UNIT_;
+  static constexpr int NFULL = NACC / UNIT_;               // iterations in which every lane has a word
+  static constexpr int REM = NACC % UNIT_;
+  static constexpr int LAST_I = (NACC - 1) / UNIT_;        // where the row's last word sits
+  static constexpr int LAST_UL = (NACC - 1) % UNIT_;
+  static __device__ __forceinline__ bool has(int i, int ul) { return i < NFULL || ul < REM; }
+};
+
+template <int DT, int UNIT_, int LCT>
+struct PairSoftmaxFwd {
+  static constexpr int kKernel = kSoftmaxFwd;
+  static constexpr int UNIT = UNIT_;
+  using P = P2<DT>;
+  using G = PairGeom<UNIT_, LCT>;
+  struct State {};
+  static __device__ __forceinline__ void init(State&) {}
+  static __device__ __forceinline__ uint32_t rows_per_group(uint32_t) { return 2u; }
+
+  // HP = 0: the row starts on an even element (high half of its last word is foreign);
+  // HP = 1: it starts on an odd element (low half of its first word is foreign).
+  template <int HP>
+  static __device__ __forceinline__ void row(Unit<UNIT_>& u, const StagePtrs& p, uint32_t r, bool active) {
+    const uint32_t a0 = (r * (uint32_t)LCT) >> 1;
+    const int ul = u.ul;
+    float e[G::ITERS][2];
+    float m = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < G::ITERS; ++i) {
+      e[i][0] = -INFINITY;
+      e[i][1] = -INFINITY;
+      if (active && G::has(i, ul)) {
+        const typename P::Raw w = P::load(p.data, a0 + ul + UNIT_ * i);
+        e[i][0] = P::lo(w);
+        e[i][1] = P::hi(w);
+      }
+      if (HP == 1 && i == 0 && ul == 0) e[i][0] = -INFINITY;
+      if (HP == 0 && i == G::LAST_I && ul == G::LAST_UL) e[i][1] = -INFINITY;
+      m = fmaxf(m, fmaxf(e[i][0], e[i][1]));
+    }
+    m = u.template reduce<kOpMax>(m);
+    if (!active) m = 0.0f;
+    float z = 0.0f;
+#pragma unroll
+    for (int i = 0; i < G::ITERS; ++i) {
+      e[i][0] = exp_eval<DT>(e[i][0] - m);  // foreign / absent elements: exp(-inf) = 0
+      e[i][1] = exp_eval<DT>(e[i][1] - m);
+      z += e[i][0] + e[i][1];
+    }
+    z = u.template reduce<kOpSum>(z);
+    const float rz = __fdiv_rn(1.0f, active ? z : 1.0f);
+    float mn = INFINITY, mx = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < G::ITERS; ++i) {
+      const typename P::Raw w = P::pack(e[i][0] * rz, e[i][1] * rz);
+      e[i][0] = P::lo(w);  // y as written
+      e[i][1] = P::hi(w);
+      const bool mine = active && G::has(i, ul);
+      const bool drop_lo = HP == 1 && i == 0 && ul == 0;
+      const bool drop_hi = HP == 0 && i == G::LAST_I && ul == G::LAST_UL;
+      if (mine) {
+        if (drop_lo) P::store_hi(p.data, a0 + ul + UNIT_ * i, w);
+        else if (drop_hi) P::store_lo(p.data, a0 + ul + UNIT_ * i, w);
+        else P::store(p.data, a0 + ul + UNIT_ * i, w);
+        const float v0 = drop_lo ? e[i][1] : e[i][0], v1 = drop_hi ? e[i][0] : e[i][1];
+        mn = fminf(mn, fminf(v0, v1));
+        mx = fmaxf(mx, fmaxf(v0, v1));
+      }
+    }
+    mn = u.template reduce<kOpMin>(mn);
+    mx = u.template reduce<kOpMax>(mx);
+    const QRange q = make_qrange(mn, mx);
+    if (active && ul == 0) { p.meta[2 * r] = q.mn; p.meta[2 * r + 1] = q.s; }
+#pragma unroll
+    for (int i = 0; i < G::ITERS; ++i) {
+      if (active && G::has(i, ul)) {
+        const bool drop_lo = HP == 1 && i == 0 && ul == 0;
+        const bool drop_hi = HP == 0 && i == G::LAST_I && ul == G::LAST_UL;
+        CodePacker<2> pk;
+        pk.init();
+        pk.add(0, drop_lo ? q.mn : e[i][0], q);
+        pk.add(1, drop_hi ? q.mn : e[i][1], q);  // a dropped element codes as 0
+        uint32_t byte = pk.acc & 0xFFu;
+        if (drop_lo) byte |= p.codes[a0 + ul + UNIT_ * i] & 0x0Fu;  // low nibble: the previous row's
+        p.codes[a0 + ul + UNIT_ * i] = (unsigned char)byte;
+      }
+    }
+  }
+
+  static __device__ __forceinline__ void group(Unit<UNIT_>& u, State&, const StagePtrs& p, float*, uint32_t grp,
+                                               bool active, uint32_t) {
+    const uint32_t r = active ? 2 * grp : 0;
+    row<0>(u, p, r, active);
+    u.sync();  // the odd row reads the shared word and code byte the even row left
+    row<1>(u, p, r + 1, active);
+    u.sync();
+  }
+};
+
+template <int DT, int UNIT_, int LCT>
+struct PairSoftmaxBwd {
+  static constexpr int kKernel = kSoftmaxBwd;
+  static constexpr int UNIT = UNIT_;
+  using P = P2<DT>;
+  using G = PairGeom<UNIT_, LCT>;
+  struct State {};
+  static __device__ __forceinline__ void init(State&) {}
+  static __device__ __forceinline__ uint32_t rows_per_group(uint32_t) { return 2u; }
+
+  template <int HP>
+  static __device__ __forceinline__ void row(Unit<UNIT_>& u, const StagePtrs& p, uint32_t r, bool active) {
+    const uint32_t a0 = (r * (uint32_t)LCT) >> 1;
+    const int ul = u.ul;
+    const float mn = active ? p.meta[2 * r] : 0.0f;
+    const float s = active ? p.meta[2 * r + 1] : 0.0f;
+    float g[G::ITERS][2], yh[G::ITERS][2];
+    float dot = 0.0f;
+#pragma unroll
+    for (int i = 0; i < G::ITERS; ++i) {
+      g[i][0] = 0.0f;
+      g[i][1] = 0.0f;
+      yh[i][0] = 0.0f;
+      yh[i][1] = 0.0f;
+      if (active && G::has(i, ul)) {
+        const typename P::Raw w = P::load(p.data, a0 + ul + UNIT_ * i);
+        const uint32_t b = p.codes[a0 + ul + UNIT_ * i];
+        g[i][0] = P::lo(w);
+        g[i][1] = P::hi(w);
+        yh[i][0] = dequant(b & 0xFu, mn, s);
+        yh[i][1] = dequant(b >> 4, mn, s);
+      }
+      if (HP == 1 && i == 0 && ul == 0) g[i][0] = 0.0f;
+      if (HP == 0 && i == G::LAST_I && ul == G::LAST_UL) g[i][1] = 0.0f;
+      dot = fmaf(g[i][0], yh[i][0], dot);
+      dot = fmaf(g[i][1], yh[i][1], dot);
+    }
+    dot = u.template reduce<kOpSum>(dot);
+#pragma unroll
+    for (int i = 0; i < G::ITERS; ++i) {
+      if (active && G::has(i, ul)) {
+        const typename P::Raw w = P::pack(yh[i][0] * (g[i][0] - dot), yh[i][1] * (g[i][1] - dot));
+        const bool drop_lo = HP == 1 && i == 0 && ul == 0;
+        const bool drop_hi = HP == 0 && i == G::LAST_I && ul == G::LAST_UL;
+        if (drop_lo) P::store_hi(p.data, a0 + ul + UNIT_ * i, w);
+        else if (drop_hi) P::store_lo(p.data, a0 + ul + UNIT_ * i, w);
+        else P::store(p.data, a0 + ul + UNIT_ * i, w);
+      }
+    }
+  }
+
+  static __device__ __forceinline__ void group(Unit<UNIT_>& u, State&, const StagePtrs& p, float*, uint32_t grp,
+                                               bool active, uint32_t) {
+    const uint32_t r = active ? 2 * grp : 0;
+    row<0>(u, p, r, active);
+    u.sync();  // the odd row's first word holds the even row's last result
+    row<1>(u, p, r + 1, active);
+    u.sync();
+  }
+};
+
 // ---------------------------------------------------------------- the kernel
-template <int KERNEL, int DT, int VMODE, int UNIT, int ITERS>
+template <class WORK>
 __global__ void __launch_bounds__(288) tile_kernel(TileKernelArgs a) {
   extern __shared__ __align__(1024) unsigned char smem[];
+  constexpr int KERNEL = WORK::kKernel;
+  constexpr int UNIT = WORK::UNIT;
   constexpr bool kFwd = (KERNEL == kGeluFwd || KERNEL == kSoftmaxFwd);
 
   uint64_t* full = (uint64_t*)smem;                 // [stages]
@@ -590,22 +1149,20 @@ __global__ void __launch_bounds__(288) tile_kernel(TileKernelArgs a) {
   }
 
   // -------------------------------------------------------------- consumer warps
-  using W = RowWork<KERNEL, DT, VMODE, UNIT, ITERS>;
   const int ctid = threadIdx.x;  // consumer warps come first
   Unit<UNIT> u;
   u.ul = ctid % UNIT;
   u.uid = ctid / UNIT;
-  u.red = (float*)(smem + kRedOffset) + u.uid * 4;
+  u.red = (float*)(smem + kRedOffset) + u.uid * 4;  // [slot(2)][16 floats]; unit k owns floats 4k..4k+3
   u.phase = 0;
-  // red layout: [slot(2)][16 floats]; unit k uses floats 4k..4k+3 of each slot
   const uint32_t n_units = (uint32_t)(n_cwarps * 32 / UNIT);
   int* abort_flag = (int*)(smem + kFlagOffset) + (UNIT > 32 ? u.uid : 0);
   float* tab = (float*)(smem + kTabOffset) + u.uid * 16;
-  float tab_mn = __int_as_float(0x7fc00000), tab_s = tab_mn;  // NaN: nothing cached yet
+  typename WORK::State state;
+  WORK::init(state);
 
   const uint32_t L = a.row_len;
-  const uint32_t G = (VMODE == kPair && (L & 1u)) ? 2u : 1u;  // rows handled back to back
-  const uint32_t n_groups = a.tile_rows / G;
+  const uint32_t n_groups = a.tile_rows / WORK::rows_per_group(L);
   const uint32_t rounds = (n_groups + n_units - 1) / n_units;
 
   for (uint64_t it = 0; it < my_tiles; ++it) {
@@ -619,20 +1176,20 @@ __global__ void __launch_bounds__(288) tile_kernel(TileKernelArgs a) {
     }
     if (!ok) break;
     unsigned char* st = smem + kHeaderBytes + (size_t)s * a.stage_bytes;
-    unsigned char* data = st;
-    unsigned char* codes = st + a.code_off;
-    float* meta_s = (float*)(st + a.meta_off);
+    StagePtrs sp{st, st + a.code_off, (float*)(st + a.meta_off)};
     for (uint32_t rd = 0; rd < rounds; ++rd) {
-      const uint32_t grp = rd * n_units + u.uid;
-      const bool active = grp < n_groups;
-      for (uint32_t h = 0; h < G; ++h) {
-        const uint32_t r = active ? grp * G + h : 0;
-        if (KERNEL == kGeluFwd) W::gelu_fwd(u, data, codes, meta_s, r, L, active);
-        if (KERNEL == kSoftmaxFwd) W::softmax_fwd(u, data, codes, meta_s, r, L, active);
-        if (KERNEL == kGeluBwd) W::gelu_bwd(u, data, codes, meta_s, tab, tab_mn, tab_s, r, L, active);
-        if (KERNEL == kSoftmaxBwd) W::softmax_bwd(u, data, codes, meta_s, r, L, active);
-        u.sync();  // the next row may share a word / code byte with this one
+      uint32_t grp = rd * n_units + u.uid;
+      bool active = grp < n_groups;
+      if (UNIT < 32 && a.spread_units) {
+        // the units of one warp take groups n_groups / (units per warp) apart, which for
+        // the odd attention widths puts their words in different shared-memory banks
+        constexpr uint32_t upw = 32 / (UNIT < 32 ? UNIT : 32);
+        const uint32_t per = n_groups / upw;
+        const uint32_t slot = rd * (uint32_t)n_cwarps + (uint32_t)warp;
+        grp = (u.uid % upw) * per + slot;
+        active = slot < per;
       }
+      WORK::group(u, state, sp, tab, grp, active, L);
     }
     fence_proxy_async();  // this thread's shared-memory writes -> visible to the copy engine
     __syncwarp();
@@ -640,65 +1197,115 @@ __global__ void __launch_bounds__(288) tile_kernel(TileKernelArgs a) {
   }
 }
 
+// ---------------------------------------------------------------- launching
 constexpr uint32_t kMaxSmem = 227 * 1024;
 
-// Largest per-lane access count instantiated for an access kind.
-template <int DT, int VMODE>
-constexpr int kMaxIters() { return (DT == kBF16 && VMODE == kVec16) ? 8 : 16; }
-
-template <int KERNEL, int DT, int VMODE, int UNIT, int ITERS>
-cudaError_t launch_inst(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
-  auto kfn = tile_kernel<KERNEL, DT, VMODE, UNIT, ITERS>;
-  static bool configured = false;  // per instantiation; the attribute is per device context
-  static int configured_dev = -1;
+template <class WORK>
+cudaError_t launch_work(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
+  auto kfn = tile_kernel<WORK>;
+  static int configured_dev = -1;  // per instantiation; the attribute belongs to a device's context
   int dev = 0;
   cudaGetDevice(&dev);
-  if (!configured || configured_dev != dev) {
+  if (configured_dev != dev) {
     cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem);
     if (e != cudaSuccess) return e;
-    configured = true;
     configured_dev = dev;
   }
   kfn<<<p.grid, (p.warps + 1) * 32, p.smem_bytes, st>>>(ka);
   return cudaGetLastError();
 }
 
+// The general policy, by unit size and register bound.
 template <int KERNEL, int DT, int VMODE, int UNIT>
-cudaError_t launch_iters(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
+cudaError_t launch_generic_iters(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
+  constexpr int kMax = (DT == kBF16 && VMODE == kVec16) ? 8 : 16;  // elements per lane stay <= 64
   switch (p.iters) {
-    case 1: return launch_inst<KERNEL, DT, VMODE, UNIT, 1>(p, ka, st);
-    case 2: return launch_inst<KERNEL, DT, VMODE, UNIT, 2>(p, ka, st);
-    case 4: return launch_inst<KERNEL, DT, VMODE, UNIT, 4>(p, ka, st);
-    case 8: return launch_inst<KERNEL, DT, VMODE, UNIT, 8>(p, ka, st);
+    case 1: return launch_work<GenericWork<KERNEL, DT, VMODE, UNIT, 1>>(p, ka, st);
+    case 2: return launch_work<GenericWork<KERNEL, DT, VMODE, UNIT, 2>>(p, ka, st);
+    case 4: return launch_work<GenericWork<KERNEL, DT, VMODE, UNIT, 4>>(p, ka, st);
+    case 8: return launch_work<GenericWork<KERNEL, DT, VMODE, UNIT, 8>>(p, ka, st);
     case 16:
-      // 16 accesses of 8 bfloat16 would be 128 elements per lane: not instantiated
-      if (kMaxIters<DT, VMODE>() >= 16) return launch_inst<KERNEL, DT, VMODE, UNIT, kMaxIters<DT, VMODE>() >= 16 ? 16 : 8>(p, ka, st);
-  }
-  return cudaErrorInvalidValue;
-}
-
-template <int KERNEL, int DT, int VMODE>
-cudaError_t launch_unit(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
-  switch (p.unit_lanes) {
-    case 8: return launch_iters<KERNEL, DT, VMODE, 8>(p, ka, st);
-    case 16: return launch_iters<KERNEL, DT, VMODE, 16>(p, ka, st);
-    case 32: return launch_iters<KERNEL, DT, VMODE, 32>(p, ka, st);
-    case 128: return launch_iters<KERNEL, DT, VMODE, 128>(p, ka, st);
+      if (kMax >= 16) return launch_work<GenericWork<KERNEL, DT, VMODE, UNIT, kMax>>(p, ka, st);
   }
   return cudaErrorInvalidValue;
 }
 
 template <int KERNEL, int DT>
-cudaError_t launch_vmode(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
-  return p.vec_elems == 2 ? launch_unit<KERNEL, DT, kPair>(p, ka, st)
-                          : launch_unit<KERNEL, DT, kVec16>(p, ka, st);
+cudaError_t launch_generic(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
+  if (p.vec_elems == 2) {
+    switch (p.unit_lanes) {
+      case 8: return launch_generic_iters<KERNEL, DT, kPair, 8>(p, ka, st);
+      case 32: return launch_generic_iters<KERNEL, DT, kPair, 32>(p, ka, st);
+    }
+  } else if constexpr (KERNEL == kSoftmaxFwd || KERNEL == kSoftmaxBwd) {
+    if (p.unit_lanes == 128) return launch_generic_iters<KERNEL, DT, kVec16, 128>(p, ka, st);
+  }
+  return cudaErrorInvalidValue;
 }
 
+template <template <int, int, int> class WORK, int DT, int UNIT>
+cudaError_t launch_softmax_nv(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
+  switch (p.iters) {
+    case 1: return launch_work<WORK<DT, UNIT, 1>>(p, ka, st);
+    case 2: return launch_work<WORK<DT, UNIT, 2>>(p, ka, st);
+    case 4: return launch_work<WORK<DT, UNIT, 4>>(p, ka, st);
+    case 8: return launch_work<WORK<DT, UNIT, 8>>(p, ka, st);
+    case 16:
+      if (DT == kF32) return launch_work<WORK<DT, UNIT, DT == kF32 ? 16 : 8>>(p, ka, st);
+  }
+  return cudaErrorInvalidValue;
+}
+
+template <template <int, int, int> class WORK, int DT>
+cudaError_t launch_softmax_stream(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
+  switch (p.unit_lanes) {
+    case 8: return launch_softmax_nv<WORK, DT, 8>(p, ka, st);
+    case 16: return launch_softmax_nv<WORK, DT, 16>(p, ka, st);
+    case 32: return launch_softmax_nv<WORK, DT, 32>(p, ka, st);
+  }
+  return cudaErrorInvalidValue;
+}
+
+template <template <int, int> class WORK, int DT>
+cudaError_t launch_gelu_stream(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
+  switch (p.unit_lanes) {
+    case 8: return launch_work<WORK<DT, 8>>(p, ka, st);
+    case 16: return launch_work<WORK<DT, 16>>(p, ka, st);
+    case 32: return launch_work<WORK<DT, 32>>(p, ka, st);
+  }
+  return cudaErrorInvalidValue;
+}
+
+template <template <int, int, int> class WORK, int DT>
+cudaError_t launch_pair_fixed(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
+  if (p.unit_lanes != 8) return cudaErrorInvalidValue;
+  switch (ka.row_len) {
+    case 197: return launch_work<WORK<DT, 8, 197>>(p, ka, st);
+    case 257: return launch_work<WORK<DT, 8, 257>>(p, ka, st);
+  }
+  return cudaErrorInvalidValue;
+}
+
+template <int KERNEL, int DT>
+cudaError_t launch_variant(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
+  if (p.variant == kVariantStream) {
+    if constexpr (KERNEL == kGeluFwd) return launch_gelu_stream<StreamGeluFwd, DT>(p, ka, st);
+    if constexpr (KERNEL == kGeluBwd) return launch_gelu_stream<StreamGeluBwd, DT>(p, ka, st);
+    if constexpr (KERNEL == kSoftmaxFwd) return launch_softmax_stream<StreamSoftmaxFwd, DT>(p, ka, st);
+    if constexpr (KERNEL == kSoftmaxBwd) return launch_softmax_stream<StreamSoftmaxBwd, DT>(p, ka, st);
+  }
+  if (p.variant == kVariantPairFixed) {
+    if constexpr (KERNEL == kSoftmaxFwd) return launch_pair_fixed<PairSoftmaxFwd, DT>(p, ka, st);
+    if constexpr (KERNEL == kSoftmaxBwd) return launch_pair_fixed<PairSoftmaxBwd, DT>(p, ka, st);
+    return cudaErrorInvalidValue;
+  }
+  return launch_generic<KERNEL, DT>(p, ka, st);
+}
 
 // One translation unit per entry point instantiates this.
 template <int KERNEL>
 cudaError_t launch_tile_kernel(int dt, const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
-  return dt == kF32 ? launch_vmode<KERNEL, kF32>(p, ka, st) : launch_vmode<KERNEL, kBF16>(p, ka, st);
+  return dt == kF32 ? launch_variant<KERNEL, kF32>(p, ka, st) : launch_variant<KERNEL, kBF16>(p, ka, st);
 }
 
 }  // namespace

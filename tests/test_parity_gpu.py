@@ -111,6 +111,8 @@ def test_in_place(dt):
 def test_benchmark_shapes_take_the_pipelined_path():
     for sh in (synth.VIT_B16_B8_F32, synth.VIT_B16_B64, synth.VIT_L16_B64, synth.VIT_H14_B32):
         for kernel in range(4):
+            if kernel >= 2 and sh is synth.VIT_B16_B8_F32:
+                continue  # the single-layer workload is GELU only
             n, L = (sh.gelu_elems, sh.hidden) if kernel < 2 else (sh.softmax_elems, sh.tokens)
             plan = binding.s2a_describe_plan(kernel, n, L, sh.dtype)
             assert plan.startswith("tile") and plan.endswith("tail_rows=0"), plan
