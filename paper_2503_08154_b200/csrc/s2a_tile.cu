@@ -83,8 +83,8 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L) {
   if (vec16 && !force_generic && is_gelu) {
     // streamed: nothing held in registers; a warp per row unless the row is short
     variant = kVariantStream;
-    unit = n_acc >= 32 ? 32u : (n_acc >= 16 ? 16u : 8u);
-    if (env_unit == 8 || env_unit == 16 || env_unit == 32) unit = (uint32_t)env_unit;
+    unit = n_acc >= 256 ? 64u : (n_acc >= 32 ? 32u : (n_acc >= 16 ? 16u : 8u));
+    if (env_unit == 8 || env_unit == 16 || env_unit == 32 || env_unit == 64 || env_unit == 128) unit = (uint32_t)env_unit;
   } else if (vec16 && !force_generic) {
     // softmax on 16-byte vectors: up to 32 (at most 64) elements per lane in registers
     const uint32_t cap = 32u / epa, cap2 = 64u / epa;
@@ -123,8 +123,11 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L) {
   }
 
   uint32_t warps = unit == 128 ? 8u : 4u;
+  int ctas_per_sm = 2;
+  if (variant == kVariantStream && is_gelu) ctas_per_sm = 4;
+  if (variant == kVariantPairFixed) ctas_per_sm = 4;
   warps = (uint32_t)env_int("S2A_WARPS", (int)warps);
-  if (warps < 1 || warps > 8 || (warps * 32) % unit != 0) return p;
+  if (warps < 1 || warps > 16 || (warps * 32) % unit != 0) return p;
   const uint32_t n_units = warps * 32 / unit;
   const uint32_t G = (!vec16 && (L & 1u)) ? 2u : 1u;
 
@@ -134,7 +137,10 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L) {
   const uint32_t want_rows = n_units * G;
   while (rows % want_rows != 0 && (uint64_t)(rows + r_min) * L * esize <= kMaxStageBytes) rows += r_min;
   while ((uint64_t)rows * L * esize < 16 * 1024 && (uint64_t)rows * 2 * L * esize <= kMaxStageBytes) rows *= 2;
-  if (variant == kVariantPairFixed && rows < 64 && (uint64_t)64 * L * esize <= kMaxStageBytes) rows = 64;
+  if ((variant == kVariantStream && is_gelu) || variant == kVariantPairFixed) {
+    rows = r_min;  // small tiles: more CTAs per SM, each with its own pipeline
+    while (rows % (n_units * G) != 0 && (uint64_t)(rows + r_min) * L * esize <= kMaxStageBytes) rows += r_min;
+  }
   rows = (uint32_t)env_int("S2A_TILE_ROWS", (int)rows);
   if (rows == 0 || rows % r_min != 0 || (uint64_t)rows * L * esize > kMaxStageBytes) return p;
 
@@ -145,21 +151,23 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L) {
   const uint32_t meta_off = code_off + align_up(code_bytes, 128);
   const uint32_t stage_bytes = meta_off + align_up(meta_bytes, 128);
 
-  int ctas_per_sm = env_int("S2A_CTAS_PER_SM", 2);
+  // CTAs per SM and stages per CTA: the wanted CTA count if it leaves room for 3 stages,
+  // else fewer CTAs; 2 stages only as a last resort
+  ctas_per_sm = env_int("S2A_CTAS_PER_SM", ctas_per_sm);
   if (ctas_per_sm < 1) ctas_per_sm = 1;
-  uint32_t budget = kMaxSmem / (uint32_t)ctas_per_sm - 1024;
-  uint32_t stages = (budget - kHeaderBytes) / stage_bytes;
-  if (stages > 4) stages = 4;
-  stages = (uint32_t)env_int("S2A_STAGES", (int)stages);
-  if (stages > (uint32_t)kMaxStages) stages = kMaxStages;
-  if (stages < 2) {
-    ctas_per_sm = 1;
-    stages = (kMaxSmem - kHeaderBytes) / stage_bytes;
-    if (stages > 4) stages = 4;
-    if (stages < 2) return p;
+  const int env_stages = env_int("S2A_STAGES", 0);
+  uint32_t stages = 0;
+  int chosen = 0;
+  for (int pass = 0; pass < 2 && chosen == 0; ++pass) {
+    const uint32_t want = env_stages > 0 ? (uint32_t)env_stages : (pass == 0 ? 3u : 2u);
+    for (int c = ctas_per_sm; c >= 1 && chosen == 0; --c) {
+      const uint32_t budget = kMaxSmem / (uint32_t)c - 1024;
+      if (budget >= kHeaderBytes + want * stage_bytes) { chosen = c; stages = want; }
+    }
   }
+  if (chosen == 0 || stages > (uint32_t)kMaxStages) return p;
+  ctas_per_sm = chosen;
   const uint32_t smem = kHeaderBytes + stages * stage_bytes;
-  if (smem > kMaxSmem) return p;
 
   p.n_tiles = n_rows / rows;
   if (p.n_tiles == 0) return TilePlan{};

@@ -29,8 +29,8 @@ namespace {
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr int kMaxStages = 8;
 constexpr int kHeaderBytes = 4096;  // barriers, reduction scratch, derivative tables
-constexpr int kRedOffset = 256;     // float[2 slots][4 units][4 warps]  (multi-warp units)
-constexpr int kFlagOffset = 768;    // int[4]: abort flag per multi-warp unit
+constexpr int kRedOffset = 256;     // float[2 slots][16 units][4 warps]  (multi-warp units)
+constexpr int kFlagOffset = 768;    // int[16]: abort flag per multi-warp unit
 constexpr int kTabOffset = 1024;    // float[units][16]: Eq. 12 table per unit (<= 32 units)
 
 enum { kVec16 = 0, kPair = 1 };
@@ -80,10 +80,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait for the phase with the given parity to complete.
+// Bounded wait for the phase with the given parity to complete.  SLEEP_NS > 0 backs off
+// between tries (used by the copy lane, which would otherwise take issue slots from the
+// warps it is waiting for).
+template <int SLEEP_NS = 0>
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned int* err, unsigned err_bit) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i)
+  for (uint32_t i = 0; i < kSpinLimit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
+    if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
+  }
   atomicOr(err, err_bit);
   return false;
 }
@@ -254,7 +259,7 @@ struct Unit {
     for (int o = W / 2; o > 0; o >>= 1) v = op2<OP>(v, __shfl_xor_sync(0xffffffffu, v, o));
     if (UNIT > 32) {
       constexpr int NW = UNIT / 32;
-      float* slot = red + (phase & 1) * 16;
+      float* slot = red + (phase & 1) * 64;
       if ((ul & 31) == 0) slot[ul >> 5] = v;
       named_bar_sync(1 + uid, UNIT);
       v = slot[0];
@@ -301,23 +306,22 @@ __device__ __forceinline__ RowGeom row_geom(uint32_t r, uint32_t L) {
 // Fast sigmoid-GELU pieces for the bfloat16 path (result is rounded to 8 bits).
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
-  asm("ex2.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
 __device__ __forceinline__ float rcp_approx(float x) {
   float y;
-  asm("rcp.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
 
 template <int DT>
 __device__ __forceinline__ float gelu_eval(float x) {
   if (DT == kF32) return gelu_value(x);
-  // t = exp(-|1.702 x|); y = (z >= 0 ? x : x t) / (1 + t)
-  const float z = kSlope * x;
-  const float t = ex2_approx(-1.4426950408889634f * fabsf(z));
-  const float num = z >= 0.0f ? x : x * t;
-  return num * rcp_approx(1.0f + t);
+  // y = x / (1 + 2^(-1.702 log2(e) x)).  For x < -52 the power overflows and y becomes
+  // -0 instead of a value below 2^-120: the bfloat16 path flushes such results.
+  constexpr float c = -1.702f * 1.4426950408889634f;
+  return x * rcp_approx(1.0f + ex2_approx(c * x));
 }
 
 template <int DT>
@@ -533,6 +537,7 @@ struct StagePtrs {
 template <int KERNEL, int DT, int VMODE, int UNIT_, int ITERS>
 struct GenericWork {
   static constexpr int kKernel = KERNEL;
+  static constexpr int kMaxRegs = 128;
   static constexpr int UNIT = UNIT_;
   using W = RowWork<KERNEL, DT, VMODE, UNIT_, ITERS>;
   struct State {
@@ -658,6 +663,7 @@ struct CodePacker {
 
 template <int DT, int UNIT_>
 struct StreamGeluFwd {
+  static constexpr int kMaxRegs = 64;
   static constexpr int kKernel = kGeluFwd;
   static constexpr int UNIT = UNIT_;
   using V = V16<DT>;
@@ -701,6 +707,7 @@ struct StreamGeluFwd {
 // read them from a shared-memory table.
 template <int DT, int UNIT_>
 struct StreamGeluBwd {
+  static constexpr int kMaxRegs = 64;
   static constexpr int kKernel = kGeluBwd;
   static constexpr int UNIT = UNIT_;
   using V = V16<DT>;
@@ -720,7 +727,7 @@ struct StreamGeluBwd {
     const float s = active ? p.meta[2 * r + 1] : st.tab_s;
     // The 16 values of Eq. 12 this row can take, in binary64; kept while (min, s) repeat.
     if (mn != st.tab_mn || s != st.tab_s) {
-      if (UNIT_ == 32) {
+      if (UNIT_ >= 32) {
         st.d = (float)gelu_sine_derivative((uint32_t)(u.ul & 15), mn, s);
       } else {
 #pragma unroll
@@ -732,7 +739,7 @@ struct StreamGeluBwd {
       st.tab_mn = mn;
       st.tab_s = s;
     }
-    if (UNIT_ != 32) u.sync();
+    if (UNIT_ < 32) u.sync();
     const uint32_t nv = active ? L / V::EPA : 0u;
     unsigned char* row = p.data + (size_t)r * L * Io<DT>::kBytes;
     const unsigned char* crow = p.codes + (size_t)r * (L / 2);
@@ -751,7 +758,7 @@ struct StreamGeluBwd {
 #pragma unroll
       for (int k = 0; k < V::EPA; ++k) {
         float d;
-        if (UNIT_ == 32) d = __shfl_sync(0xffffffffu, st.d, (int)(bits >> (4 * k)));  // lane = code mod 16 (+16)
+        if (UNIT_ >= 32) d = __shfl_sync(0xffffffffu, st.d, (int)(bits >> (4 * k)));  // lane = code mod 16 (+16)
         else d = tab[(bits >> (4 * k)) & 0xFu];
         v[k] *= d;
       }
@@ -763,6 +770,7 @@ struct StreamGeluBwd {
 // Softmax forward on 16-byte vectors, NV vectors per lane kept in registers.
 template <int DT, int UNIT_, int NV>
 struct StreamSoftmaxFwd {
+  static constexpr int kMaxRegs = NV * V16<DT>::EPA >= 32 ? 128 : 80;
   static constexpr int kKernel = kSoftmaxFwd;
   static constexpr int UNIT = UNIT_;
   using V = V16<DT>;
@@ -834,6 +842,7 @@ struct StreamSoftmaxFwd {
 
 template <int DT, int UNIT_, int NV>
 struct StreamSoftmaxBwd {
+  static constexpr int kMaxRegs = NV * V16<DT>::EPA >= 32 ? 128 : 80;
   static constexpr int kKernel = kSoftmaxBwd;
   static constexpr int UNIT = UNIT_;
   using V = V16<DT>;
@@ -926,6 +935,7 @@ struct PairGeom {
 
 template <int DT, int UNIT_, int LCT>
 struct PairSoftmaxFwd {
+  static constexpr int kMaxRegs = 104;
   static constexpr int kKernel = kSoftmaxFwd;
   static constexpr int UNIT = UNIT_;
   using P = P2<DT>;
@@ -1016,6 +1026,7 @@ struct PairSoftmaxFwd {
 
 template <int DT, int UNIT_, int LCT>
 struct PairSoftmaxBwd {
+  static constexpr int kMaxRegs = 104;
   static constexpr int kKernel = kSoftmaxBwd;
   static constexpr int UNIT = UNIT_;
   using P = P2<DT>;
@@ -1077,7 +1088,7 @@ struct PairSoftmaxBwd {
 
 // ---------------------------------------------------------------- the kernel
 template <class WORK>
-__global__ void __launch_bounds__(288) tile_kernel(TileKernelArgs a) {
+__global__ void __maxnreg__(WORK::kMaxRegs) tile_kernel(TileKernelArgs a) {
   extern __shared__ __align__(1024) unsigned char smem[];
   constexpr int KERNEL = WORK::kKernel;
   constexpr int UNIT = WORK::UNIT;
@@ -1097,7 +1108,7 @@ __global__ void __launch_bounds__(288) tile_kernel(TileKernelArgs a) {
       mbar_init(&done[s], (uint32_t)n_cwarps);
     }
     int* flags = (int*)(smem + kFlagOffset);
-    for (int k = 0; k < 4; ++k) flags[k] = 0;
+    for (int k = 0; k < 16; ++k) flags[k] = 0;
     fence_barrier_init();
   }
   __syncthreads();
@@ -1124,7 +1135,7 @@ __global__ void __launch_bounds__(288) tile_kernel(TileKernelArgs a) {
     uint64_t it = 0;
     bool ok = true;
     for (; it < my_tiles; ++it) {
-      if (!mbar_wait(&done[it % S], (uint32_t)((it / S) & 1), a.error_word, kErrDrainWait)) { ok = false; break; }
+      if (!mbar_wait<200>(&done[it % S], (uint32_t)((it / S) & 1), a.error_word, kErrDrainWait)) { ok = false; break; }
       const uint64_t t = blockIdx.x + it * gridDim.x;
       unsigned char* st = stage_ptr(it);
       bulk_store(a.out + t * a.data_bytes, st, a.data_bytes);
@@ -1133,9 +1144,9 @@ __global__ void __launch_bounds__(288) tile_kernel(TileKernelArgs a) {
         bulk_store(a.meta + t * a.meta_bytes, st + a.meta_off, a.meta_bytes);
       }
       bulk_commit();
-      if (it >= 1 && issued < my_tiles) {
-        bulk_wait_read<1>();  // the stores of tile it-1 have left shared memory
-        issue_load(issued);   // == it - 1 + S: refills the stage of tile it-1
+      if (issued < my_tiles) {
+        bulk_wait_read<0>();  // the stores of this tile have left shared memory
+        issue_load(issued);   // == it + S: refills the stage just drained
         ++issued;
       }
     }
@@ -1153,7 +1164,7 @@ __global__ void __launch_bounds__(288) tile_kernel(TileKernelArgs a) {
   Unit<UNIT> u;
   u.ul = ctid % UNIT;
   u.uid = ctid / UNIT;
-  u.red = (float*)(smem + kRedOffset) + u.uid * 4;  // [slot(2)][16 floats]; unit k owns floats 4k..4k+3
+  u.red = (float*)(smem + kRedOffset) + u.uid * 4;  // [slot(2)][64 floats]; unit k owns floats 4k..4k+3
   u.phase = 0;
   const uint32_t n_units = (uint32_t)(n_cwarps * 32 / UNIT);
   int* abort_flag = (int*)(smem + kFlagOffset) + (UNIT > 32 ? u.uid : 0);
@@ -1272,6 +1283,8 @@ cudaError_t launch_gelu_stream(const TilePlan& p, const TileKernelArgs& ka, cuda
     case 8: return launch_work<WORK<DT, 8>>(p, ka, st);
     case 16: return launch_work<WORK<DT, 16>>(p, ka, st);
     case 32: return launch_work<WORK<DT, 32>>(p, ka, st);
+    case 64: return launch_work<WORK<DT, 64>>(p, ka, st);
+    case 128: return launch_work<WORK<DT, 128>>(p, ka, st);
   }
   return cudaErrorInvalidValue;
 }
