@@ -187,40 +187,54 @@ def stored_traffic(kernel, workload):
 
 
 # ------------------------------------------------------------------ the CPU oracle legs
-def oracle_sample_rate(shape, seed, threads):
-    """Times the oracle, as it stands, on one block's worth of rows (bounded sample)."""
+def oracle_time_block(shape, arrays, threads):
+    """Forward+backward of both nonlinearities through the oracle on one block's arrays.
+    Returns (algorithmic bytes, elements, seconds)."""
     from oracle import s2a_oracle as o
-    has_softmax = shape.name != synth.VIT_B16_B8_F32.name
+    gx, gg, sx, sg = arrays
     item = synth.io_itemsize(shape.dtype)
-    rows_g = min(shape.gelu_rows, max(1, 12_000_000 // shape.hidden))
-    rows_s = min(shape.softmax_rows, max(1, 12_000_000 // shape.tokens))
-    gx, gg, sx, sg = host_inputs(shape, 1, seed, rows_g, rows_s, has_softmax)[0]
-    o.lib()
     t0 = time.perf_counter()
     y, c, m = o.gelu_fwd(gx, shape.hidden, shape.dtype, threads)
     o.gelu_bwd(gg, c, m, shape.hidden, shape.dtype, threads)
     nbytes = 2 * algorithmic_bytes(gx.size, shape.hidden, item)
     nelem = gx.size
-    if has_softmax:
+    if sx is not None:
         y, c, m = o.softmax_fwd(sx, shape.tokens, shape.dtype, threads)
         o.softmax_bwd(sg, c, m, shape.tokens, shape.dtype, threads)
         nbytes += 2 * algorithmic_bytes(sx.size, shape.tokens, item)
         nelem += sx.size
-    dt = time.perf_counter() - t0
-    sample = "fwd+bwd on the first %d GELU rows%s of block 0" % (
-        rows_g, (" and %d softmax rows" % rows_s) if has_softmax else "")
-    return nbytes / dt / 1e9, nelem / dt / 1e9, dt, sample
+    return nbytes, nelem, time.perf_counter() - t0
+
+
+def oracle_sample_rate(shape, blocks_arrays, threads, core_seconds=12.0):
+    """Times the oracle, as it stands, on whole blocks of the workload until about
+    `core_seconds` of CPU work (threads x wall time) have been spent."""
+    from oracle import s2a_oracle as o
+    o.lib()
+    nbytes = nelem = 0
+    secs = 0.0
+    used = 0
+    for arrays in blocks_arrays:
+        b, e, t = oracle_time_block(shape, arrays, threads)
+        nbytes, nelem, secs, used = nbytes + b, nelem + e, secs + t, used + 1
+        if secs * threads >= core_seconds:
+            break
+    sample = "fwd+bwd of GELU%s on %d of the workload's blocks, full size (%.1f core-seconds)" % (
+        " and softmax" if blocks_arrays[0][2] is not None else "", used, secs * threads)
+    return nbytes / secs / 1e9, nelem / secs / 1e9, secs, sample
 
 
 def run_reference(args, shape, blocks):
     """--impl reference: the oracle on the host cores, each step a bounded sample."""
     from oracle import s2a_oracle as o
     threads = o.hardware_threads()
+    has_softmax = shape.name != synth.VIT_B16_B8_F32.name
+    arrays = host_inputs(shape, 1, args.seed, with_softmax=has_softmax)
     rates = []
     t_all = time.perf_counter()
     sample = ""
     for i in range(args.warmup + args.steps):
-        gbs, gel, dt, sample = oracle_sample_rate(shape, args.seed, threads)
+        gbs, gel, dt, sample = oracle_sample_rate(shape, arrays, threads, core_seconds=0.0)
         if i >= args.warmup:
             rates.append((gbs, gel, dt))
         if time.perf_counter() - t_all > 150 and len(rates) >= 1:
@@ -317,32 +331,58 @@ def run_ours(args, shape, blocks, rank, world):
     if binding.s2a_device_error() != 0:
         raise RuntimeError("a kernel gave up on a bounded wait during warm-up")
 
-    # ---- timed region: K steps, an event before every launch and one at the end
+    # ---- timed region: K steps back to back, one event on the stream at each end.  (An
+    # event between two launches would defeat programmatic dependent launch, so the
+    # per-kernel figures are taken in separate loops below.)
     n_calls = len(calls)
-    events = [[torch.cuda.Event(enable_timing=True) for _ in range(n_calls + 1)] for _ in range(args.steps)]
     sampler = ClockSampler(getattr(torch.cuda.get_device_properties(local), "uuid", ""), local)
     sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     t0 = time.perf_counter()
+    ev0.record(stream)
     for k in range(args.steps):
-        ev = events[k]
-        for i, (_, fn, a) in enumerate(calls):
-            ev[i].record(stream)
-            rc = fn(*a)
-            if rc:
-                raise RuntimeError(binding.status_string(rc))
-        ev[n_calls].record(stream)
+        step()
+    ev1.record(stream)
     barrier()
     t1 = time.perf_counter()
     clocks = sampler.finish(t0, t1)
-    total_ms = events[0][0].elapsed_time(events[-1][n_calls])
+    total_ms = ev0.elapsed_time(ev1)
     if binding.s2a_device_error() != 0:
         raise RuntimeError("a kernel gave up on a bounded wait during the timed region")
 
-    per_kernel_ms = {k: [] for k in per_launch}
+    # ---- per kernel: the same launches grouped by kernel, K * blocks back to back
+    per_kernel_ms = {}
+    for name in per_launch:
+        mine = [(fn, a) for n_, fn, a in calls if n_ == name]
+        for fn, a in mine:
+            fn(*a)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(stream)
+        for k in range(args.steps):
+            for fn, a in mine:
+                fn(*a)
+        e1.record(stream)
+        barrier()
+        per_kernel_ms[name] = e0.elapsed_time(e1) / (args.steps * len(mine))
+
+    # ---- per kernel with an event before every launch of a step (for comparison: this
+    # serialises the launches and adds the event's own cost to each)
+    bracket_steps = min(args.steps, 20)
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(n_calls + 1)] for _ in range(bracket_steps)]
+    barrier()
+    for k in range(bracket_steps):
+        ev = events[k]
+        for i, (_, fn, a) in enumerate(calls):
+            ev[i].record(stream)
+            fn(*a)
+        ev[n_calls].record(stream)
+    barrier()
+    bracketed_ms = {k: [] for k in per_launch}
     for ev in events:
         for i, (name, _, _) in enumerate(calls):
-            per_kernel_ms[name].append(ev[i].elapsed_time(ev[i + 1]))
+            bracketed_ms[name].append(ev[i].elapsed_time(ev[i + 1]))
 
     if world > 1:
         t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
@@ -396,14 +436,16 @@ def run_ours(args, shape, blocks, rank, world):
 
     peak, peak_kind = measured_peak()
     per_kernel = {}
-    for k, ms in per_kernel_ms.items():
-        avg = statistics.mean(ms)
+    step_ms = total_ms / args.steps
+    for k, avg in per_kernel_ms.items():
         gbs = per_launch[k] / (avg * 1e-3) / 1e9
-        per_kernel[k] = {"avg_ms": avg, "launches": len(ms), "algorithmic_bytes": per_launch[k], "GBps": gbs,
+        per_kernel[k] = {"avg_ms": avg, "launches_per_step": blocks, "algorithmic_bytes": per_launch[k], "GBps": gbs,
                          "gelem_per_s": elems[k] / (avg * 1e-3) / 1e9, "frac_of_%s_peak" % peak_kind: gbs / peak,
-                         "frac_of_8TBps": gbs / NOMINAL_HBM_GBS, "share_of_step": sum(ms) / (total_ms)}
+                         "frac_of_8TBps": gbs / NOMINAL_HBM_GBS, "share_of_step": avg * blocks / step_ms,
+                         "avg_ms_event_bracketed": statistics.mean(bracketed_ms[k])}
     dominant = max(per_kernel, key=lambda k: per_kernel[k]["share_of_step"])
     roofline = {"bound": "hbm", "kernel": "s2a_" + dominant, "achieved": per_kernel[dominant]["GBps"], "peak": peak,
+                "timing": "CUDA events around %d back-to-back launches of this kernel over the step's %d blocks" % (args.steps * blocks, blocks),
                 "peak_source": "%s copy bandwidth" % peak_kind, "unit": "GB/s",
                 "frac": per_kernel[dominant]["GBps"] / peak, "traffic": stored_traffic(dominant, shape.name)}
 
@@ -412,7 +454,11 @@ def run_ours(args, shape, blocks, rank, world):
     if not args.skip_cpu_baseline:
         from oracle import s2a_oracle as o
         threads = o.hardware_threads()
-        gbs, gel, dtc_s, sample = oracle_sample_rate(shape, args.seed, threads)
+        np_blocks = []
+        for blk in host:
+            np_blocks.append(tuple(None if t is None else (t.numpy().view(np.uint16) if t.dtype == torch.int16 else t.numpy())
+                                   for t in blk))
+        gbs, gel, dtc_s, sample = oracle_sample_rate(shape, np_blocks, threads)
         cpu_baseline = {"value": gbs, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": sample,
                         "gelem_per_s": gel, "seconds": dtc_s}
 

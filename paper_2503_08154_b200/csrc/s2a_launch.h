@@ -40,6 +40,7 @@ struct TilePlan {
   uint32_t smem_bytes;  // dynamic shared memory per CTA
   uint32_t grid;        // CTAs launched
   uint64_t n_tiles;     // full tiles covered; remaining rows go to the row-at-a-time path
+  uint32_t overlap_launch;  // 1: launched with programmatic stream serialization
 };
 
 struct TileArgs {

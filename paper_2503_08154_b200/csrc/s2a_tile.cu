@@ -60,7 +60,7 @@ unsigned int* error_word_address() {
 
 // Launch-shape policy.  Environment overrides (for tuning sweeps): S2A_PATH=rowwise
 // disables this path; S2A_UNIT, S2A_TILE_ROWS, S2A_WARPS, S2A_STAGES, S2A_CTAS_PER_SM,
-// S2A_VARIANT=generic.
+// S2A_VARIANT=generic, S2A_FIXED=0, S2A_PDL=0.
 TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L) {
   TilePlan p{};
   const char* path = getenv("S2A_PATH");
@@ -84,7 +84,12 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L) {
     // streamed: nothing held in registers; a warp per row unless the row is short
     variant = kVariantStream;
     unit = n_acc >= 256 ? 64u : (n_acc >= 32 ? 32u : (n_acc >= 16 ? 16u : 8u));
+    if (dt == kF32 && n_acc >= 512) unit = 128;  // the same vectors per lane as bfloat16 with 64
     if (env_unit == 8 || env_unit == 16 || env_unit == 32 || env_unit == 64 || env_unit == 128) unit = (uint32_t)env_unit;
+    // a fixed vector count per lane (6, 8 or 10) when the row length allows it
+    if (unit >= 64 && n_acc % unit == 0 && (n_acc / unit == 6 || n_acc / unit == 8 || n_acc / unit == 10) &&
+        env_int("S2A_FIXED", 1) != 0)
+      iters = n_acc / unit;
   } else if (vec16 && !force_generic) {
     // softmax on 16-byte vectors: up to 32 (at most 64) elements per lane in registers
     const uint32_t cap = 32u / epa, cap2 = 64u / epa;
@@ -182,6 +187,7 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L) {
   uint64_t grid = (uint64_t)sm_count() * (uint32_t)ctas_per_sm;
   if (grid > p.n_tiles) grid = p.n_tiles;
   p.grid = (uint32_t)grid;
+  p.overlap_launch = env_int("S2A_PDL", 1) != 0 ? 1u : 0u;
   return p;
 }
 

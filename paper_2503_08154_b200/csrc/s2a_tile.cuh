@@ -123,6 +123,15 @@ __device__ __forceinline__ void bulk_wait_read() {
 __device__ __forceinline__ void bulk_wait_all() {
   asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
+// Programmatic dependent launch: the next kernel of the stream may be scheduled while
+// this one drains, and parks at grid_dependency_wait() until this one has completed and
+// its writes are visible.  Both are no-ops for a kernel launched without the attribute.
+__device__ __forceinline__ void grid_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void grid_dependency_wait() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
 __device__ __forceinline__ void named_bar_sync(int id, int threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
@@ -661,7 +670,9 @@ struct CodePacker {
   }
 };
 
-template <int DT, int UNIT_>
+// NVL > 0 fixes the number of vectors per lane (row_len == NVL * UNIT * EPA), which lets
+// the compiler drop every loop counter and bound check; NVL == 0 is the general loop.
+template <int DT, int UNIT_, int NVL>
 struct StreamGeluFwd {
   static constexpr int kMaxRegs = 64;
   static constexpr int kKernel = kGeluFwd;
@@ -671,33 +682,46 @@ struct StreamGeluFwd {
   static __device__ __forceinline__ void init(State&) {}
   static __device__ __forceinline__ uint32_t rows_per_group(uint32_t) { return 1u; }
 
+  static __device__ __forceinline__ void vec(unsigned char* row, unsigned char* crow, uint32_t j, const QRange& q) {
+    float v[V::EPA];
+    V::widen(*(const typename V::Raw*)(row + j * 16u), v);
+    CodePacker<V::EPA> pk;
+    pk.init();
+#pragma unroll
+    for (int k = 0; k < V::EPA; ++k) {
+      pk.add(k, fminf(fmaxf(v[k], -kClip), kClip), q);
+      v[k] = gelu_eval<DT>(v[k]);
+    }
+    *(typename V::Raw*)(row + j * 16u) = V::narrow(v);
+    V::store_codes(crow, j, pk.acc);
+  }
+
   static __device__ __forceinline__ void group(Unit<UNIT_>& u, State&, const StagePtrs& p, float*, uint32_t r,
                                                bool active, uint32_t L) {
+    if (UNIT_ >= 32 && !active) return;  // whole warps leave together
     const uint32_t nv = active ? L / V::EPA : 0u;
     unsigned char* row = p.data + (size_t)r * L * Io<DT>::kBytes;
     unsigned char* crow = p.codes + (size_t)r * (L / 2);
     typename V::MinMax mm;
     mm.init();
+    if (NVL > 0) {
+#pragma unroll
+      for (int i = 0; i < NVL; ++i) mm.add(*(const typename V::Raw*)(row + (u.ul + UNIT_ * i) * 16u));
+    } else {
 #pragma unroll 4
-    for (uint32_t j = u.ul; j < nv; j += UNIT_) mm.add(*(const typename V::Raw*)(row + j * 16u));
+      for (uint32_t j = u.ul; j < nv; j += UNIT_) mm.add(*(const typename V::Raw*)(row + j * 16u));
+    }
     const float mn = u.template reduce<kOpMin>(mm.lo());
     const float mx = u.template reduce<kOpMax>(mm.hi());
     // min / max of the clipped row = clipped min / max of the row (the clip is monotone)
     const QRange q = make_qrange(fminf(fmaxf(mn, -kClip), kClip), fminf(fmaxf(mx, -kClip), kClip));
     if (active && u.ul == 0) { p.meta[2 * r] = q.mn; p.meta[2 * r + 1] = q.s; }
-#pragma unroll 2
-    for (uint32_t j = u.ul; j < nv; j += UNIT_) {
-      float v[V::EPA];
-      V::widen(*(const typename V::Raw*)(row + j * 16u), v);
-      CodePacker<V::EPA> pk;
-      pk.init();
+    if (NVL > 0) {
 #pragma unroll
-      for (int k = 0; k < V::EPA; ++k) {
-        pk.add(k, fminf(fmaxf(v[k], -kClip), kClip), q);
-        v[k] = gelu_eval<DT>(v[k]);
-      }
-      *(typename V::Raw*)(row + j * 16u) = V::narrow(v);
-      V::store_codes(crow, j, pk.acc);
+      for (int i = 0; i < NVL; ++i) vec(row, crow, u.ul + UNIT_ * i, q);
+    } else {
+#pragma unroll 2
+      for (uint32_t j = u.ul; j < nv; j += UNIT_) vec(row, crow, j, q);
     }
   }
 };
@@ -705,7 +729,7 @@ struct StreamGeluFwd {
 // GELU backward.  With a whole warp on one row the 16 derivative values live one per
 // lane (twice over) and are fetched with a shuffle indexed by the code; smaller units
 // read them from a shared-memory table.
-template <int DT, int UNIT_>
+template <int DT, int UNIT_, int NVL>
 struct StreamGeluBwd {
   static constexpr int kMaxRegs = 64;
   static constexpr int kKernel = kGeluBwd;
@@ -740,30 +764,40 @@ struct StreamGeluBwd {
       st.tab_s = s;
     }
     if (UNIT_ < 32) u.sync();
+    if (UNIT_ >= 32 && !active) return;  // whole warps leave together
     const uint32_t nv = active ? L / V::EPA : 0u;
     unsigned char* row = p.data + (size_t)r * L * Io<DT>::kBytes;
     const unsigned char* crow = p.codes + (size_t)r * (L / 2);
-    // every lane runs the same number of rounds so that the shuffles stay warp-wide
-    const uint32_t rounds = (nv + UNIT_ - 1) / UNIT_;
-#pragma unroll 2
-    for (uint32_t it = 0; it < rounds; ++it) {
-      const uint32_t j = it * UNIT_ + u.ul;
-      const bool ok = j < nv;
-      float v[V::EPA];
-      uint32_t bits = 0;
-      if (ok) {
-        V::widen(*(const typename V::Raw*)(row + j * 16u), v);
-        bits = V::load_codes(crow, j);
-      }
+    if (NVL > 0) {
 #pragma unroll
-      for (int k = 0; k < V::EPA; ++k) {
-        float d;
-        if (UNIT_ >= 32) d = __shfl_sync(0xffffffffu, st.d, (int)(bits >> (4 * k)));  // lane = code mod 16 (+16)
-        else d = tab[(bits >> (4 * k)) & 0xFu];
-        v[k] *= d;
+      for (int i = 0; i < NVL; ++i) vec(st, tab, row, crow, u.ul + UNIT_ * i, true);
+    } else {
+      // every lane runs the same number of rounds so that the shuffles stay warp-wide
+      const uint32_t rounds = (nv + UNIT_ - 1) / UNIT_;
+#pragma unroll 2
+      for (uint32_t it = 0; it < rounds; ++it) {
+        const uint32_t j = it * UNIT_ + u.ul;
+        vec(st, tab, row, crow, j, j < nv);
       }
-      if (ok) *(typename V::Raw*)(row + j * 16u) = V::narrow(v);
     }
+  }
+
+  static __device__ __forceinline__ void vec(const State& st, const float* tab, unsigned char* row,
+                                             const unsigned char* crow, uint32_t j, bool ok) {
+    float v[V::EPA];
+    uint32_t bits = 0;
+    if (ok) {
+      V::widen(*(const typename V::Raw*)(row + j * 16u), v);
+      bits = V::load_codes(crow, j);
+    }
+#pragma unroll
+    for (int k = 0; k < V::EPA; ++k) {
+      float d;
+      if (UNIT_ >= 32) d = __shfl_sync(0xffffffffu, st.d, (int)(bits >> (4 * k)));  // lane = code mod 16 (+16)
+      else d = tab[(bits >> (4 * k)) & 0xFu];
+      v[k] *= d;
+    }
+    if (ok) *(typename V::Raw*)(row + j * 16u) = V::narrow(v);
   }
 };
 
@@ -1024,6 +1058,116 @@ struct PairSoftmaxFwd {
   }
 };
 
+// bfloat16 form of the forward: maxima and minima are taken on packed bfloat16 pairs,
+// and the exponent's argument is one fused multiply-add.
+template <int UNIT_, int LCT>
+struct PairSoftmaxFwd<kBF16, UNIT_, LCT> {
+  static constexpr int kMaxRegs = 104;
+  static constexpr int kKernel = kSoftmaxFwd;
+  static constexpr int UNIT = UNIT_;
+  using G = PairGeom<UNIT_, LCT>;
+  struct State {};
+  static __device__ __forceinline__ void init(State&) {}
+  static __device__ __forceinline__ uint32_t rows_per_group(uint32_t) { return 2u; }
+
+  static __device__ __forceinline__ uint32_t max2(uint32_t a, uint32_t b) {
+    __nv_bfloat162 r = __hmax2(*(__nv_bfloat162*)&a, *(__nv_bfloat162*)&b);
+    return *(uint32_t*)&r;
+  }
+  static __device__ __forceinline__ uint32_t min2(uint32_t a, uint32_t b) {
+    __nv_bfloat162 r = __hmin2(*(__nv_bfloat162*)&a, *(__nv_bfloat162*)&b);
+    return *(uint32_t*)&r;
+  }
+  static __device__ __forceinline__ float lo(uint32_t w) { return __uint_as_float(w << 16); }
+  static __device__ __forceinline__ float hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+  // An inactive unit (no row pair left in this round) runs on row 0 and stores nothing, so
+  // that every lane takes part in the shuffles without per-element guards.
+  template <int HP>
+  static __device__ __forceinline__ void row(Unit<UNIT_>& u, const StagePtrs& p, uint32_t r, bool active) {
+    constexpr uint32_t kNegInf2 = 0xFF80FF80u;
+    const uint32_t a0 = (r * (uint32_t)LCT) >> 1;
+    const int ul = u.ul;
+    const uint32_t* words = (const uint32_t*)p.data + a0 + ul;
+    uint32_t raw[G::ITERS];
+    uint32_t mx2 = kNegInf2;
+#pragma unroll
+    for (int i = 0; i < G::ITERS; ++i) {
+      uint32_t w = kNegInf2;
+      if (G::has(i, ul)) w = words[UNIT_ * i];
+      if (HP == 1 && i == 0 && ul == 0) w = (w & 0xffff0000u) | 0xFF80u;                     // foreign low half
+      if (HP == 0 && i == G::LAST_I && ul == G::LAST_UL) w = (w & 0x0000ffffu) | 0xFF800000u;  // foreign high half
+      raw[i] = w;
+      mx2 = max2(mx2, w);
+    }
+    const float m = u.template reduce<kOpMax>(fmaxf(lo(mx2), hi(mx2)));
+    constexpr float kLog2e = 1.4426950408889634f;
+    const float nm = -m * kLog2e;
+    float e[G::ITERS][2];
+    float z = 0.0f;
+#pragma unroll
+    for (int i = 0; i < G::ITERS; ++i) {
+      e[i][0] = ex2_approx(fmaf(lo(raw[i]), kLog2e, nm));  // foreign / absent: 2^-inf = 0
+      e[i][1] = ex2_approx(fmaf(hi(raw[i]), kLog2e, nm));
+      z += e[i][0];
+      z += e[i][1];
+    }
+    z = u.template reduce<kOpSum>(z);
+    const float rz = __fdiv_rn(1.0f, z);
+    uint32_t mn2 = 0x7F807F80u;
+    mx2 = kNegInf2;
+    uint32_t* out = (uint32_t*)p.data + a0 + ul;
+#pragma unroll
+    for (int i = 0; i < G::ITERS; ++i) {
+      __nv_bfloat162 b = __floats2bfloat162_rn(e[i][0] * rz, e[i][1] * rz);
+      const uint32_t w = *(uint32_t*)&b;  // y as written
+      raw[i] = w;
+      const bool drop_lo = HP == 1 && i == 0 && ul == 0;
+      const bool drop_hi = HP == 0 && i == G::LAST_I && ul == G::LAST_UL;
+      if (G::has(i, ul)) {
+        uint32_t wm = w;  // for min/max a foreign half is replaced by its neighbour
+        if (drop_lo) wm = (w & 0xffff0000u) | (w >> 16);
+        if (drop_hi) wm = (w & 0x0000ffffu) | (w << 16);
+        mn2 = min2(mn2, wm);
+        mx2 = max2(mx2, wm);
+        if (active) {
+          if (drop_lo) *((uint16_t*)(out + UNIT_ * i) + 1) = (uint16_t)(w >> 16);
+          else if (drop_hi) *(uint16_t*)(out + UNIT_ * i) = (uint16_t)w;
+          else out[UNIT_ * i] = w;
+        }
+      }
+    }
+    const float mn = u.template reduce<kOpMin>(fminf(lo(mn2), hi(mn2)));
+    const float mx = u.template reduce<kOpMax>(fmaxf(lo(mx2), hi(mx2)));
+    const QRange q = make_qrange(mn, mx);
+    if (active && ul == 0) { p.meta[2 * r] = q.mn; p.meta[2 * r + 1] = q.s; }
+    unsigned char* cb = p.codes + a0 + ul;
+#pragma unroll
+    for (int i = 0; i < G::ITERS; ++i) {
+      if (active && G::has(i, ul)) {
+        const bool drop_lo = HP == 1 && i == 0 && ul == 0;
+        const bool drop_hi = HP == 0 && i == G::LAST_I && ul == G::LAST_UL;
+        CodePacker<2> pk;
+        pk.init();
+        pk.add(0, drop_lo ? q.mn : lo(raw[i]), q);
+        pk.add(1, drop_hi ? q.mn : hi(raw[i]), q);  // a dropped element codes as 0
+        uint32_t byte = pk.acc & 0xFFu;
+        if (drop_lo) byte |= cb[UNIT_ * i] & 0x0Fu;  // low nibble: the previous row's
+        cb[UNIT_ * i] = (unsigned char)byte;
+      }
+    }
+  }
+
+  static __device__ __forceinline__ void group(Unit<UNIT_>& u, State&, const StagePtrs& p, float*, uint32_t grp,
+                                               bool active, uint32_t) {
+    const uint32_t r = active ? 2 * grp : 0;
+    row<0>(u, p, r, active);
+    u.sync();  // the odd row reads the shared word and code byte the even row left
+    row<1>(u, p, r + 1, active);
+    u.sync();
+  }
+};
+
 template <int DT, int UNIT_, int LCT>
 struct PairSoftmaxBwd {
   static constexpr int kMaxRegs = 104;
@@ -1035,27 +1179,26 @@ struct PairSoftmaxBwd {
   static __device__ __forceinline__ void init(State&) {}
   static __device__ __forceinline__ uint32_t rows_per_group(uint32_t) { return 2u; }
 
+  // An inactive unit runs on row 0 and stores nothing (see the forward).
   template <int HP>
   static __device__ __forceinline__ void row(Unit<UNIT_>& u, const StagePtrs& p, uint32_t r, bool active) {
     const uint32_t a0 = (r * (uint32_t)LCT) >> 1;
     const int ul = u.ul;
-    const float mn = active ? p.meta[2 * r] : 0.0f;
-    const float s = active ? p.meta[2 * r + 1] : 0.0f;
+    const float mn = p.meta[2 * r];
+    const float s = p.meta[2 * r + 1];
     float g[G::ITERS][2], yh[G::ITERS][2];
     float dot = 0.0f;
 #pragma unroll
     for (int i = 0; i < G::ITERS; ++i) {
-      g[i][0] = 0.0f;
-      g[i][1] = 0.0f;
-      yh[i][0] = 0.0f;
-      yh[i][1] = 0.0f;
-      if (active && G::has(i, ul)) {
+      if (G::has(i, ul)) {
         const typename P::Raw w = P::load(p.data, a0 + ul + UNIT_ * i);
         const uint32_t b = p.codes[a0 + ul + UNIT_ * i];
         g[i][0] = P::lo(w);
         g[i][1] = P::hi(w);
         yh[i][0] = dequant(b & 0xFu, mn, s);
         yh[i][1] = dequant(b >> 4, mn, s);
+      } else {
+        g[i][0] = 0.0f; g[i][1] = 0.0f; yh[i][0] = 0.0f; yh[i][1] = 0.0f;
       }
       if (HP == 1 && i == 0 && ul == 0) g[i][0] = 0.0f;
       if (HP == 0 && i == G::LAST_I && ul == G::LAST_UL) g[i][1] = 0.0f;
@@ -1110,12 +1253,14 @@ __global__ void __maxnreg__(WORK::kMaxRegs) tile_kernel(TileKernelArgs a) {
     int* flags = (int*)(smem + kFlagOffset);
     for (int k = 0; k < 16; ++k) flags[k] = 0;
     fence_barrier_init();
+    grid_launch_dependents();
   }
   __syncthreads();
 
   if (warp == n_cwarps) {
     // ------------------------------------------------------------ copy warp
     if (lane != 0) return;
+    grid_dependency_wait();  // everything before this line touched shared memory only
     auto stage_ptr = [&](uint64_t it) { return smem + kHeaderBytes + (size_t)(it % S) * a.stage_bytes; };
     auto issue_load = [&](uint64_t it) {
       const uint64_t t = blockIdx.x + it * gridDim.x;
@@ -1222,8 +1367,17 @@ cudaError_t launch_work(const TilePlan& p, const TileKernelArgs& ka, cudaStream_
     if (e != cudaSuccess) return e;
     configured_dev = dev;
   }
-  kfn<<<p.grid, (p.warps + 1) * 32, p.smem_bytes, st>>>(ka);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(p.grid);
+  cfg.blockDim = dim3((p.warps + 1) * 32);
+  cfg.dynamicSmemBytes = p.smem_bytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = p.overlap_launch ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kfn, ka);
 }
 
 // The general policy, by unit size and register bound.
@@ -1277,14 +1431,27 @@ cudaError_t launch_softmax_stream(const TilePlan& p, const TileKernelArgs& ka, c
   return cudaErrorInvalidValue;
 }
 
-template <template <int, int> class WORK, int DT>
+template <template <int, int, int> class WORK, int DT, int UNIT>
+cudaError_t launch_gelu_nvl(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
+  if (UNIT >= 64) {  // fixed vector counts exist for the multi-warp units only
+    constexpr int U = UNIT >= 64 ? UNIT : 64;
+    switch (p.iters) {
+      case 6: return launch_work<WORK<DT, U, 6>>(p, ka, st);
+      case 8: return launch_work<WORK<DT, U, 8>>(p, ka, st);
+      case 10: return launch_work<WORK<DT, U, 10>>(p, ka, st);
+    }
+  }
+  return launch_work<WORK<DT, UNIT, 0>>(p, ka, st);
+}
+
+template <template <int, int, int> class WORK, int DT>
 cudaError_t launch_gelu_stream(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
   switch (p.unit_lanes) {
-    case 8: return launch_work<WORK<DT, 8>>(p, ka, st);
-    case 16: return launch_work<WORK<DT, 16>>(p, ka, st);
-    case 32: return launch_work<WORK<DT, 32>>(p, ka, st);
-    case 64: return launch_work<WORK<DT, 64>>(p, ka, st);
-    case 128: return launch_work<WORK<DT, 128>>(p, ka, st);
+    case 8: return launch_gelu_nvl<WORK, DT, 8>(p, ka, st);
+    case 16: return launch_gelu_nvl<WORK, DT, 16>(p, ka, st);
+    case 32: return launch_gelu_nvl<WORK, DT, 32>(p, ka, st);
+    case 64: return launch_gelu_nvl<WORK, DT, 64>(p, ka, st);
+    case 128: return launch_gelu_nvl<WORK, DT, 128>(p, ka, st);
   }
   return cudaErrorInvalidValue;
 }
