@@ -156,23 +156,23 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L) {
   const uint32_t meta_off = code_off + align_up(code_bytes, 128);
   const uint32_t stage_bytes = meta_off + align_up(meta_bytes, 128);
 
-  // CTAs per SM and stages per CTA: the wanted CTA count if it leaves room for 3 stages,
-  // else fewer CTAs; 2 stages only as a last resort
+  // CTAs per SM and stages per CTA.  Every tile kernel asks for a power-of-two fraction
+  // of an SM's shared memory (1/4, 1/2 or all of it) and always for the WHOLE fraction:
+  // with programmatic dependent launch the next kernel's CTAs move into the slots that
+  // this kernel's CTAs leave, which only works smoothly when the slots have equal sizes
+  // (measured: 50.5 KB and 52.5 KB requests in alternation cost 3.7 us per launch).
   ctas_per_sm = env_int("S2A_CTAS_PER_SM", ctas_per_sm);
-  if (ctas_per_sm < 1) ctas_per_sm = 1;
+  if (ctas_per_sm != 1 && ctas_per_sm != 2 && ctas_per_sm != 4) ctas_per_sm = 2;
   const int env_stages = env_int("S2A_STAGES", 0);
-  uint32_t stages = 0;
-  int chosen = 0;
-  for (int pass = 0; pass < 2 && chosen == 0; ++pass) {
-    const uint32_t want = env_stages > 0 ? (uint32_t)env_stages : (pass == 0 ? 3u : 2u);
-    for (int c = ctas_per_sm; c >= 1 && chosen == 0; --c) {
-      const uint32_t budget = kMaxSmem / (uint32_t)c - 1024;
-      if (budget >= kHeaderBytes + want * stage_bytes) { chosen = c; stages = want; }
-    }
+  uint32_t stages = 0, smem = 0;
+  for (int c = ctas_per_sm; c >= 1 && stages == 0; c /= 2) {
+    const uint32_t budget = kMaxSmem / (uint32_t)c - 1024;  // 1 KiB per CTA is the system's
+    uint32_t fit = budget > kHeaderBytes ? (budget - kHeaderBytes) / stage_bytes : 0;
+    if (fit > 4) fit = 4;
+    if (env_stages > 0 && (uint32_t)env_stages <= fit) fit = (uint32_t)env_stages;
+    if (fit >= 2) { stages = fit; ctas_per_sm = c; smem = budget; }
   }
-  if (chosen == 0 || stages > (uint32_t)kMaxStages) return p;
-  ctas_per_sm = chosen;
-  const uint32_t smem = kHeaderBytes + stages * stage_bytes;
+  if (stages == 0) return p;
 
   p.n_tiles = n_rows / rows;
   if (p.n_tiles == 0) return TilePlan{};

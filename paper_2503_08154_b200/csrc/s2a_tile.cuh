@@ -1256,11 +1256,14 @@ __global__ void __maxnreg__(WORK::kMaxRegs) tile_kernel(TileKernelArgs a) {
     grid_launch_dependents();
   }
   __syncthreads();
+  // Everything above touched shared memory only.  All threads park here (not only the
+  // copy lane) so that an early-launched CTA does not spin on its barriers, taking issue
+  // slots from the previous kernel's last CTAs.
+  grid_dependency_wait();
 
   if (warp == n_cwarps) {
     // ------------------------------------------------------------ copy warp
     if (lane != 0) return;
-    grid_dependency_wait();  // everything before this line touched shared memory only
     auto stage_ptr = [&](uint64_t it) { return smem + kHeaderBytes + (size_t)(it % S) * a.stage_bytes; };
     auto issue_load = [&](uint64_t it) {
       const uint64_t t = blockIdx.x + it * gridDim.x;
@@ -1364,6 +1367,10 @@ cudaError_t launch_work(const TilePlan& p, const TileKernelArgs& ka, cudaStream_
   cudaGetDevice(&dev);
   if (configured_dev != dev) {
     cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem);
+    if (e != cudaSuccess) return e;
+    // Always the largest shared-memory carve-out: kernels of different kinds then leave the
+    // SMs in the same configuration, and consecutive launches need no reconfiguration.
+    e = cudaFuncSetAttribute(kfn, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
     if (e != cudaSuccess) return e;
     configured_dev = dev;
   }
