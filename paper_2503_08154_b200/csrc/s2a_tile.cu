@@ -86,10 +86,11 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L) {
     unit = n_acc >= 256 ? 64u : (n_acc >= 32 ? 32u : (n_acc >= 16 ? 16u : 8u));
     if (dt == kF32 && n_acc >= 512) unit = 128;  // the same vectors per lane as bfloat16 with 64
     if (env_unit == 8 || env_unit == 16 || env_unit == 32 || env_unit == 64 || env_unit == 128) unit = (uint32_t)env_unit;
-    // a fixed vector count per lane (6, 8 or 10) when the row length allows it
-    if (unit >= 64 && n_acc % unit == 0 && (n_acc / unit == 6 || n_acc / unit == 8 || n_acc / unit == 10) &&
-        env_int("S2A_FIXED", 1) != 0)
-      iters = n_acc / unit;
+    // a fixed vector count per lane (3..6, 8 or 10) when the row length allows it
+    if (unit >= 64 && n_acc % unit == 0 && env_int("S2A_FIXED", 1) != 0) {
+      const uint32_t per = n_acc / unit;
+      if ((per >= 3 && per <= 6) || per == 8 || per == 10) iters = per;
+    }
   } else if (vec16 && !force_generic) {
     // softmax on 16-byte vectors: up to 32 (at most 64) elements per lane in registers
     const uint32_t cap = 32u / epa, cap2 = 64u / epa;

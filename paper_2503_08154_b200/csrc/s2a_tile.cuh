@@ -1443,6 +1443,9 @@ cudaError_t launch_gelu_nvl(const TilePlan& p, const TileKernelArgs& ka, cudaStr
   if (UNIT >= 64) {  // fixed vector counts exist for the multi-warp units only
     constexpr int U = UNIT >= 64 ? UNIT : 64;
     switch (p.iters) {
+      case 3: return launch_work<WORK<DT, U, 3>>(p, ka, st);
+      case 4: return launch_work<WORK<DT, U, 4>>(p, ka, st);
+      case 5: return launch_work<WORK<DT, U, 5>>(p, ka, st);
       case 6: return launch_work<WORK<DT, U, 6>>(p, ka, st);
       case 8: return launch_work<WORK<DT, U, 8>>(p, ka, st);
       case 10: return launch_work<WORK<DT, U, 10>>(p, ka, st);
