@@ -1,0 +1,100 @@
+"""Bandwidth sweep of the four kernels over tensor sizes and row lengths.
+
+    python -m paper_2503_08154_b200.bandwidth_sweep [--quick] [--seeds 5]
+
+GELU: 1e6 .. 2e9 elements (row length 4096), bfloat16 and float32.  Softmax: row lengths
+64 / 197 / 257 / 1024 / 4096 with 1e4 .. 1e7 rows (combinations above 2e9 elements are
+skipped).  Inputs are N(0,1), drawn on the device from seeds 0..S-1; every figure is the
+median over the seeds of forward+backward algorithmic bytes per second, timed with CUDA
+events over back-to-back launches on rotating buffers.  One JSON line per case.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import statistics
+
+import torch
+
+from . import binding
+
+PEAK_NOTE = "algorithmic bytes = 2*n*itemsize + n/2 + 8*rows per kernel"
+
+
+def _time_pair(kind: str, rows: int, L: int, dtype, seed: int, target_bytes: float = 1.5e9):
+    n = rows * L
+    item = 2 if dtype == torch.bfloat16 else 4
+    per_set = 4 * n * item
+    sets = max(1, min(6, int(target_bytes // per_set)))
+    if per_set * sets < 3e8:  # keep the working set above the 126 MB L2
+        sets = max(sets, min(8, int(3e8 // per_set) + 1))
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    xs = [torch.randn(n, device="cuda", generator=g).to(dtype) for _ in range(sets)]
+    gs = [torch.randn(n, device="cuda", generator=g).to(dtype) for _ in range(sets)]
+    ys = [torch.empty_like(x) for x in xs]
+    gins = [torch.empty_like(x) for x in xs]
+    st = [binding.alloc_stash(n, L, "cuda") for _ in range(sets)]
+    fwd = binding.s2a_gelu_fwd if kind == "gelu" else binding.s2a_softmax_fwd
+    bwd = binding.s2a_gelu_bwd if kind == "gelu" else binding.s2a_softmax_bwd
+    iters = max(4, min(200, int(2e10 // (n * item * 4))))
+
+    def loop(fn):
+        for i in range(min(3, sets)):
+            fn(i)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(iters):
+            fn(i % sets)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e-3 / iters
+
+    t_f = loop(lambda i: fwd(xs[i], ys[i], st[i][0], st[i][1], L))
+    t_b = loop(lambda i: bwd(gs[i], st[i][0], st[i][1], gins[i], L))
+    if binding.s2a_device_error() != 0:
+        raise RuntimeError("a kernel gave up on a bounded wait")
+    alg = 2 * n * item + (n + 1) // 2 + 8 * rows
+    return alg / t_f / 1e9, alg / t_b / 1e9, 2 * alg / (t_f + t_b) / 1e9
+
+
+def cases(quick: bool):
+    out = []
+    for n in ((1e6, 1e8) if quick else (1e6, 1e7, 1e8, 1e9, 2e9)):
+        rows = max(2, int(n) // 4096)
+        for dtype in (torch.bfloat16, torch.float32):
+            out.append(("gelu", rows, 4096, dtype))
+    for L in (64, 197, 257, 1024, 4096):
+        for rows in ((10**4, 10**6) if quick else (10**4, 10**5, 10**6, 10**7)):
+            if rows * L > 2e9 or (quick and rows * L > 3e8):
+                continue
+            for dtype in (torch.bfloat16, torch.float32):
+                out.append(("softmax", rows, L, dtype))
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--quick", action="store_true")
+    ap.add_argument("--seeds", type=int, default=5)
+    args = ap.parse_args()
+    for kind, rows, L, dtype in cases(args.quick):
+        res = []
+        for seed in range(args.seeds):
+            res.append(_time_pair(kind, rows, L, dtype, seed))
+            torch.cuda.empty_cache()
+        med = [statistics.median(r[k] for r in res) for k in range(3)]
+        spread = max(r[2] for r in res) - min(r[2] for r in res)
+        kid = binding.GELU_FWD if kind == "gelu" else binding.SOFTMAX_FWD
+        print(json.dumps({
+            "kernel_pair": kind, "rows": rows, "row_len": L, "elems": rows * L,
+            "io_dtype": "bf16" if dtype == torch.bfloat16 else "f32", "seeds": args.seeds,
+            "fwd_GBps": round(med[0], 1), "bwd_GBps": round(med[1], 1), "fwd_bwd_GBps": round(med[2], 1),
+            "fwd_bwd_gelem_per_s": round(med[2] / ((2 * (2 if dtype == torch.bfloat16 else 4) + 0.5) + 8.0 / L), 2),
+            "spread_GBps": round(spread, 1), "note": PEAK_NOTE,
+            "plan": binding.s2a_describe_plan(kid, rows * L, L, binding.BF16 if dtype == torch.bfloat16 else binding.F32),
+        }), flush=True)
+
+
+if __name__ == "__main__":
+    main()

@@ -209,6 +209,45 @@ def test_vit_block_full_size(shape):
     print("%s: softmax edge flips vs oracle: %d of %d" % (shape.name, flips, x.size))
 
 
+def test_tensor_beyond_2_to_31_elements_uses_64_bit_indexing():
+    """2.2e9 bfloat16 elements (the largest size of the bandwidth sweep): a seeded block of
+    rows is repeated down the tensor, every repeat must come out identical, and the first
+    and the last repeat are compared with the oracle element by element."""
+    L, block_rows, repeats = 4096, 1024, 525          # 2,202,009,600 elements
+    free, _ = torch.cuda.mem_get_info()
+    n = L * block_rows * repeats
+    if free < 2.6 * 2 * n:
+        pytest.skip("not enough free device memory for a 2.2e9-element tensor")
+    x, g = _gelu_inputs(block_rows, L, BF16, seed=5)
+    xb = pu.to_device(x, BF16)
+    xd = xb.repeat(repeats)
+    assert xd.numel() == n and n > 2 ** 31
+    yd = torch.empty_like(xd)
+    codes, meta = binding.alloc_stash(n, L, xd.device)
+    binding.s2a_gelu_fwd(xd, yd, codes, meta, L)
+    torch.cuda.synchronize()
+    assert binding.s2a_device_error() == 0
+    y_o, codes_o, meta_o = o.gelu_fwd(x, L, BF16, threads=THREADS)
+    yv = yd.view(repeats, -1)
+    cv = codes.view(repeats, -1)
+    mv = meta.view(repeats, -1)
+    assert bool((yv == yv[0]).all()) and bool((cv == cv[0]).all()) and bool((mv == mv[0]).all())
+    for rep in (0, repeats - 1):
+        assert np.array_equal(cv[rep].cpu().numpy(), codes_o)
+        assert np.array_equal(mv[rep].cpu().numpy(), meta_o)
+        pu.assert_close(pu.widen(pu.to_host(yv[rep], BF16), BF16), pu.widen(y_o, BF16), BF16, "gelu y (large)")
+    del yd, yv
+    gd = pu.to_device(g, BF16).repeat(repeats)
+    gin = torch.empty_like(gd)
+    binding.s2a_gelu_bwd(gd, codes, meta, gin, L)
+    torch.cuda.synchronize()
+    assert binding.s2a_device_error() == 0
+    gin_o = o.gelu_bwd(g, codes_o, meta_o, L, BF16, threads=THREADS)
+    gv = gin.view(repeats, -1)
+    assert bool((gv == gv[0]).all())
+    pu.assert_close(pu.widen(pu.to_host(gv[repeats - 1], BF16), BF16), pu.widen(gin_o, BF16), BF16, "gelu grad_in (large)")
+
+
 def test_stash_bytes_are_half_a_byte_per_element_plus_row_metadata():
     for sh in (synth.VIT_B16_B64, synth.VIT_L16_B64, synth.VIT_H14_B32):
         total = 0
