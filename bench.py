@@ -254,6 +254,24 @@ def run_reference(args, shape, blocks):
     print(json.dumps(line))
 
 
+# ------------------------------------------------------------------ aggregation over ranks
+def max_over_ranks(ms: float, world: int, device=None) -> float:
+    """The slowest rank's time: every rank runs an independent replica of the same step, so
+    the job's time is the maximum and its throughput is world * per-replica work / max."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_throughput(step_bytes: int, steps: int, ms: float, world: int) -> float:
+    """Whole-job GB/s of `world` replicas that each moved step_bytes * steps in `ms`."""
+    return world * step_bytes * steps / (ms * 1e-3) / 1e9
+
+
 # ------------------------------------------------------------------ the CUDA path
 def run_ours(args, shape, blocks, rank, world):
     import torch
@@ -384,10 +402,7 @@ def run_ours(args, shape, blocks, rank, world):
         for i, (name, _, _) in enumerate(calls):
             bracketed_ms[name].append(ev[i].elapsed_time(ev[i + 1]))
 
-    if world > 1:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, world, dev)
 
     # ---- end to end: pinned host inputs in, results out, every step
     e2e = None
@@ -422,12 +437,9 @@ def run_ours(args, shape, blocks, rank, world):
         e1.record(stream)
         barrier()
         e2e_ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
+        e2e_ms = max_over_ranks(e2e_ms, world, dev)
         io_bytes = blocks * 2 * item * (shape.gelu_elems + (shape.softmax_elems if has_softmax else 0))
-        e2e = {"value": world * step_bytes * args.e2e_steps / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s",
+        e2e = {"value": aggregate_throughput(step_bytes, args.e2e_steps, e2e_ms, world), "unit": "GB/s",
                "h2d_bytes_per_step": io_bytes, "d2h_bytes_per_step": io_bytes, "steps": args.e2e_steps,
                "ms_per_step": e2e_ms / args.e2e_steps}
 
@@ -449,7 +461,7 @@ def run_ours(args, shape, blocks, rank, world):
                 "peak_source": "%s copy bandwidth" % peak_kind, "unit": "GB/s",
                 "frac": per_kernel[dominant]["GBps"] / peak, "traffic": stored_traffic(dominant, shape.name)}
 
-    value = world * step_bytes * args.steps / (total_ms * 1e-3) / 1e9
+    value = aggregate_throughput(step_bytes, args.steps, total_ms, world)
     cpu_baseline = None
     if not args.skip_cpu_baseline:
         from oracle import s2a_oracle as o
