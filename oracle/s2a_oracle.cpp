@@ -342,6 +342,30 @@ int s2a_oracle_quantize_tensor(const void* v, uint8_t* codes, float* meta, size_
   return 0;
 }
 
+// ---- ReLU (Section 3.2, "ReLU layer"): the derivative takes the values 0 and 1 only, so
+// the stash is one bit per element: 1 where x > 0.  Bit (e mod 8) of byte e / 8, least
+// significant bit first, over the flat element index; unused bits of the last byte are 0.
+// Forward: y = x where x > 0, else +0.  Backward: grad_in = grad_out where the bit is set,
+// else +0.
+int s2a_oracle_relu_fwd(const void* x, void* y, uint8_t* mask, size_t n, int dt) {
+  for (size_t b = 0; b < (n + 7) / 8; ++b) mask[b] = 0;
+  for (size_t e = 0; e < n; ++e) {
+    double xe = load_elem(x, e, dt);
+    bool pos = xe > 0.0;
+    store_elem(y, e, dt, pos ? xe : 0.0);
+    if (pos) mask[e >> 3] |= (uint8_t)(1u << (e & 7));
+  }
+  return 0;
+}
+
+int s2a_oracle_relu_bwd(const void* g, const uint8_t* mask, void* gin, size_t n, int dt) {
+  for (size_t e = 0; e < n; ++e) {
+    bool pos = (mask[e >> 3] >> (e & 7)) & 1;
+    store_elem(gin, e, dt, pos ? load_elem(g, e, dt) : 0.0);
+  }
+  return 0;
+}
+
 // Number of hardware threads the row-parallel driver can use.
 int s2a_oracle_hardware_threads() {
   unsigned h = std::thread::hardware_concurrency();

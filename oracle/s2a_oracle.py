@@ -75,6 +75,10 @@ def lib() -> ctypes.CDLL:
             getattr(L, name).restype = i32
         L.s2a_oracle_quantize_tensor.argtypes = [vp, vp, vp, sz, sz, i32, i32, i32]
         L.s2a_oracle_quantize_tensor.restype = i32
+        L.s2a_oracle_relu_fwd.argtypes = [vp, vp, vp, sz, i32]
+        L.s2a_oracle_relu_fwd.restype = i32
+        L.s2a_oracle_relu_bwd.argtypes = [vp, vp, vp, sz, i32]
+        L.s2a_oracle_relu_bwd.restype = i32
         L.s2a_oracle_hardware_threads.argtypes = []
         L.s2a_oracle_hardware_threads.restype = i32
         _lib = L
@@ -218,6 +222,28 @@ def softmax_fwd(x, row_len: int, dt: int, threads: int = 1):
 
 def softmax_bwd(g, codes, meta, row_len: int, dt: int, threads: int = 1):
     return _bwd(lib().s2a_oracle_softmax_bwd, g, codes, meta, row_len, dt, threads)
+
+
+def mask_bytes(n: int) -> int:
+    return (n + 7) // 8
+
+
+def relu_fwd(x, dt: int):
+    """Returns (y, bit mask) for the ReLU forward with the 1-bit stash."""
+    x = _check_io(x, dt).reshape(-1)
+    y = np.empty_like(x)
+    mask = np.zeros(mask_bytes(x.size), dtype=np.uint8)
+    lib().s2a_oracle_relu_fwd(_ptr(x), _ptr(y), _ptr(mask), x.size, dt)
+    return y, mask
+
+
+def relu_bwd(g, mask, dt: int):
+    g = _check_io(g, dt).reshape(-1)
+    mask = np.ascontiguousarray(mask, dtype=np.uint8)
+    assert mask.size >= mask_bytes(g.size)
+    gin = np.empty_like(g)
+    lib().s2a_oracle_relu_bwd(_ptr(g), _ptr(mask), _ptr(gin), g.size, dt)
+    return gin
 
 
 def quantize_tensor(v, row_len: int, dt: int, clip_to_2: bool = False, threads: int = 1):

@@ -346,6 +346,32 @@ def test_bad_shapes_are_rejected_and_empty_is_fine():
     assert y.size == 0 and c.size == 0 and m.size == 0
 
 
+# ------------------------------------------------------------------ ReLU 1-bit stash
+@pytest.mark.parametrize("dt", [F32, BF16])
+@pytest.mark.parametrize("n", [1, 7, 8, 9, 1000, 4099])
+def test_relu_mask_against_numpy(dt, n):
+    x32 = synth.normal(4, ("relu", n, dt), n)
+    x32[::5] = 0.0
+    if n > 3:
+        x32[3] = -0.0
+    x = synth.to_io(x32, dt)
+    g = synth.to_io(synth.normal(4, ("relug", n, dt), n), dt)
+    xw = o.widen(x, dt)
+    y, mask = o.relu_fwd(x, dt)
+    assert np.array_equal(o.widen(y, dt), np.maximum(xw, 0.0))
+    assert not np.signbit(o.widen(y, dt)).any()                       # -0 and negatives become +0
+    assert np.array_equal(mask, np.packbits(xw > 0, bitorder="little"))
+    assert mask.size == (n + 7) // 8                                   # one bit per element
+    gin = o.relu_bwd(g, mask, dt)
+    assert np.array_equal(o.widen(gin, dt), np.where(xw > 0, o.widen(g, dt), 0.0))
+    # the derivative takes the two values 0 and 1 only: finite differences of the forward
+    h = 1e-3
+    far = np.abs(xw) > 2 * h
+    fd = (np.maximum(xw + h, 0) - np.maximum(xw - h, 0)) / (2 * h)
+    bits = np.unpackbits(mask, bitorder="little")[:n]
+    assert np.allclose(fd[far], bits[far])
+
+
 # ------------------------------------------------------------------ memory accounting
 def test_stash_size_and_the_papers_memory_delta():
     # 0.5 B per element, against the 4 B of the 32-bit activation the paper replaces
