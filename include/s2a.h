@@ -102,6 +102,27 @@ int s2a_softmax_fwd(const void* x, void* y, uint8_t* codes, float* meta, size_t 
 int s2a_softmax_bwd(const void* grad_out, const uint8_t* codes, const float* meta, void* grad_in,
                     size_t n_elems, size_t row_len, int dt, void* cuda_stream);
 
+/* Bytes of the ReLU bit mask for n_elems elements: (n_elems + 7) / 8. */
+size_t s2a_mask_bytes(size_t n_elems);
+
+/* ReLU forward with a 1-bit stash (Section 3.2, "ReLU layer": the derivative takes the
+ * values 0 and 1 only).  y = x where x > 0, else +0.  Element e of the flat tensor owns bit
+ * (e mod 8), least significant first, of mask byte e / 8; unused bits of the last byte are
+ * written as 0.  No rows, no metadata.
+ *   x     in   n_elems elements of type dt (16-byte aligned)
+ *   y     out  n_elems elements of type dt (16-byte aligned, may alias x)
+ *   mask  out  s2a_mask_bytes(n_elems) bytes
+ */
+int s2a_relu_fwd(const void* x, void* y, uint8_t* mask, size_t n_elems, int dt, void* cuda_stream);
+
+/* ReLU backward from the mask: grad_in = grad_out where the element's bit is set, else +0.
+ *   grad_out in   n_elems elements of type dt (16-byte aligned)
+ *   mask     in   as written by s2a_relu_fwd
+ *   grad_in  out  n_elems elements of type dt (16-byte aligned, may alias grad_out)
+ */
+int s2a_relu_bwd(const void* grad_out, const uint8_t* mask, void* grad_in, size_t n_elems, int dt,
+                 void* cuda_stream);
+
 /* The pipelined kernels wait on shared-memory barriers with an iteration limit; a
  * wait that runs out records a bit in a per-device word and the kernel returns early.
  * This call copies that word of the CURRENT device into *flags (0 = no kernel ever gave

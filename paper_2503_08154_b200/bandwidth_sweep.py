@@ -58,6 +58,33 @@ def _time_pair(kind: str, rows: int, L: int, dtype, seed: int, target_bytes: flo
     return alg / t_f / 1e9, alg / t_b / 1e9, 2 * alg / (t_f + t_b) / 1e9
 
 
+def _time_relu(n: int, dtype, seed: int):
+    item = 2 if dtype == torch.bfloat16 else 4
+    sets = max(1, min(8, int(3e8 // (4 * n * item)) + 1))
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    xs = [torch.randn(n, device="cuda", generator=g).to(dtype) for _ in range(sets)]
+    ys = [torch.empty_like(x) for x in xs]
+    ms = [torch.empty(binding.mask_bytes(n), dtype=torch.uint8, device="cuda") for _ in range(sets)]
+    iters = max(4, min(200, int(2e10 // (n * item * 4))))
+
+    def loop(fn):
+        for i in range(min(3, sets)):
+            fn(i)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(iters):
+            fn(i % sets)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e-3 / iters
+
+    t_f = loop(lambda i: binding.s2a_relu_fwd(xs[i], ys[i], ms[i]))
+    t_b = loop(lambda i: binding.s2a_relu_bwd(xs[i], ms[i], ys[i]))
+    alg = 2 * n * item + (n + 7) // 8
+    return alg / t_f / 1e9, alg / t_b / 1e9, 2 * alg / (t_f + t_b) / 1e9
+
+
 def cases(quick: bool):
     out = []
     for n in ((1e6, 1e8) if quick else (1e6, 1e7, 1e8, 1e9, 2e9)):
@@ -78,6 +105,17 @@ def main():
     ap.add_argument("--quick", action="store_true")
     ap.add_argument("--seeds", type=int, default=5)
     args = ap.parse_args()
+    for n in ((10**6, 10**8) if args.quick else (10**6, 10**7, 10**8, 10**9, 2 * 10**9)):
+        for dtype in (torch.bfloat16, torch.float32):
+            res = []
+            for seed in range(args.seeds):
+                res.append(_time_relu(int(n), dtype, seed))
+                torch.cuda.empty_cache()
+            med = [statistics.median(r[k] for r in res) for k in range(3)]
+            print(json.dumps({"kernel_pair": "relu", "elems": int(n), "io_dtype": "bf16" if dtype == torch.bfloat16 else "f32",
+                              "seeds": args.seeds, "fwd_GBps": round(med[0], 1), "bwd_GBps": round(med[1], 1),
+                              "fwd_bwd_GBps": round(med[2], 1),
+                              "note": "algorithmic bytes = 2*n*itemsize + n/8 per kernel"}), flush=True)
     for kind, rows, L, dtype in cases(args.quick):
         res = []
         for seed in range(args.seeds):

@@ -22,6 +22,7 @@ GELU_FWD, GELU_BWD, SOFTMAX_FWD, SOFTMAX_BWD = 0, 1, 2, 3
 EXPORTS = (
     "s2a_codes_bytes", "s2a_meta_bytes", "s2a_status_string", "s2a_gelu_fwd", "s2a_gelu_bwd",
     "s2a_softmax_fwd", "s2a_softmax_bwd", "s2a_device_error", "s2a_describe_plan",
+    "s2a_mask_bytes", "s2a_relu_fwd", "s2a_relu_bwd",
 )
 
 _lib = None
@@ -50,6 +51,12 @@ def lib() -> ctypes.CDLL:
             f = getattr(L, name)
             f.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_size_t, c.c_size_t,
                           c.c_int, c.c_void_p]
+            f.restype = c.c_int
+        L.s2a_mask_bytes.argtypes = [c.c_size_t]
+        L.s2a_mask_bytes.restype = c.c_size_t
+        for name in ("s2a_relu_fwd", "s2a_relu_bwd"):
+            f = getattr(L, name)
+            f.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p, c.c_size_t, c.c_int, c.c_void_p]
             f.restype = c.c_int
         L.s2a_device_error.argtypes = [c.POINTER(c.c_uint), c.c_int]
         L.s2a_device_error.restype = c.c_int
@@ -143,6 +150,31 @@ def s2a_softmax_fwd(x, y, codes, meta, row_len: int) -> None:
 
 def s2a_softmax_bwd(grad_out, codes, meta, grad_in, row_len: int) -> None:
     _bwd(lib().s2a_softmax_bwd, grad_out, codes, meta, grad_in, row_len)
+
+
+def mask_bytes(n_elems: int) -> int:
+    return int(lib().s2a_mask_bytes(n_elems))
+
+
+def s2a_relu_fwd(x, y, mask) -> None:
+    _dev(x, "x"), _dev(y, "y"), _dev(mask, "mask")
+    n = x.numel()
+    if y.numel() != n or y.dtype != x.dtype:
+        raise S2AError("y must match x in size and dtype")
+    if mask.dtype != torch.uint8 or mask.numel() < mask_bytes(n):
+        raise S2AError("mask must be uint8 with at least mask_bytes(n) elements")
+    check(lib().s2a_relu_fwd(x.data_ptr(), y.data_ptr(), mask.data_ptr(), n, dtype_code(x), _stream_ptr()))
+
+
+def s2a_relu_bwd(grad_out, mask, grad_in) -> None:
+    _dev(grad_out, "grad_out"), _dev(grad_in, "grad_in"), _dev(mask, "mask")
+    n = grad_out.numel()
+    if grad_in.numel() != n or grad_in.dtype != grad_out.dtype:
+        raise S2AError("grad_in must match grad_out in size and dtype")
+    if mask.dtype != torch.uint8 or mask.numel() < mask_bytes(n):
+        raise S2AError("mask must be uint8 with at least mask_bytes(n) elements")
+    check(lib().s2a_relu_bwd(grad_out.data_ptr(), mask.data_ptr(), grad_in.data_ptr(), n,
+                             dtype_code(grad_out), _stream_ptr()))
 
 
 def s2a_device_error(clear: bool = False) -> int:

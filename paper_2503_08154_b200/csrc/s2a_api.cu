@@ -90,6 +90,25 @@ int s2a_softmax_bwd(const void* grad_out, const uint8_t* codes, const float* met
              const_cast<float*>(meta), n_elems, row_len, dt, cuda_stream);
 }
 
+size_t s2a_mask_bytes(size_t n_elems) { return (n_elems + 7) / 8; }
+
+static int run_relu(bool fwd, const void* in, void* out, uint8_t* mask, size_t n, int dt, void* stream) {
+  if (dt != S2A_F32 && dt != S2A_BF16) return S2A_ERR_DTYPE;
+  if (n == 0) return S2A_OK;
+  if (!in || !out || !mask) return S2A_ERR_NULL;
+  if (misaligned(in, 16) || misaligned(out, 16)) return S2A_ERR_ALIGN;
+  return launch_relu(fwd, dt, in, out, mask, n, (cudaStream_t)stream) == cudaSuccess ? S2A_OK : S2A_ERR_CUDA;
+}
+
+int s2a_relu_fwd(const void* x, void* y, uint8_t* mask, size_t n_elems, int dt, void* cuda_stream) {
+  return run_relu(true, x, y, mask, n_elems, dt, cuda_stream);
+}
+
+int s2a_relu_bwd(const void* grad_out, const uint8_t* mask, void* grad_in, size_t n_elems, int dt,
+                 void* cuda_stream) {
+  return run_relu(false, grad_out, grad_in, const_cast<uint8_t*>(mask), n_elems, dt, cuda_stream);
+}
+
 int s2a_device_error(unsigned int* flags, int clear) {
   if (!flags) return S2A_ERR_NULL;
   return read_error_word(flags, clear != 0) == cudaSuccess ? S2A_OK : S2A_ERR_CUDA;

@@ -23,6 +23,9 @@ struct RowwiseArgs {
 
 cudaError_t launch_rowwise(int kernel, int dt, const RowwiseArgs& a, cudaStream_t st);
 
+// ReLU with its 1-bit mask: in = x (forward) or grad_out (backward), out = y or grad_in.
+cudaError_t launch_relu(bool fwd, int dt, const void* in, void* out, uint8_t* mask, uint64_t n, cudaStream_t st);
+
 // ---------------------------------------------------------------- pipelined tiles
 // A tile is `tile_rows` consecutive rows whose flat element span starts and ends on a
 // multiple of 32 elements, so that its data and its code bytes can move with 16-byte

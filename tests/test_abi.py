@@ -37,6 +37,16 @@ def test_size_helpers(lib):
     assert binding.meta_bytes(n, 3072) == 8 * 64 * 197
 
 
+def test_relu_argument_checks(lib):
+    a = ctypes.c_void_p(0x1000)
+    assert binding.mask_bytes(0) == 0 and binding.mask_bytes(1) == 1 and binding.mask_bytes(8) == 1
+    assert binding.mask_bytes(9) == 2
+    assert lib.s2a_relu_fwd(None, a, a, 8, 0, None) == 1
+    assert lib.s2a_relu_fwd(ctypes.c_void_p(0x1008), a, a, 8, 0, None) == 3
+    assert lib.s2a_relu_bwd(a, a, a, 8, 9, None) == 4
+    assert lib.s2a_relu_bwd(a, a, a, 0, 1, None) == 0
+
+
 def test_status_strings(lib):
     assert binding.status_string(0) == "S2A_OK"
     for code, word in ((1, "NULL"), (2, "SHAPE"), (3, "ALIGN"), (4, "DTYPE"), (5, "CUDA"), (6, "DEVICE")):

@@ -248,6 +248,38 @@ def test_tensor_beyond_2_to_31_elements_uses_64_bit_indexing():
     pu.assert_close(pu.widen(pu.to_host(gv[repeats - 1], BF16), BF16), pu.widen(gin_o, BF16), BF16, "gelu grad_in (large)")
 
 
+# ------------------------------------------------------------------ ReLU with a 1-bit stash
+@pytest.mark.parametrize("dt", [F32, BF16])
+@pytest.mark.parametrize("n", [1, 7, 8, 9, 1023, 1024 * 8, 100003, 5_000_001, 40_000_008])
+def test_relu_mask(n, dt):
+    x32 = synth.normal(6, ("relu", n, dt), n)
+    x32[::7] = 0.0
+    x32[3::11] = -0.0
+    x = synth.to_io(x32, dt)
+    g = synth.to_io(synth.normal(6, ("relug", n, dt), n), dt)
+    y_o, mask_o = o.relu_fwd(x, dt)
+    gin_o = o.relu_bwd(g, mask_o, dt)
+    item = synth.io_itemsize(dt)
+    tdt = pu.torch_dtype(dt)
+    for inplace in (False, True):
+        xd, gd = pu.to_device(x, dt), pu.to_device(g, dt)
+        yg, mg, og = pu.Guarded(n * item), pu.Guarded(binding.mask_bytes(n)), pu.Guarded(n * item)
+        if inplace:
+            yg.view(tdt).copy_(xd)
+            og.view(tdt).copy_(gd)
+        binding.s2a_relu_fwd(yg.view(tdt) if inplace else xd, yg.view(tdt), mg.view(torch.uint8))
+        md = torch.from_numpy(mask_o).cuda()
+        binding.s2a_relu_bwd(og.view(tdt) if inplace else gd, md, og.view(tdt))
+        torch.cuda.synchronize()
+        for buf, what in ((yg, "y"), (mg, "mask"), (og, "grad_in")):
+            buf.check("relu " + what)
+        # exact: the ReLU stash is lossless
+        assert np.array_equal(pu.to_host(yg.view(tdt), dt).view(np.uint8), y_o.view(np.uint8))
+        assert np.array_equal(mg.view(torch.uint8).cpu().numpy(), mask_o)
+        assert np.array_equal(pu.to_host(og.view(tdt), dt).view(np.uint8), gin_o.view(np.uint8))
+    assert binding.mask_bytes(n) == (n + 7) // 8
+
+
 def test_stash_bytes_are_half_a_byte_per_element_plus_row_metadata():
     for sh in (synth.VIT_B16_B64, synth.VIT_L16_B64, synth.VIT_H14_B32):
         total = 0
