@@ -265,6 +265,31 @@ int s2a_oracle_gelu_fwd(const void* x, void* y, uint8_t* codes, float* meta, siz
   return 0;
 }
 
+// ---- GELU forward, per-TENSOR range: the other reading of "quantized between the maximal
+// and minimal value" (Section 3.2, "GeLU layer"): Eq. 8's min and max are taken over the
+// whole clipped tensor instead of over each row.  Every row's metadata carries the same
+// (min, s), so the backward pass is unchanged.
+int s2a_oracle_gelu_fwd_tensor_range(const void* x, void* y, uint8_t* codes, float* meta, size_t n,
+                                     size_t L, int dt) {
+  if (n == 0) return 0;
+  if (bad_shape(n, L)) return 2;
+  std::vector<float> c(n);
+  std::vector<uint8_t> q(n);
+  for (size_t e = 0; e < n; ++e) {
+    double xe = load_elem(x, e, dt);
+    c[e] = (float)std::min(std::max(xe, -2.0), 2.0);
+    store_elem(y, e, dt, gelu(xe));
+  }
+  float mn, s;
+  quantize_row(c.data(), n, q.data(), &mn, &s);  // one "row": the whole tensor
+  for (size_t r = 0; r < n / L; ++r) {
+    meta[2 * r] = mn;
+    meta[2 * r + 1] = s;
+  }
+  pack_codes(q.data(), n, codes);
+  return 0;
+}
+
 // ---- GELU backward: Eq. 9 then Eq. 12 at x_hat, times grad_out.
 int s2a_oracle_gelu_bwd(const void* g, const uint8_t* codes, const float* meta, void* gin,
                         size_t n, size_t L, int dt, int threads) {

@@ -73,6 +73,8 @@ def lib() -> ctypes.CDLL:
         for name in ("s2a_oracle_gelu_bwd", "s2a_oracle_softmax_bwd"):
             getattr(L, name).argtypes = [vp, vp, vp, vp, sz, sz, i32, i32]
             getattr(L, name).restype = i32
+        L.s2a_oracle_gelu_fwd_tensor_range.argtypes = [vp, vp, vp, vp, sz, sz, i32]
+        L.s2a_oracle_gelu_fwd_tensor_range.restype = i32
         L.s2a_oracle_quantize_tensor.argtypes = [vp, vp, vp, sz, sz, i32, i32, i32]
         L.s2a_oracle_quantize_tensor.restype = i32
         L.s2a_oracle_relu_fwd.argtypes = [vp, vp, vp, sz, i32]
@@ -210,6 +212,12 @@ def _bwd(fn, g, codes, meta, L, dt, threads):
 def gelu_fwd(x, row_len: int, dt: int, threads: int = 1):
     """Returns (y, packed codes, meta) for the GELU forward with the 4-bit stash."""
     return _fwd(lib().s2a_oracle_gelu_fwd, x, row_len, dt, threads)
+
+
+def gelu_fwd_tensor_range(x, row_len: int, dt: int):
+    """GELU forward whose 4-bit stash uses ONE (min, s) for the whole tensor."""
+    fn = lib().s2a_oracle_gelu_fwd_tensor_range
+    return _fwd(lambda a, b, c, d, n, L, t, _threads: fn(a, b, c, d, n, L, t), x, row_len, dt, 1)
 
 
 def gelu_bwd(g, codes, meta, row_len: int, dt: int, threads: int = 1):

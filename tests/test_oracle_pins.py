@@ -346,6 +346,40 @@ def test_bad_shapes_are_rejected_and_empty_is_fine():
     assert y.size == 0 and c.size == 0 and m.size == 0
 
 
+# ------------------------------------------------------------------ per-tensor range reading
+@pytest.mark.parametrize("dt", [F32, BF16])
+def test_gelu_tensor_range_reading(dt):
+    rows, L = 6, 40
+    # small-variance rows: no row reaches the clip, rows have different ranges
+    x32 = synth.normal(8, ("tr", dt), rows * L) * 0.3
+    x32[5] = 1.9
+    x = synth.to_io(x32, dt)
+    y, codes, meta = o.gelu_fwd_tensor_range(x, L, dt)
+    y_row, codes_row, meta_row = o.gelu_fwd(x, L, dt)
+    assert np.array_equal(y, y_row)                        # only the stash differs
+    c = np.clip(o.widen(x, dt), -2, 2).astype(np.float32)
+    want, tie = _exact_codes(c)                            # Eq. 8 over the whole tensor, exactly
+    q = o.unpack(codes, rows * L)
+    ok = ~np.array(tie)
+    assert np.array_equal(q[ok], np.array(want)[ok])
+    assert np.all(meta[0::2] == np.float32(c.min()))
+    assert np.all(meta[1::2] == np.float32(np.float32(c.max() - c.min()) / np.float32(15)))
+    assert not np.array_equal(codes, codes_row)            # and it IS a different stash here
+    # on a tensor whose every row saturates the clip the two readings coincide
+    xs = synth.to_io(synth.gelu_preact(8, ("trs", dt), 4 * 3072), dt)
+    a = o.gelu_fwd_tensor_range(xs, 3072, dt)
+    b = o.gelu_fwd(xs, 3072, dt)
+    for u, v in zip(a, b):
+        assert np.array_equal(u, v)
+    # the backward pass takes this stash as it is
+    g = synth.to_io(synth.normal(8, ("trg", dt), rows * L), dt)
+    gin = o.widen(o.gelu_bwd(g, codes, meta, L, dt), dt)
+    xh = q.astype(np.float64) * float(meta[1]) + float(meta[0])
+    wantg = o.widen(g, dt) * (sp.expit(A * xh) + B * np.sin(W * xh))
+    tol = 2.0 ** -24 if dt == F32 else 2.0 ** -8
+    assert np.all(np.abs(gin - wantg) <= tol * np.abs(wantg) + 1e-40)
+
+
 # ------------------------------------------------------------------ ReLU 1-bit stash
 @pytest.mark.parametrize("dt", [F32, BF16])
 @pytest.mark.parametrize("n", [1, 7, 8, 9, 1000, 4099])
