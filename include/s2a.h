@@ -102,6 +102,26 @@ int s2a_softmax_fwd(const void* x, void* y, uint8_t* codes, float* meta, size_t 
 int s2a_softmax_bwd(const void* grad_out, const uint8_t* codes, const float* meta, void* grad_in,
                     size_t n_elems, size_t row_len, int dt, void* cuda_stream);
 
+/* Bytes of scratch memory s2a_gelu_fwd_tensor_range needs for n_elems elements:
+ * 8 + 8 * ceil(n_elems / 65536). */
+size_t s2a_tensor_range_scratch_bytes(size_t n_elems);
+
+/* GELU forward whose stash uses ONE quantiser range for the whole tensor -- the other
+ * reading of Section 3.2, "GeLU layer" ("quantized between the maximal and minimal value"):
+ * Eq. 8's min and max are taken over the whole clipped tensor.  y is as for s2a_gelu_fwd;
+ * every row's metadata carries the same (min, s), so s2a_gelu_bwd consumes the stash
+ * unchanged.  The range must be known before the first code, so x is read twice
+ * (6.5 bytes per bfloat16 element instead of 4.5).  Three kernels are enqueued.
+ *   x, y, codes, meta  as for s2a_gelu_fwd, except that y must NOT alias x
+ *   scratch            device memory, s2a_tensor_range_scratch_bytes(n_elems) bytes, 8-byte
+ *                      aligned, owned by the caller; contents on entry are ignored, and it
+ *                      must not be used by other work on the GPU until the call's kernels
+ *                      have finished
+ * Errors as for s2a_gelu_fwd; x == y returns S2A_ERR_ALIGN.
+ */
+int s2a_gelu_fwd_tensor_range(const void* x, void* y, uint8_t* codes, float* meta, void* scratch,
+                              size_t n_elems, size_t row_len, int dt, void* cuda_stream);
+
 /* Bytes of the ReLU bit mask for n_elems elements: (n_elems + 7) / 8. */
 size_t s2a_mask_bytes(size_t n_elems);
 

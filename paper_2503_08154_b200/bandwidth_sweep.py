@@ -85,6 +85,31 @@ def _time_relu(n: int, dtype, seed: int):
     return alg / t_f / 1e9, alg / t_b / 1e9, 2 * alg / (t_f + t_b) / 1e9
 
 
+def _time_tensor_range(rows: int, L: int, dtype, seed: int):
+    n = rows * L
+    item = 2 if dtype == torch.bfloat16 else 4
+    sets = max(1, min(8, int(3e8 // (2 * n * item)) + 1))
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    xs = [torch.randn(n, device="cuda", generator=g).to(dtype) for _ in range(sets)]
+    ys = [torch.empty_like(x) for x in xs]
+    st = [binding.alloc_stash(n, L, "cuda") for _ in range(sets)]
+    scratch = torch.empty(binding.tensor_range_scratch_bytes(n), dtype=torch.uint8, device="cuda")
+    iters = max(4, min(200, int(2e10 // (n * item * 4))))
+    for i in range(min(3, sets)):
+        binding.s2a_gelu_fwd_tensor_range(xs[i], ys[i], st[i][0], st[i][1], scratch, L)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(iters):
+        k = i % sets
+        binding.s2a_gelu_fwd_tensor_range(xs[k], ys[k], st[k][0], st[k][1], scratch, L)
+    e1.record()
+    torch.cuda.synchronize()
+    t = e0.elapsed_time(e1) * 1e-3 / iters
+    alg = 3 * n * item + (n + 1) // 2 + 8 * rows   # x twice, y, codes, metadata
+    return alg / t / 1e9
+
+
 def cases(quick: bool):
     out = []
     for n in ((1e6, 1e8) if quick else (1e6, 1e7, 1e8, 1e9, 2e9)):
@@ -116,6 +141,15 @@ def main():
                               "seeds": args.seeds, "fwd_GBps": round(med[0], 1), "bwd_GBps": round(med[1], 1),
                               "fwd_bwd_GBps": round(med[2], 1),
                               "note": "algorithmic bytes = 2*n*itemsize + n/8 per kernel"}), flush=True)
+    for n in ((10**6, 10**8) if args.quick else (10**6, 10**7, 10**8, 10**9)):
+        for dtype in (torch.bfloat16, torch.float32):
+            rows = max(2, int(n) // 4096)
+            res = [_time_tensor_range(rows, 4096, dtype, seed) for seed in range(args.seeds)]
+            torch.cuda.empty_cache()
+            print(json.dumps({"kernel": "gelu_fwd_tensor_range", "rows": rows, "row_len": 4096, "elems": rows * 4096,
+                              "io_dtype": "bf16" if dtype == torch.bfloat16 else "f32", "seeds": args.seeds,
+                              "GBps": round(statistics.median(res), 1),
+                              "note": "algorithmic bytes = 3*n*itemsize + n/2 + 8*rows (x is read twice)"}), flush=True)
     for kind, rows, L, dtype in cases(args.quick):
         res = []
         for seed in range(args.seeds):

@@ -23,6 +23,7 @@ EXPORTS = (
     "s2a_codes_bytes", "s2a_meta_bytes", "s2a_status_string", "s2a_gelu_fwd", "s2a_gelu_bwd",
     "s2a_softmax_fwd", "s2a_softmax_bwd", "s2a_device_error", "s2a_describe_plan",
     "s2a_mask_bytes", "s2a_relu_fwd", "s2a_relu_bwd",
+    "s2a_tensor_range_scratch_bytes", "s2a_gelu_fwd_tensor_range",
 )
 
 _lib = None
@@ -52,6 +53,11 @@ def lib() -> ctypes.CDLL:
             f.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_size_t, c.c_size_t,
                           c.c_int, c.c_void_p]
             f.restype = c.c_int
+        L.s2a_tensor_range_scratch_bytes.argtypes = [c.c_size_t]
+        L.s2a_tensor_range_scratch_bytes.restype = c.c_size_t
+        L.s2a_gelu_fwd_tensor_range.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
+                                                c.c_size_t, c.c_size_t, c.c_int, c.c_void_p]
+        L.s2a_gelu_fwd_tensor_range.restype = c.c_int
         L.s2a_mask_bytes.argtypes = [c.c_size_t]
         L.s2a_mask_bytes.restype = c.c_size_t
         for name in ("s2a_relu_fwd", "s2a_relu_bwd"):
@@ -150,6 +156,27 @@ def s2a_softmax_fwd(x, y, codes, meta, row_len: int) -> None:
 
 def s2a_softmax_bwd(grad_out, codes, meta, grad_in, row_len: int) -> None:
     _bwd(lib().s2a_softmax_bwd, grad_out, codes, meta, grad_in, row_len)
+
+
+def tensor_range_scratch_bytes(n_elems: int) -> int:
+    return int(lib().s2a_tensor_range_scratch_bytes(n_elems))
+
+
+def s2a_gelu_fwd_tensor_range(x, y, codes, meta, scratch, row_len: int) -> None:
+    """GELU forward with one quantiser range for the whole tensor; `scratch` is a uint8 CUDA
+    tensor of at least tensor_range_scratch_bytes(x.numel()) bytes."""
+    _dev(x, "x"), _dev(y, "y"), _dev(codes, "codes"), _dev(meta, "meta"), _dev(scratch, "scratch")
+    n = x.numel()
+    if y.numel() != n or y.dtype != x.dtype:
+        raise S2AError("y must match x in size and dtype")
+    if codes.dtype != torch.uint8 or meta.dtype != torch.float32:
+        raise S2AError("codes must be uint8 and meta float32")
+    if row_len > 0 and (codes.numel() < codes_bytes(n) or meta.numel() * 4 < meta_bytes(n, row_len)):
+        raise S2AError("codes/meta buffers are too small")
+    if scratch.numel() * scratch.element_size() < tensor_range_scratch_bytes(n):
+        raise S2AError("scratch is too small")
+    check(lib().s2a_gelu_fwd_tensor_range(x.data_ptr(), y.data_ptr(), codes.data_ptr(), meta.data_ptr(),
+                                          scratch.data_ptr(), n, row_len, dtype_code(x), _stream_ptr()))
 
 
 def mask_bytes(n_elems: int) -> int:

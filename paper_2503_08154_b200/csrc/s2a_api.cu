@@ -90,6 +90,20 @@ int s2a_softmax_bwd(const void* grad_out, const uint8_t* codes, const float* met
              const_cast<float*>(meta), n_elems, row_len, dt, cuda_stream);
 }
 
+size_t s2a_tensor_range_scratch_bytes(size_t n_elems) { return (size_t)tensor_range_scratch_bytes(n_elems); }
+
+int s2a_gelu_fwd_tensor_range(const void* x, void* y, uint8_t* codes, float* meta, void* scratch,
+                              size_t n_elems, size_t row_len, int dt, void* cuda_stream) {
+  int rc = check_args(x, y, codes, meta, n_elems, row_len, dt);
+  if (rc != S2A_OK || n_elems == 0) return rc;
+  if (!scratch) return S2A_ERR_NULL;
+  if (misaligned(scratch, 8)) return S2A_ERR_ALIGN;
+  // x is read again after y has been written: the two may not alias in this variant
+  if (x == (const void*)y) return S2A_ERR_ALIGN;
+  return launch_gelu_fwd_tensor_range(dt, x, y, codes, meta, (float*)scratch, n_elems, n_elems / row_len,
+                                      (cudaStream_t)cuda_stream) == cudaSuccess ? S2A_OK : S2A_ERR_CUDA;
+}
+
 size_t s2a_mask_bytes(size_t n_elems) { return (n_elems + 7) / 8; }
 
 static int run_relu(bool fwd, const void* in, void* out, uint8_t* mask, size_t n, int dt, void* stream) {

@@ -26,6 +26,12 @@ cudaError_t launch_rowwise(int kernel, int dt, const RowwiseArgs& a, cudaStream_
 // ReLU with its 1-bit mask: in = x (forward) or grad_out (backward), out = y or grad_in.
 cudaError_t launch_relu(bool fwd, int dt, const void* in, void* out, uint8_t* mask, uint64_t n, cudaStream_t st);
 
+// GELU forward with one quantiser range for the whole tensor (two reads of x).  `scratch`
+// is device memory of tensor_range_scratch_bytes(n) bytes, 8-byte aligned.
+uint64_t tensor_range_scratch_bytes(uint64_t n);
+cudaError_t launch_gelu_fwd_tensor_range(int dt, const void* x, void* y, uint8_t* codes, float* meta, float* scratch,
+                                         uint64_t n, uint64_t n_rows, cudaStream_t st);
+
 // ---------------------------------------------------------------- pipelined tiles
 // A tile is `tile_rows` consecutive rows whose flat element span starts and ends on a
 // multiple of 32 elements, so that its data and its code bytes can move with 16-byte

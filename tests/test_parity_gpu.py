@@ -248,6 +248,49 @@ def test_tensor_beyond_2_to_31_elements_uses_64_bit_indexing():
     pu.assert_close(pu.widen(pu.to_host(gv[repeats - 1], BF16), BF16), pu.widen(gin_o, BF16), BF16, "gelu grad_in (large)")
 
 
+# ------------------------------------------------------------------ per-tensor range variant
+@pytest.mark.parametrize("dt", [F32, BF16])
+@pytest.mark.parametrize("rows,L,scale", [(3, 5, 0.3), (1, 1, 1.0), (7, 197, 0.2), (300, 66, 0.4), (64, 3072, 0.25),
+                                          (1576, 3072, 1.3), (40, 65536, 0.5), (3, 100003, 0.3)])
+def test_gelu_tensor_range(rows, L, scale, dt):
+    n = rows * L
+    x = synth.to_io(synth.gelu_preact(7, ("gtr", rows, L, dt), n) * np.float32(scale), dt)
+    g = synth.to_io(synth.normal(7, ("gtrg", rows, L, dt), n), dt)
+    y_o, codes_o, meta_o = o.gelu_fwd_tensor_range(x, L, dt)
+    item = synth.io_itemsize(dt)
+    tdt = pu.torch_dtype(dt)
+    xd = pu.to_device(x, dt)
+    yg, cg, mg = pu.Guarded(n * item), pu.Guarded(binding.codes_bytes(n)), pu.Guarded(binding.meta_bytes(n, L))
+    sg = pu.Guarded(binding.tensor_range_scratch_bytes(n))
+    binding.s2a_gelu_fwd_tensor_range(xd, yg.view(tdt), cg.view(torch.uint8), mg.view(torch.float32),
+                                      sg.view(torch.uint8), L)
+    torch.cuda.synchronize()
+    for buf, what in ((yg, "y"), (cg, "codes"), (mg, "meta"), (sg, "scratch")):
+        buf.check("gelu_fwd_tensor_range " + what)
+    assert np.array_equal(pu.to_host(xd, dt), x)
+    assert np.array_equal(cg.view(torch.uint8).cpu().numpy(), codes_o)
+    assert np.array_equal(mg.view(torch.float32).cpu().numpy().view(np.uint32), meta_o.view(np.uint32))
+    pu.assert_close(pu.widen(pu.to_host(yg.view(tdt), dt), dt), pu.widen(y_o, dt), dt, "gelu y (tensor range)")
+    # the ordinary backward consumes this stash
+    gin_o = o.gelu_bwd(g, codes_o, meta_o, L, dt, threads=THREADS)
+    gin_g = pu.gpu_bwd("gelu", g, codes_o, meta_o, L, dt)
+    pu.assert_close(pu.widen(gin_g, dt), pu.widen(gin_o, dt), dt, "gelu grad_in (tensor range)")
+
+
+def test_gelu_tensor_range_rejects_aliasing_and_missing_scratch():
+    L = binding.lib()
+    x = torch.zeros(64, device="cuda")
+    y = torch.zeros(64, device="cuda")
+    codes, meta = binding.alloc_stash(64, 8, "cuda")
+    scratch = torch.zeros(64, dtype=torch.uint8, device="cuda")
+    s = torch.cuda.current_stream().cuda_stream
+    f = L.s2a_gelu_fwd_tensor_range
+    assert f(x.data_ptr(), x.data_ptr(), codes.data_ptr(), meta.data_ptr(), scratch.data_ptr(), 64, 8, 0, s) == 3
+    assert f(x.data_ptr(), y.data_ptr(), codes.data_ptr(), meta.data_ptr(), None, 64, 8, 0, s) == 1
+    assert f(x.data_ptr(), y.data_ptr(), codes.data_ptr(), meta.data_ptr(), scratch.data_ptr(), 63, 8, 0, s) == 2
+    assert binding.tensor_range_scratch_bytes(1) == 16 and binding.tensor_range_scratch_bytes(65537) == 24
+
+
 # ------------------------------------------------------------------ ReLU with a 1-bit stash
 @pytest.mark.parametrize("dt", [F32, BF16])
 @pytest.mark.parametrize("n", [1, 7, 8, 9, 1023, 1024 * 8, 100003, 5_000_001, 40_000_008])
