@@ -55,7 +55,8 @@ typedef enum {
   S2A_ERR_ALIGN = 3,  /* a pointer is not aligned as stated above                */
   S2A_ERR_DTYPE = 4,  /* dt is neither S2A_F32 nor S2A_BF16                      */
   S2A_ERR_CUDA = 5,   /* the CUDA runtime refused the launch                     */
-  S2A_ERR_DEVICE = 6  /* a kernel gave up on a bounded wait (see s2a_device_error) */
+  S2A_ERR_DEVICE = 6, /* a kernel gave up on a bounded wait (see s2a_device_error) */
+  S2A_ERR_TOO_LARGE = 7 /* beyond the built-in scratch of s2a_gelu_fwd_tensor_range_static */
 } s2a_status;
 
 /* Bytes of packed codes for n_elems elements: (n_elems + 1) / 2. */
@@ -121,6 +122,39 @@ size_t s2a_tensor_range_scratch_bytes(size_t n_elems);
  */
 int s2a_gelu_fwd_tensor_range(const void* x, void* y, uint8_t* codes, float* meta, void* scratch,
                               size_t n_elems, size_t row_len, int dt, void* cuda_stream);
+
+/* Largest n_elems s2a_gelu_fwd_tensor_range_static accepts: 536,870,912 (8192 chunks of
+ * 65,536 elements). */
+size_t s2a_tensor_range_static_max_elems(void);
+
+/* s2a_gelu_fwd_tensor_range for callers that cannot hand the library any scratch memory.
+ * (The paper has no counterpart to this entry point; it exists for the sake of such
+ * callers only and computes exactly what s2a_gelu_fwd_tensor_range computes.)
+ *
+ * Who this is for: code that is not allowed to allocate device memory at the point of the
+ * call -- a plug-in whose host application owns the device allocator, a serving or
+ * real-time loop in which a cudaMalloc would synchronise the device and stall every other
+ * stream, a program that must fix its whole memory plan before it starts -- and that has
+ * no spare buffer of its own to lend.  This entry point calls no cudaMalloc, cudaFree or
+ * any other allocating routine.  Its range partials go to a fixed array of 65,544 bytes
+ * that is part of the library image: every GPU that loads libs2a.so holds that array from
+ * load to exit, whether or not this function is ever called.
+ *
+ * Limits and rules:
+ * - n_elems <= s2a_tensor_range_static_max_elems(); a larger tensor returns
+ *   S2A_ERR_TOO_LARGE and nothing is enqueued (use the variant with caller scratch).
+ * - All calls on one GPU share the one array.  It keeps whatever the previous call left;
+ *   nothing in it needs to start at zero, because each call overwrites every slot it later
+ *   reads.  Two calls whose kernels can run at the same time on the same GPU (different
+ *   streams, different host threads) race on it and produce wrong codes: keep such calls
+ *   on one stream or order them yourself.
+ * - The first call on each GPU looks up the array's device address (with that GPU current);
+ *   make that first call outside any stream capture.
+ * Arguments, aliasing rule (y must not alias x) and the other errors are those of
+ * s2a_gelu_fwd_tensor_range without `scratch`.
+ */
+int s2a_gelu_fwd_tensor_range_static(const void* x, void* y, uint8_t* codes, float* meta, size_t n_elems,
+                                     size_t row_len, int dt, void* cuda_stream);
 
 /* Bytes of the ReLU bit mask for n_elems elements: (n_elems + 7) / 8. */
 size_t s2a_mask_bytes(size_t n_elems);

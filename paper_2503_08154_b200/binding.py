@@ -24,6 +24,7 @@ EXPORTS = (
     "s2a_softmax_fwd", "s2a_softmax_bwd", "s2a_device_error", "s2a_describe_plan",
     "s2a_mask_bytes", "s2a_relu_fwd", "s2a_relu_bwd",
     "s2a_tensor_range_scratch_bytes", "s2a_gelu_fwd_tensor_range",
+    "s2a_tensor_range_static_max_elems", "s2a_gelu_fwd_tensor_range_static",
 )
 
 _lib = None
@@ -58,6 +59,11 @@ def lib() -> ctypes.CDLL:
         L.s2a_gelu_fwd_tensor_range.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
                                                 c.c_size_t, c.c_size_t, c.c_int, c.c_void_p]
         L.s2a_gelu_fwd_tensor_range.restype = c.c_int
+        L.s2a_tensor_range_static_max_elems.argtypes = []
+        L.s2a_tensor_range_static_max_elems.restype = c.c_size_t
+        L.s2a_gelu_fwd_tensor_range_static.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_size_t,
+                                                       c.c_size_t, c.c_int, c.c_void_p]
+        L.s2a_gelu_fwd_tensor_range_static.restype = c.c_int
         L.s2a_mask_bytes.argtypes = [c.c_size_t]
         L.s2a_mask_bytes.restype = c.c_size_t
         for name in ("s2a_relu_fwd", "s2a_relu_bwd"):
@@ -177,6 +183,27 @@ def s2a_gelu_fwd_tensor_range(x, y, codes, meta, scratch, row_len: int) -> None:
         raise S2AError("scratch is too small")
     check(lib().s2a_gelu_fwd_tensor_range(x.data_ptr(), y.data_ptr(), codes.data_ptr(), meta.data_ptr(),
                                           scratch.data_ptr(), n, row_len, dtype_code(x), _stream_ptr()))
+
+
+def tensor_range_static_max_elems() -> int:
+    return int(lib().s2a_tensor_range_static_max_elems())
+
+
+def s2a_gelu_fwd_tensor_range_static(x, y, codes, meta, row_len: int) -> None:
+    """s2a_gelu_fwd_tensor_range without a scratch argument, for callers that may not
+    allocate device memory: the range partials live in a fixed array inside the library
+    (shared by all calls on a GPU -- do not overlap them), and tensors beyond
+    tensor_range_static_max_elems() elements are refused."""
+    _dev(x, "x"), _dev(y, "y"), _dev(codes, "codes"), _dev(meta, "meta")
+    n = x.numel()
+    if y.numel() != n or y.dtype != x.dtype:
+        raise S2AError("y must match x in size and dtype")
+    if codes.dtype != torch.uint8 or meta.dtype != torch.float32:
+        raise S2AError("codes must be uint8 and meta float32")
+    if row_len > 0 and (codes.numel() < codes_bytes(n) or meta.numel() * 4 < meta_bytes(n, row_len)):
+        raise S2AError("codes/meta buffers are too small")
+    check(lib().s2a_gelu_fwd_tensor_range_static(x.data_ptr(), y.data_ptr(), codes.data_ptr(), meta.data_ptr(),
+                                                 n, row_len, dtype_code(x), _stream_ptr()))
 
 
 def mask_bytes(n_elems: int) -> int:

@@ -64,6 +64,9 @@ const char* s2a_status_string(int status) {
     case S2A_ERR_DTYPE: return "S2A_ERR_DTYPE: dt must be S2A_F32 or S2A_BF16";
     case S2A_ERR_CUDA: return "S2A_ERR_CUDA: the CUDA runtime refused the launch";
     case S2A_ERR_DEVICE: return "S2A_ERR_DEVICE: a kernel gave up on a bounded wait";
+    case S2A_ERR_TOO_LARGE:
+      return "S2A_ERR_TOO_LARGE: n_elems exceeds the built-in scratch of the allocation-free entry point "
+             "(536,870,912 elements); use s2a_gelu_fwd_tensor_range with your own scratch";
     default: return "unknown s2a status";
   }
 }
@@ -102,6 +105,18 @@ int s2a_gelu_fwd_tensor_range(const void* x, void* y, uint8_t* codes, float* met
   if (x == (const void*)y) return S2A_ERR_ALIGN;
   return launch_gelu_fwd_tensor_range(dt, x, y, codes, meta, (float*)scratch, n_elems, n_elems / row_len,
                                       (cudaStream_t)cuda_stream) == cudaSuccess ? S2A_OK : S2A_ERR_CUDA;
+}
+
+size_t s2a_tensor_range_static_max_elems(void) { return (size_t)tensor_range_static_max_elems(); }
+
+int s2a_gelu_fwd_tensor_range_static(const void* x, void* y, uint8_t* codes, float* meta, size_t n_elems,
+                                     size_t row_len, int dt, void* cuda_stream) {
+  int rc = check_args(x, y, codes, meta, n_elems, row_len, dt);
+  if (rc != S2A_OK || n_elems == 0) return rc;
+  if (n_elems > tensor_range_static_max_elems()) return S2A_ERR_TOO_LARGE;
+  if (x == (const void*)y) return S2A_ERR_ALIGN;
+  return launch_gelu_fwd_tensor_range_static(dt, x, y, codes, meta, n_elems, n_elems / row_len,
+                                             (cudaStream_t)cuda_stream) == cudaSuccess ? S2A_OK : S2A_ERR_CUDA;
 }
 
 size_t s2a_mask_bytes(size_t n_elems) { return (n_elems + 7) / 8; }

@@ -32,6 +32,12 @@ uint64_t tensor_range_scratch_bytes(uint64_t n);
 cudaError_t launch_gelu_fwd_tensor_range(int dt, const void* x, void* y, uint8_t* codes, float* meta, float* scratch,
                                          uint64_t n, uint64_t n_rows, cudaStream_t st);
 
+// The same three kernels with their scratch in a static device array of the library; no
+// allocation anywhere.  n must not exceed tensor_range_static_max_elems().
+uint64_t tensor_range_static_max_elems();
+cudaError_t launch_gelu_fwd_tensor_range_static(int dt, const void* x, void* y, uint8_t* codes, float* meta,
+                                                uint64_t n, uint64_t n_rows, cudaStream_t st);
+
 // ---------------------------------------------------------------- pipelined tiles
 // A tile is `tile_rows` consecutive rows whose flat element span starts and ends on a
 // multiple of 32 elements, so that its data and its code bytes can move with 16-byte

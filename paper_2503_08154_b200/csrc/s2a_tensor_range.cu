@@ -140,7 +140,36 @@ __global__ void __launch_bounds__(kThreads) fixed_range_fwd(const void* x, void*
   }
 }
 
+// Scratch of the allocation-free entry point: room for the range partials of
+// kStaticChunks chunks.  It lives in every GPU that loads the library, from load to exit,
+// and is shared by all calls of that entry point on the device.
+constexpr uint32_t kStaticChunks = 8192;  // 8192 * 65,536 = 536,870,912 elements at most
+static __device__ __align__(256) float g_static_range_scratch[2 + 2 * kStaticChunks];  // 65,544 bytes
+
 }  // namespace
+
+uint64_t tensor_range_static_max_elems() { return (uint64_t)kStaticChunks * kChunk; }
+
+// In host code `g_static_range_scratch` is only a handle for the runtime, not an address
+// the GPU understands: the device address is looked up once per device (with that device
+// current) and that pointer is what the kernels receive.
+cudaError_t launch_gelu_fwd_tensor_range_static(int dt, const void* x, void* y, uint8_t* codes, float* meta,
+                                                uint64_t n, uint64_t n_rows, cudaStream_t st) {
+  static float* device_address[64] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (device_address[dev] == nullptr) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_static_range_scratch);
+    if (e != cudaSuccess) return e;
+    device_address[dev] = (float*)p;
+  }
+  // Nothing in the scratch has to start at zero: the first kernel overwrites the partial of
+  // every chunk this call uses, the second overwrites the folded range, the third only reads.
+  return launch_gelu_fwd_tensor_range(dt, x, y, codes, meta, device_address[dev], n, n_rows, st);
+}
 
 uint64_t tensor_range_scratch_bytes(uint64_t n) {
   return 8 + 8 * ((n + kChunk - 1) / kChunk);
