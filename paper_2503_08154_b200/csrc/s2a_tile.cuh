@@ -285,6 +285,24 @@ struct Unit {
   }
 };
 
+// Row minimum and maximum of bfloat16-valued numbers in ONE shuffle sequence: the pair
+// (min, -max) travels as a packed bfloat16x2 and is folded with a packed minimum (negation
+// is exact).  Sub-warp and warp units only.
+template <int UNIT>
+__device__ __forceinline__ void reduce_minmax_bf16(float& mn, float& mx) {
+  static_assert(UNIT <= 32, "warp-level reduction");
+  __nv_bfloat162 p = __floats2bfloat162_rn(mn, -mx);  // exact: both are bfloat16 values (or +-inf)
+  uint32_t w = *(uint32_t*)&p;
+#pragma unroll
+  for (int o = UNIT / 2; o > 0; o >>= 1) {
+    uint32_t other = __shfl_xor_sync(0xffffffffu, w, o);
+    __nv_bfloat162 r = __hmin2(*(__nv_bfloat162*)&w, *(__nv_bfloat162*)&other);
+    w = *(uint32_t*)&r;
+  }
+  mn = __uint_as_float(w << 16);
+  mx = -__uint_as_float(w & 0xffff0000u);
+}
+
 // Geometry of one row inside a tile, in accesses.
 struct RowGeom {
   uint32_t a0;    // first access (tile-relative)
@@ -835,29 +853,38 @@ struct StreamSoftmaxFwd {
     m = u.template reduce<kOpMax>(m);
     if (!active) m = 0.0f;
     float z = 0.0f;
+    constexpr float kLog2e = 1.4426950408889634f;
+    const float nm = -m * kLog2e;
 #pragma unroll
     for (int i = 0; i < NV; ++i)
 #pragma unroll
       for (int k = 0; k < EPA; ++k) {
-        e[i][k] = exp_eval<DT>(e[i][k] - m);
+        // bfloat16: the exponent's argument is one fused multiply-add (the result is rounded to 8 bits)
+        e[i][k] = DT == kBF16 ? ex2_approx(fmaf(e[i][k], kLog2e, nm)) : exp_eval<DT>(e[i][k] - m);
         z += e[i][k];
       }
     z = u.template reduce<kOpSum>(z);
     const float rz = __fdiv_rn(1.0f, active ? z : 1.0f);
-    float mn = INFINITY, mx = -INFINITY;
+    typename V::MinMax mm;
+    mm.init();
 #pragma unroll
     for (int i = 0; i < NV; ++i) {
       const uint32_t j = u.ul + UNIT_ * i;
       if (j < nv) {
 #pragma unroll
         for (int k = 0; k < EPA; ++k) e[i][k] *= rz;
-        *(typename V::Raw*)(row + j * 16u) = V::narrow(e[i]);  // e now holds y as written
-#pragma unroll
-        for (int k = 0; k < EPA; ++k) { mn = fminf(mn, e[i][k]); mx = fmaxf(mx, e[i][k]); }
+        const typename V::Raw yw = V::narrow(e[i]);  // e now holds y as written
+        *(typename V::Raw*)(row + j * 16u) = yw;
+        mm.add(yw);
       }
     }
-    mn = u.template reduce<kOpMin>(mn);
-    mx = u.template reduce<kOpMax>(mx);
+    float mn = mm.lo(), mx = mm.hi();
+    if (DT == kBF16) {
+      reduce_minmax_bf16<UNIT_>(mn, mx);
+    } else {
+      mn = u.template reduce<kOpMin>(mn);
+      mx = u.template reduce<kOpMax>(mx);
+    }
     const QRange q = make_qrange(mn, mx);
     if (active && u.ul == 0) { p.meta[2 * r] = q.mn; p.meta[2 * r + 1] = q.s; }
 #pragma unroll
@@ -1137,8 +1164,8 @@ struct PairSoftmaxFwd<kBF16, UNIT_, LCT> {
         }
       }
     }
-    const float mn = u.template reduce<kOpMin>(fminf(lo(mn2), hi(mn2)));
-    const float mx = u.template reduce<kOpMax>(fmaxf(lo(mx2), hi(mx2)));
+    float mn = fminf(lo(mn2), hi(mn2)), mx = fmaxf(lo(mx2), hi(mx2));
+    reduce_minmax_bf16<UNIT_>(mn, mx);
     const QRange q = make_qrange(mn, mx);
     if (active && ul == 0) { p.meta[2 * r] = q.mn; p.meta[2 * r + 1] = q.s; }
     unsigned char* cb = p.codes + a0 + ul;
