@@ -265,6 +265,62 @@ int s2a_oracle_gelu_fwd(const void* x, void* y, uint8_t* codes, float* meta, siz
   return 0;
 }
 
+}  // extern "C"
+
+namespace {
+// ---- SiLU / Swish (Section 3.2, last sentence of "GeLU layer": the design "is also
+// effective for similar non-parametric functions, such as SiLU and Swish"; the paper gives
+// no constants for them).  Reading taken here: y = x * sigmoid(x); the input is clipped to
+// [-C, C] with C = 2 * 1.702 (the same range of the sigmoid's argument as GELU's [-2, 2]),
+// quantised per row with Eq. 8, and the backward pass evaluates the EXACT derivative
+// sigmoid(x)(1 + x(1 - sigmoid(x))) at the dequantised input.
+const double kSiluClip = (double)(2.0f * 1.702f);
+
+double silu(double x) { return x * sigmoid(x); }
+double silu_grad(double x) {
+  double s = sigmoid(x);
+  return s * (1.0 + x * (1.0 - s));
+}
+}  // namespace
+
+extern "C" {
+double s2a_oracle_silu(double x) { return silu(x); }
+double s2a_oracle_silu_grad(double x) { return silu_grad(x); }
+
+int s2a_oracle_silu_fwd(const void* x, void* y, uint8_t* codes, float* meta, size_t n, size_t L, int dt,
+                        int threads) {
+  if (n == 0) return 0;
+  if (bad_shape(n, L)) return 2;
+  std::vector<uint8_t> q(n);
+  for_rows(n / L, threads, [&](size_t r) {
+    std::vector<float> c(L);
+    for (size_t i = 0; i < L; ++i) {
+      double xi = load_elem(x, r * L + i, dt);
+      c[i] = (float)std::min(std::max(xi, -kSiluClip), kSiluClip);  // exact: the bound is binary32
+      store_elem(y, r * L + i, dt, silu(xi));
+    }
+    quantize_row(c.data(), L, &q[r * L], &meta[2 * r], &meta[2 * r + 1]);
+  });
+  pack_codes(q.data(), n, codes);
+  return 0;
+}
+
+int s2a_oracle_silu_bwd(const void* g, const uint8_t* codes, const float* meta, void* gin, size_t n, size_t L,
+                        int dt, int threads) {
+  if (n == 0) return 0;
+  if (bad_shape(n, L)) return 2;
+  std::vector<uint8_t> q(n);
+  unpack_codes(codes, n, q.data());
+  for_rows(n / L, threads, [&](size_t r) {
+    float mn = meta[2 * r], s = meta[2 * r + 1];
+    for (size_t i = 0; i < L; ++i) {
+      double xh = dequantize(q[r * L + i], mn, s);
+      store_elem(gin, r * L + i, dt, load_elem(g, r * L + i, dt) * silu_grad(xh));
+    }
+  });
+  return 0;
+}
+
 // ---- GELU forward, per-TENSOR range: the other reading of "quantized between the maximal
 // and minimal value" (Section 3.2, "GeLU layer"): Eq. 8's min and max are taken over the
 // whole clipped tensor instead of over each row.  Every row's metadata carries the same

@@ -46,7 +46,8 @@ def lib() -> ctypes.CDLL:
         L = ctypes.CDLL(build())
         c = ctypes
         sz, vp, dbl, flt, i32 = c.c_size_t, c.c_void_p, c.c_double, c.c_float, c.c_int
-        for name in ("s2a_oracle_gelu", "s2a_oracle_gelu_grad_exact", "s2a_oracle_gelu_grad_sine"):
+        for name in ("s2a_oracle_gelu", "s2a_oracle_gelu_grad_exact", "s2a_oracle_gelu_grad_sine",
+                     "s2a_oracle_silu", "s2a_oracle_silu_grad"):
             getattr(L, name).argtypes = [dbl]
             getattr(L, name).restype = dbl
         L.s2a_oracle_softmax_row.argtypes = [vp, vp, sz]
@@ -67,10 +68,10 @@ def lib() -> ctypes.CDLL:
         L.s2a_oracle_round_bf16.restype = c.c_uint16
         L.s2a_oracle_bf16_to_float.argtypes = [c.c_uint16]
         L.s2a_oracle_bf16_to_float.restype = flt
-        for name in ("s2a_oracle_gelu_fwd", "s2a_oracle_softmax_fwd"):
+        for name in ("s2a_oracle_gelu_fwd", "s2a_oracle_softmax_fwd", "s2a_oracle_silu_fwd"):
             getattr(L, name).argtypes = [vp, vp, vp, vp, sz, sz, i32, i32]
             getattr(L, name).restype = i32
-        for name in ("s2a_oracle_gelu_bwd", "s2a_oracle_softmax_bwd"):
+        for name in ("s2a_oracle_gelu_bwd", "s2a_oracle_softmax_bwd", "s2a_oracle_silu_bwd"):
             getattr(L, name).argtypes = [vp, vp, vp, vp, sz, sz, i32, i32]
             getattr(L, name).restype = i32
         L.s2a_oracle_gelu_fwd_tensor_range.argtypes = [vp, vp, vp, vp, sz, sz, i32]
@@ -222,6 +223,23 @@ def gelu_fwd_tensor_range(x, row_len: int, dt: int):
 
 def gelu_bwd(g, codes, meta, row_len: int, dt: int, threads: int = 1):
     return _bwd(lib().s2a_oracle_gelu_bwd, g, codes, meta, row_len, dt, threads)
+
+
+def silu(x: float) -> float:
+    return lib().s2a_oracle_silu(float(x))
+
+
+def silu_grad(x: float) -> float:
+    return lib().s2a_oracle_silu_grad(float(x))
+
+
+def silu_fwd(x, row_len: int, dt: int, threads: int = 1):
+    """Returns (y, packed codes, meta) for the SiLU forward with the 4-bit stash."""
+    return _fwd(lib().s2a_oracle_silu_fwd, x, row_len, dt, threads)
+
+
+def silu_bwd(g, codes, meta, row_len: int, dt: int, threads: int = 1):
+    return _bwd(lib().s2a_oracle_silu_bwd, g, codes, meta, row_len, dt, threads)
 
 
 def softmax_fwd(x, row_len: int, dt: int, threads: int = 1):

@@ -380,6 +380,52 @@ def test_gelu_tensor_range_reading(dt):
     assert np.all(np.abs(gin - wantg) <= tol * np.abs(wantg) + 1e-40)
 
 
+# ------------------------------------------------------------------ SiLU / Swish
+def test_silu_closed_forms_and_derivative():
+    assert o.silu(0.0) == 0.0 and o.silu_grad(0.0) == 0.5
+    h = 1e-5
+    for x in np.linspace(-9, 9, 721):
+        assert o.silu(x) == pytest.approx(x * sp.expit(x), rel=1e-14, abs=1e-300)
+        assert o.silu(x) - o.silu(-x) == pytest.approx(x, abs=1e-14)          # sigma(x) + sigma(-x) = 1
+        fd = (o.silu(x + h) - o.silu(x - h)) / (2 * h)
+        assert o.silu_grad(x) == pytest.approx(fd, abs=1e-8)
+        assert o.silu_grad(x) + o.silu_grad(-x) == pytest.approx(1.0, abs=1e-14)
+    fine = np.array([o.silu_grad(x) for x in np.linspace(-8, 8, 16001)])
+    assert -0.1 < fine.min() < -0.09 and 1.09 < fine.max() < 1.1              # the same band as GELU's
+    # SiLU is the sigmoid-GELU with its argument stretched by 1.702
+    for x in (-3.0, -0.7, 0.4, 2.5):
+        assert o.silu(A * x) == pytest.approx(A * o.gelu(x), rel=1e-13)
+        assert o.silu_grad(A * x) == pytest.approx(o.gelu_grad_exact(x), rel=1e-12)
+
+
+@pytest.mark.parametrize("dt", [F32, BF16])
+@pytest.mark.parametrize("rows,L", [(6, 64), (5, 197), (3, 1), (2, 3072)])
+def test_silu_tensor_path(dt, rows, L):
+    n = rows * L
+    clip = float(np.float32(2.0) * np.float32(1.702))
+    x = synth.to_io(synth.gelu_preact(15, ("silu", rows, L), n) * 2.2, dt)
+    gout = synth.to_io(synth.normal(15, ("silug", rows, L), n), dt)
+    y, codes, meta = o.silu_fwd(x, L, dt)
+    xw = o.widen(x, dt)
+    y_lib = xw * sp.expit(xw)
+    tol = 2.0 ** -24 if dt == F32 else 2.0 ** -8
+    assert np.all(np.abs(o.widen(y, dt) - y_lib) <= tol * np.abs(y_lib) + 1e-40)
+    q = o.unpack(codes, n).reshape(rows, L)
+    c = np.clip(xw, -clip, clip).reshape(rows, L)
+    for r in range(rows):
+        want, tie = _exact_codes(c[r].astype(np.float32))
+        ok = ~np.array(tie)
+        assert np.array_equal(q[r][ok], np.array(want)[ok])
+        assert meta[2 * r] == np.float32(c[r].min())
+    if L >= 64:
+        assert np.abs(xw).max() > clip and meta[0] == np.float32(-clip)       # the clip is exercised
+    gin = o.widen(o.silu_bwd(gout, codes, meta, L, dt), dt).reshape(rows, L)
+    xh = q.astype(np.float64) * meta[1::2, None].astype(np.float64) + meta[0::2, None].astype(np.float64)
+    sg = sp.expit(xh)
+    want = o.widen(gout, dt).reshape(rows, L) * (sg * (1 + xh * (1 - sg)))
+    assert np.all(np.abs(gin - want) <= tol * np.abs(want) + 1e-40)
+
+
 # ------------------------------------------------------------------ ReLU 1-bit stash
 @pytest.mark.parametrize("dt", [F32, BF16])
 @pytest.mark.parametrize("n", [1, 7, 8, 9, 1000, 4099])
