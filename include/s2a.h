@@ -103,6 +103,21 @@ int s2a_softmax_fwd(const void* x, void* y, uint8_t* codes, float* meta, size_t 
 int s2a_softmax_bwd(const void* grad_out, const uint8_t* codes, const float* meta, void* grad_in,
                     size_t n_elems, size_t row_len, int dt, void* cuda_stream);
 
+/* SiLU / Swish forward and backward with the same 4-bit input stash.  The paper names
+ * these functions (Section 3.2, end of "GeLU layer": the design "is also effective for
+ * similar non-parametric functions, such as SiLU and Swish") without giving constants, so
+ * the reading is this library's: y = x * sigmoid(x); the input is clipped into [-C, C] with
+ * C = 2 * 1.702 = 3.404 (binary32), which spans the same range of the sigmoid's argument as
+ * GELU's [-2, 2]; Eq. 8 / Eq. 9 per row as for GELU; the backward pass multiplies grad_out by
+ * the EXACT derivative sigmoid(x_hat) * (1 + x_hat * (1 - sigmoid(x_hat))), evaluated in
+ * binary64 for the 16 values a row can take.  Arguments and rules as for s2a_gelu_fwd /
+ * s2a_gelu_bwd.
+ */
+int s2a_silu_fwd(const void* x, void* y, uint8_t* codes, float* meta, size_t n_elems, size_t row_len, int dt,
+                 void* cuda_stream);
+int s2a_silu_bwd(const void* grad_out, const uint8_t* codes, const float* meta, void* grad_in, size_t n_elems,
+                 size_t row_len, int dt, void* cuda_stream);
+
 /* Bytes of scratch memory s2a_gelu_fwd_tensor_range needs for n_elems elements:
  * 8 + 8 * ceil(n_elems / 65536). */
 size_t s2a_tensor_range_scratch_bytes(size_t n_elems);
@@ -188,7 +203,7 @@ int s2a_device_error(unsigned int* flags, int clear);
 /* How a call would be run: writes into `out` (capacity `cap` bytes, always
  * NUL-terminated) a one-line description of the kernel variant and launch shape chosen
  * for (kernel, row_len, dt, n_elems).  kernel: 0 gelu_fwd, 1 gelu_bwd, 2 softmax_fwd,
- * 3 softmax_bwd.  Host-only; launches nothing.  Returns S2A_OK or an argument error.
+ * 3 softmax_bwd, 4 silu_fwd, 5 silu_bwd.  Host-only; launches nothing.  Returns S2A_OK or an argument error.
  */
 int s2a_describe_plan(int kernel, size_t n_elems, size_t row_len, int dt, char* out, size_t cap);
 

@@ -34,8 +34,8 @@ def _time_pair(kind: str, rows: int, L: int, dtype, seed: int, target_bytes: flo
     ys = [torch.empty_like(x) for x in xs]
     gins = [torch.empty_like(x) for x in xs]
     st = [binding.alloc_stash(n, L, "cuda") for _ in range(sets)]
-    fwd = binding.s2a_gelu_fwd if kind == "gelu" else binding.s2a_softmax_fwd
-    bwd = binding.s2a_gelu_bwd if kind == "gelu" else binding.s2a_softmax_bwd
+    fwd = {"gelu": binding.s2a_gelu_fwd, "silu": binding.s2a_silu_fwd, "softmax": binding.s2a_softmax_fwd}[kind]
+    bwd = {"gelu": binding.s2a_gelu_bwd, "silu": binding.s2a_silu_bwd, "softmax": binding.s2a_softmax_bwd}[kind]
     iters = max(4, min(200, int(2e10 // (n * item * 4))))
 
     def loop(fn):
@@ -116,6 +116,8 @@ def cases(quick: bool):
         rows = max(2, int(n) // 4096)
         for dtype in (torch.bfloat16, torch.float32):
             out.append(("gelu", rows, 4096, dtype))
+            if n == 1e8:
+                out.append(("silu", rows, 4096, dtype))
     for L in (64, 197, 257, 1024, 4096):
         for rows in ((10**4, 10**6) if quick else (10**4, 10**5, 10**6, 10**7)):
             if rows * L > 2e9 or (quick and rows * L > 3e8):
@@ -157,7 +159,7 @@ def main():
             torch.cuda.empty_cache()
         med = [statistics.median(r[k] for r in res) for k in range(3)]
         spread = max(r[2] for r in res) - min(r[2] for r in res)
-        kid = binding.GELU_FWD if kind == "gelu" else binding.SOFTMAX_FWD
+        kid = {"gelu": binding.GELU_FWD, "silu": binding.SILU_FWD, "softmax": binding.SOFTMAX_FWD}[kind]
         print(json.dumps({
             "kernel_pair": kind, "rows": rows, "row_len": L, "elems": rows * L,
             "io_dtype": "bf16" if dtype == torch.bfloat16 else "f32", "seeds": args.seeds,

@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libs2a.so")
 
 F32 = 0
 BF16 = 1
-GELU_FWD, GELU_BWD, SOFTMAX_FWD, SOFTMAX_BWD = 0, 1, 2, 3
+GELU_FWD, GELU_BWD, SOFTMAX_FWD, SOFTMAX_BWD, SILU_FWD, SILU_BWD = 0, 1, 2, 3, 4, 5
 
 EXPORTS = (
     "s2a_codes_bytes", "s2a_meta_bytes", "s2a_status_string", "s2a_gelu_fwd", "s2a_gelu_bwd",
@@ -25,6 +25,7 @@ EXPORTS = (
     "s2a_mask_bytes", "s2a_relu_fwd", "s2a_relu_bwd",
     "s2a_tensor_range_scratch_bytes", "s2a_gelu_fwd_tensor_range",
     "s2a_tensor_range_static_max_elems", "s2a_gelu_fwd_tensor_range_static",
+    "s2a_silu_fwd", "s2a_silu_bwd",
 )
 
 _lib = None
@@ -49,7 +50,8 @@ def lib() -> ctypes.CDLL:
         L.s2a_meta_bytes.restype = c.c_size_t
         L.s2a_status_string.argtypes = [c.c_int]
         L.s2a_status_string.restype = c.c_char_p
-        for name in ("s2a_gelu_fwd", "s2a_softmax_fwd", "s2a_gelu_bwd", "s2a_softmax_bwd"):
+        for name in ("s2a_gelu_fwd", "s2a_softmax_fwd", "s2a_gelu_bwd", "s2a_softmax_bwd", "s2a_silu_fwd",
+                     "s2a_silu_bwd"):
             f = getattr(L, name)
             f.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_size_t, c.c_size_t,
                           c.c_int, c.c_void_p]
@@ -154,6 +156,14 @@ def s2a_gelu_fwd(x, y, codes, meta, row_len: int) -> None:
 
 def s2a_gelu_bwd(grad_out, codes, meta, grad_in, row_len: int) -> None:
     _bwd(lib().s2a_gelu_bwd, grad_out, codes, meta, grad_in, row_len)
+
+
+def s2a_silu_fwd(x, y, codes, meta, row_len: int) -> None:
+    _fwd(lib().s2a_silu_fwd, x, y, codes, meta, row_len)
+
+
+def s2a_silu_bwd(grad_out, codes, meta, grad_in, row_len: int) -> None:
+    _bwd(lib().s2a_silu_bwd, grad_out, codes, meta, grad_in, row_len)
 
 
 def s2a_softmax_fwd(x, y, codes, meta, row_len: int) -> None:

@@ -93,6 +93,17 @@ int s2a_softmax_bwd(const void* grad_out, const uint8_t* codes, const float* met
              const_cast<float*>(meta), n_elems, row_len, dt, cuda_stream);
 }
 
+int s2a_silu_fwd(const void* x, void* y, uint8_t* codes, float* meta, size_t n_elems, size_t row_len, int dt,
+                 void* cuda_stream) {
+  return run(kSiluFwd, x, y, codes, meta, n_elems, row_len, dt, cuda_stream);
+}
+
+int s2a_silu_bwd(const void* grad_out, const uint8_t* codes, const float* meta, void* grad_in, size_t n_elems,
+                 size_t row_len, int dt, void* cuda_stream) {
+  return run(kSiluBwd, grad_out, grad_in, const_cast<uint8_t*>(codes), const_cast<float*>(meta), n_elems, row_len,
+             dt, cuda_stream);
+}
+
 size_t s2a_tensor_range_scratch_bytes(size_t n_elems) { return (size_t)tensor_range_scratch_bytes(n_elems); }
 
 int s2a_gelu_fwd_tensor_range(const void* x, void* y, uint8_t* codes, float* meta, void* scratch,
@@ -146,7 +157,7 @@ int s2a_device_error(unsigned int* flags, int clear) {
 int s2a_describe_plan(int kernel, size_t n_elems, size_t row_len, int dt, char* out, size_t cap) {
   if (!out || cap == 0) return S2A_ERR_NULL;
   out[0] = 0;
-  if (kernel < 0 || kernel > 3) return S2A_ERR_SHAPE;
+  if (kernel < 0 || kernel > 5) return S2A_ERR_SHAPE;
   if (dt != S2A_F32 && dt != S2A_BF16) return S2A_ERR_DTYPE;
   if (row_len == 0 || row_len > 0x7fffffffull || n_elems % row_len != 0) return S2A_ERR_SHAPE;
   const uint64_t n_rows = n_elems / row_len;

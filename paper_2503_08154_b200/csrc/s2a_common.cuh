@@ -72,22 +72,49 @@ __device__ __forceinline__ float dequant(uint32_t code, float mn, float s) {
 }
 
 // ---------------------------------------------------------------- Eq. 10 and Eq. 12
-// y = x * sigmoid(1.702 x), evaluated through t = exp(-|1.702 x|) so that neither tail
+// The two input-stash activations.  GELU is the paper's x * sigmoid(1.702 x) with the
+// sine-fitted derivative of Eq. 12 and the clip [-2, 2].  SiLU (x * sigmoid(x)) is named by
+// the paper without constants: it is given the clip 2 * 1.702 (the same range of the
+// sigmoid's argument) and its exact derivative.
+enum { kActGelu = 0, kActSilu = 1 };
+template <int ACT> struct Act;
+template <> struct Act<kActGelu> {
+  static constexpr float kSlopeOf = kSlope;
+  static constexpr float kClipOf = kClip;
+};
+template <> struct Act<kActSilu> {
+  static constexpr float kSlopeOf = 1.0f;
+  static constexpr float kClipOf = 2.0f * 1.702f;
+};
+
+// y = x * sigmoid(a x), evaluated through t = exp(-|a x|) so that neither tail
 // overflows: sigmoid(z) = 1 / (1 + t) for z >= 0 and t / (1 + t) for z < 0.  The
-// product 1.702 x is carried as hi + lo so that its rounding does not scale the error
+// product a x is carried as hi + lo so that its rounding does not scale the error
 // of exp with |x|.
-__device__ __forceinline__ float gelu_value(float x) {
-  float z = __fmul_rn(kSlope, x);
-  float zlo = __fmaf_rn(kSlope, x, -z);
+template <int ACT>
+__device__ __forceinline__ float act_value(float x) {
+  constexpr float a = Act<ACT>::kSlopeOf;
+  float z = __fmul_rn(a, x);
+  float zlo = __fmaf_rn(a, x, -z);
   float t = expf(-fabsf(z)) * (1.0f - (z >= 0.0f ? zlo : -zlo));
   return __fdiv_rn(z >= 0.0f ? x : x * t, 1.0f + t);
 }
+__device__ __forceinline__ float gelu_value(float x) { return act_value<kActGelu>(x); }
 
-// Eq. 12 at a dequantised x_hat = code * s + min, in binary64.
-__device__ __forceinline__ double gelu_sine_derivative(uint32_t code, float mn, float s) {
+// The derivative used by the backward pass at a dequantised x_hat = code * s + min, in
+// binary64: Eq. 12 for GELU, the exact derivative for SiLU.
+template <int ACT>
+__device__ __forceinline__ double act_derivative(uint32_t code, float mn, float s) {
   double xh = (double)code * (double)s + (double)mn;
-  double sig = 1.0 / (1.0 + exp(-(double)kSlope * xh));
-  return sig + (double)kSineAmp * sin((double)kSineFreq * xh);
+  if (ACT == kActGelu) {
+    double sig = 1.0 / (1.0 + exp(-(double)kSlope * xh));
+    return sig + (double)kSineAmp * sin((double)kSineFreq * xh);
+  }
+  double sig = 1.0 / (1.0 + exp(-xh));
+  return sig * (1.0 + xh * (1.0 - sig));
+}
+__device__ __forceinline__ double gelu_sine_derivative(uint32_t code, float mn, float s) {
+  return act_derivative<kActGelu>(code, mn, s);
 }
 
 // ---------------------------------------------------------------- warp reductions

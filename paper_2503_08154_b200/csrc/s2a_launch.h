@@ -6,7 +6,13 @@
 
 namespace s2a {
 
-enum { kGeluFwd = 0, kGeluBwd = 1, kSoftmaxFwd = 2, kSoftmaxBwd = 3 };
+enum { kGeluFwd = 0, kGeluBwd = 1, kSoftmaxFwd = 2, kSoftmaxBwd = 3, kSiluFwd = 4, kSiluBwd = 5 };
+
+// Kernel-id predicates (GELU and SiLU share their code: "act" kernels).
+__host__ __device__ constexpr bool is_act_fwd(int k) { return k == kGeluFwd || k == kSiluFwd; }
+__host__ __device__ constexpr bool is_act_bwd(int k) { return k == kGeluBwd || k == kSiluBwd; }
+__host__ __device__ constexpr bool is_fwd(int k) { return is_act_fwd(k) || k == kSoftmaxFwd; }
+__host__ __device__ constexpr int act_of(int k) { return (k == kSiluFwd || k == kSiluBwd) ? 1 : 0; }
 
 // One launch of a row-at-a-time kernel over rows [row0, row0 + n_rows) of a tensor.
 // row0 * row_len must be even (whole code bytes).  `in` is x or grad_out, `out` is y or

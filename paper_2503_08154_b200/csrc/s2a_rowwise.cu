@@ -48,6 +48,8 @@ __device__ __forceinline__ uint32_t nibble_at(const uint8_t* codes, uint64_t e) 
 template <int KERNEL, int DT>
 __global__ void __launch_bounds__(kThreads) rowwise_kernel(RowwiseArgs a) {
   using T = typename Io<DT>::T;
+  constexpr int ACT = act_of(KERNEL);
+  constexpr float kActClip = Act<ACT>::kClipOf;
   __shared__ BlockScratch sc;
   __shared__ float row_mn[2], row_inv[2], row_s[2], row_aux[2];
   __shared__ float dtab[2][16];
@@ -69,7 +71,7 @@ __global__ void __launch_bounds__(kThreads) rowwise_kernel(RowwiseArgs a) {
     // ---- per-row statistics ---------------------------------------------------
     for (uint32_t h = 0; h < rows_here; ++h) {
       const uint64_t base = e0 + (uint64_t)h * L;
-      if (KERNEL == kGeluFwd) {
+      if (is_act_fwd(KERNEL)) {
         float mn = INFINITY, mx = -INFINITY;
         for (uint32_t i = tid; i < L; i += kThreads) {
           float x = Io<DT>::widen(in[base + i]);
@@ -79,7 +81,7 @@ __global__ void __launch_bounds__(kThreads) rowwise_kernel(RowwiseArgs a) {
         mn = block_reduce<1>(mn, sc, 0);
         mx = block_reduce<0>(mx, sc, 1);
         // min/max of the clipped row = clipped min/max of the row (the clip is monotone)
-        QRange q = make_qrange(fminf(fmaxf(mn, -kClip), kClip), fminf(fmaxf(mx, -kClip), kClip));
+        QRange q = make_qrange(fminf(fmaxf(mn, -kActClip), kActClip), fminf(fmaxf(mx, -kActClip), kActClip));
         if (tid == 0) { row_mn[h] = q.mn; row_inv[h] = q.inv; row_s[h] = q.s; }
       } else if (KERNEL == kSoftmaxFwd) {
         float m = -INFINITY;
@@ -102,9 +104,9 @@ __global__ void __launch_bounds__(kThreads) rowwise_kernel(RowwiseArgs a) {
         mx = block_reduce<0>(mx, sc, 1);
         QRange q = make_qrange(mn, mx);
         if (tid == 0) { row_mn[h] = q.mn; row_inv[h] = q.inv; row_s[h] = q.s; }
-      } else if (KERNEL == kGeluBwd) {
+      } else if (is_act_bwd(KERNEL)) {
         const float mn = a.meta[2 * (r0 + h)], s = a.meta[2 * (r0 + h) + 1];
-        if (tid < 16) dtab[h][tid] = (float)gelu_sine_derivative((uint32_t)tid, mn, s);
+        if (tid < 16) dtab[h][tid] = (float)act_derivative<ACT>((uint32_t)tid, mn, s);
       } else {  // kSoftmaxBwd
         const float mn = a.meta[2 * (r0 + h)], s = a.meta[2 * (r0 + h) + 1];
         float dot = 0.0f;
@@ -118,7 +120,7 @@ __global__ void __launch_bounds__(kThreads) rowwise_kernel(RowwiseArgs a) {
     }
     __syncthreads();  // statistics in shared memory, and forward outputs, now visible
 
-    if ((KERNEL == kGeluFwd || KERNEL == kSoftmaxFwd) && tid < (int)rows_here) {
+    if (is_fwd(KERNEL) && tid < (int)rows_here) {
       a.meta[2 * (r0 + tid)] = row_mn[tid];
       a.meta[2 * (r0 + tid) + 1] = row_s[tid];
     }
@@ -127,22 +129,22 @@ __global__ void __launch_bounds__(kThreads) rowwise_kernel(RowwiseArgs a) {
     const uint64_t n_bytes = (cnt + 1) >> 1;
     for (uint64_t b = tid; b < n_bytes; b += kThreads) {
       uint32_t byte = 0;
-      if (KERNEL == kGeluBwd || KERNEL == kSoftmaxBwd) byte = a.codes[(e0 >> 1) + b];
+      if (!is_fwd(KERNEL)) byte = a.codes[(e0 >> 1) + b];
 #pragma unroll
       for (int k = 0; k < 2; ++k) {
         const uint64_t rel = 2 * b + k;
         if (rel < cnt) {
           const uint32_t h = rel >= L ? 1u : 0u;
           const uint64_t e = e0 + rel;
-          if (KERNEL == kGeluFwd) {
+          if (is_act_fwd(KERNEL)) {
             float x = Io<DT>::widen(in[e]);
             QRange q{row_mn[h], row_inv[h], row_s[h]};
-            byte |= quant_code(fminf(fmaxf(x, -kClip), kClip), q) << (4 * k);
-            out[e] = Io<DT>::narrow(gelu_value(x));
+            byte |= quant_code(fminf(fmaxf(x, -kActClip), kActClip), q) << (4 * k);
+            out[e] = Io<DT>::narrow(act_value<ACT>(x));
           } else if (KERNEL == kSoftmaxFwd) {
             QRange q{row_mn[h], row_inv[h], row_s[h]};
             byte |= quant_code(Io<DT>::widen(out[e]), q) << (4 * k);
-          } else if (KERNEL == kGeluBwd) {
+          } else if (is_act_bwd(KERNEL)) {
             uint32_t code = (byte >> (4 * k)) & 0xFu;
             out[e] = Io<DT>::narrow(Io<DT>::widen(in[e]) * dtab[h][code]);
           } else {
@@ -152,7 +154,7 @@ __global__ void __launch_bounds__(kThreads) rowwise_kernel(RowwiseArgs a) {
           }
         }
       }
-      if (KERNEL == kGeluFwd || KERNEL == kSoftmaxFwd) a.codes[(e0 >> 1) + b] = (uint8_t)byte;
+      if (is_fwd(KERNEL)) a.codes[(e0 >> 1) + b] = (uint8_t)byte;
     }
     __syncthreads();  // shared statistics are reused by the next group
   }
@@ -179,6 +181,8 @@ cudaError_t launch_rowwise(int kernel, int dt, const RowwiseArgs& a, cudaStream_
     S2A_CASE(kGeluBwd)
     S2A_CASE(kSoftmaxFwd)
     S2A_CASE(kSoftmaxBwd)
+    S2A_CASE(kSiluFwd)
+    S2A_CASE(kSiluBwd)
   }
 #undef S2A_CASE
   return cudaErrorInvalidValue;

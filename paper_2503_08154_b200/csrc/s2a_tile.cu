@@ -12,6 +12,8 @@ cudaError_t launch_tile_gelu_fwd(int dt, const TilePlan& p, const void* kernel_a
 cudaError_t launch_tile_gelu_bwd(int dt, const TilePlan& p, const void* kernel_args, cudaStream_t st);
 cudaError_t launch_tile_softmax_fwd(int dt, const TilePlan& p, const void* kernel_args, cudaStream_t st);
 cudaError_t launch_tile_softmax_bwd(int dt, const TilePlan& p, const void* kernel_args, cudaStream_t st);
+cudaError_t launch_tile_silu_fwd(int dt, const TilePlan& p, const void* kernel_args, cudaStream_t st);
+cudaError_t launch_tile_silu_bwd(int dt, const TilePlan& p, const void* kernel_args, cudaStream_t st);
 
 namespace {
 
@@ -67,7 +69,8 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L) {
   if (path && path[0] == 'r') return p;
   const char* var = getenv("S2A_VARIANT");
   const bool force_generic = var && var[0] == 'g';
-  const bool is_gelu = kernel == kGeluFwd || kernel == kGeluBwd;
+  const bool is_gelu = is_act_fwd(kernel) || is_act_bwd(kernel);  // GELU and SiLU share their kernels
+  const bool is_silu = act_of(kernel) == 1;
   const uint32_t esize = dt == kF32 ? 4u : 2u;
   const uint32_t vec = 16u / esize;  // elements per 16-byte access
   const bool vec16 = (L % vec) == 0;
@@ -111,6 +114,7 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L) {
     unit = 8;
     iters = (n_acc + 7) / 8;
   }
+  if (variant == kVariantGeneric && is_silu) return p;  // SiLU has the streamed form only
   if (variant == kVariantGeneric) {
     // general register-resident form: pair accesses with 8 or 32 lanes per row, or 16-byte
     // accesses with 128 lanes per row (long softmax rows)
@@ -223,6 +227,8 @@ cudaError_t launch_tile(int kernel, int dt, const TilePlan& p, const TileArgs& a
     case kGeluBwd: return launch_tile_gelu_bwd(dt, p, &ka, st);
     case kSoftmaxFwd: return launch_tile_softmax_fwd(dt, p, &ka, st);
     case kSoftmaxBwd: return launch_tile_softmax_bwd(dt, p, &ka, st);
+    case kSiluFwd: return launch_tile_silu_fwd(dt, p, &ka, st);
+    case kSiluBwd: return launch_tile_silu_bwd(dt, p, &ka, st);
   }
   return cudaErrorInvalidValue;
 }

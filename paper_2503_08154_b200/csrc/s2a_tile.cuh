@@ -342,12 +342,12 @@ __device__ __forceinline__ float rcp_approx(float x) {
   return y;
 }
 
-template <int DT>
+template <int DT, int ACT = kActGelu>
 __device__ __forceinline__ float gelu_eval(float x) {
-  if (DT == kF32) return gelu_value(x);
+  if (DT == kF32) return act_value<ACT>(x);
   // y = x / (1 + 2^(-1.702 log2(e) x)).  For x < -52 the power overflows and y becomes
   // -0 instead of a value below 2^-120: the bfloat16 path flushes such results.
-  constexpr float c = -1.702f * 1.4426950408889634f;
+  constexpr float c = -Act<ACT>::kSlopeOf * 1.4426950408889634f;
   return x * rcp_approx(1.0f + ex2_approx(c * x));
 }
 
@@ -690,10 +690,11 @@ struct CodePacker {
 
 // NVL > 0 fixes the number of vectors per lane (row_len == NVL * UNIT * EPA), which lets
 // the compiler drop every loop counter and bound check; NVL == 0 is the general loop.
-template <int DT, int UNIT_, int NVL>
-struct StreamGeluFwd {
+template <int DT, int UNIT_, int NVL, int ACT>
+struct StreamActFwd {
   static constexpr int kMaxRegs = 64;
-  static constexpr int kKernel = kGeluFwd;
+  static constexpr int kKernel = ACT == kActGelu ? kGeluFwd : kSiluFwd;
+  static constexpr float kActClip = Act<ACT>::kClipOf;
   static constexpr int UNIT = UNIT_;
   using V = V16<DT>;
   struct State {};
@@ -707,8 +708,8 @@ struct StreamGeluFwd {
     pk.init();
 #pragma unroll
     for (int k = 0; k < V::EPA; ++k) {
-      pk.add(k, fminf(fmaxf(v[k], -kClip), kClip), q);
-      v[k] = gelu_eval<DT>(v[k]);
+      pk.add(k, fminf(fmaxf(v[k], -kActClip), kActClip), q);
+      v[k] = gelu_eval<DT, ACT>(v[k]);
     }
     *(typename V::Raw*)(row + j * 16u) = V::narrow(v);
     V::store_codes(crow, j, pk.acc);
@@ -732,7 +733,7 @@ struct StreamGeluFwd {
     const float mn = u.template reduce<kOpMin>(mm.lo());
     const float mx = u.template reduce<kOpMax>(mm.hi());
     // min / max of the clipped row = clipped min / max of the row (the clip is monotone)
-    const QRange q = make_qrange(fminf(fmaxf(mn, -kClip), kClip), fminf(fmaxf(mx, -kClip), kClip));
+    const QRange q = make_qrange(fminf(fmaxf(mn, -kActClip), kActClip), fminf(fmaxf(mx, -kActClip), kActClip));
     if (active && u.ul == 0) { p.meta[2 * r] = q.mn; p.meta[2 * r + 1] = q.s; }
     if (NVL > 0) {
 #pragma unroll
@@ -744,13 +745,16 @@ struct StreamGeluFwd {
   }
 };
 
+template <int DT, int UNIT_, int NVL> using StreamGeluFwd = StreamActFwd<DT, UNIT_, NVL, kActGelu>;
+template <int DT, int UNIT_, int NVL> using StreamSiluFwd = StreamActFwd<DT, UNIT_, NVL, kActSilu>;
+
 // GELU backward.  With a whole warp on one row the 16 derivative values live one per
 // lane (twice over) and are fetched with a shuffle indexed by the code; smaller units
 // read them from a shared-memory table.
-template <int DT, int UNIT_, int NVL>
-struct StreamGeluBwd {
+template <int DT, int UNIT_, int NVL, int ACT>
+struct StreamActBwd {
   static constexpr int kMaxRegs = 64;
-  static constexpr int kKernel = kGeluBwd;
+  static constexpr int kKernel = ACT == kActGelu ? kGeluBwd : kSiluBwd;
   static constexpr int UNIT = UNIT_;
   using V = V16<DT>;
   struct State {
@@ -770,12 +774,12 @@ struct StreamGeluBwd {
     // The 16 values of Eq. 12 this row can take, in binary64; kept while (min, s) repeat.
     if (mn != st.tab_mn || s != st.tab_s) {
       if (UNIT_ >= 32) {
-        st.d = (float)gelu_sine_derivative((uint32_t)(u.ul & 15), mn, s);
+        st.d = (float)act_derivative<ACT>((uint32_t)(u.ul & 15), mn, s);
       } else {
 #pragma unroll
         for (int c = 0; c < 16; c += (UNIT_ < 16 ? UNIT_ : 16)) {
           const int code = c + u.ul;
-          if (u.ul < 16 && code < 16) tab[code] = (float)gelu_sine_derivative((uint32_t)code, mn, s);
+          if (u.ul < 16 && code < 16) tab[code] = (float)act_derivative<ACT>((uint32_t)code, mn, s);
         }
       }
       st.tab_mn = mn;
@@ -818,6 +822,9 @@ struct StreamGeluBwd {
     if (ok) *(typename V::Raw*)(row + j * 16u) = V::narrow(v);
   }
 };
+
+template <int DT, int UNIT_, int NVL> using StreamGeluBwd = StreamActBwd<DT, UNIT_, NVL, kActGelu>;
+template <int DT, int UNIT_, int NVL> using StreamSiluBwd = StreamActBwd<DT, UNIT_, NVL, kActSilu>;
 
 // Softmax forward on 16-byte vectors, NV vectors per lane kept in registers.
 template <int DT, int UNIT_, int NV>
@@ -1262,7 +1269,7 @@ __global__ void __maxnreg__(WORK::kMaxRegs) tile_kernel(TileKernelArgs a) {
   extern __shared__ __align__(1024) unsigned char smem[];
   constexpr int KERNEL = WORK::kKernel;
   constexpr int UNIT = WORK::UNIT;
-  constexpr bool kFwd = (KERNEL == kGeluFwd || KERNEL == kSoftmaxFwd);
+  constexpr bool kFwd = is_fwd(KERNEL);
 
   uint64_t* full = (uint64_t*)smem;                 // [stages]
   uint64_t* done = (uint64_t*)smem + kMaxStages;    // [stages]
@@ -1510,7 +1517,10 @@ cudaError_t launch_variant(const TilePlan& p, const TileKernelArgs& ka, cudaStre
     if constexpr (KERNEL == kGeluBwd) return launch_gelu_stream<StreamGeluBwd, DT>(p, ka, st);
     if constexpr (KERNEL == kSoftmaxFwd) return launch_softmax_stream<StreamSoftmaxFwd, DT>(p, ka, st);
     if constexpr (KERNEL == kSoftmaxBwd) return launch_softmax_stream<StreamSoftmaxBwd, DT>(p, ka, st);
+    if constexpr (KERNEL == kSiluFwd) return launch_gelu_stream<StreamSiluFwd, DT>(p, ka, st);
+    if constexpr (KERNEL == kSiluBwd) return launch_gelu_stream<StreamSiluBwd, DT>(p, ka, st);
   }
+  if constexpr (KERNEL == kSiluFwd || KERNEL == kSiluBwd) return cudaErrorInvalidValue;  // streamed form only
   if (p.variant == kVariantPairFixed) {
     if constexpr (KERNEL == kSoftmaxFwd) return launch_pair_fixed<PairSoftmaxFwd, DT>(p, ka, st);
     if constexpr (KERNEL == kSoftmaxBwd) return launch_pair_fixed<PairSoftmaxBwd, DT>(p, ka, st);

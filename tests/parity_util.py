@@ -78,7 +78,7 @@ def gpu_fwd(kind: str, x: np.ndarray, L: int, dt: int, inplace: bool = False):
         xin = yg.view(torch_dtype(dt))
     else:
         xin = xd
-    fn = binding.s2a_gelu_fwd if kind == "gelu" else binding.s2a_softmax_fwd
+    fn = {"gelu": binding.s2a_gelu_fwd, "softmax": binding.s2a_softmax_fwd, "silu": binding.s2a_silu_fwd}[kind]
     fn(xin, yg.view(torch_dtype(dt)), cg.view(torch.uint8), mg.view(torch.float32), L)
     torch.cuda.synchronize()
     assert binding.s2a_device_error() == 0
@@ -102,7 +102,7 @@ def gpu_bwd(kind: str, g: np.ndarray, codes: np.ndarray, meta: np.ndarray, L: in
         gin = og.view(torch_dtype(dt))
     else:
         gin = gd
-    fn = binding.s2a_gelu_bwd if kind == "gelu" else binding.s2a_softmax_bwd
+    fn = {"gelu": binding.s2a_gelu_bwd, "softmax": binding.s2a_softmax_bwd, "silu": binding.s2a_silu_bwd}[kind]
     fn(gin, cd, md, og.view(torch_dtype(dt)), L)
     torch.cuda.synchronize()
     assert binding.s2a_device_error() == 0

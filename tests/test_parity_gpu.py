@@ -248,6 +248,27 @@ def test_tensor_beyond_2_to_31_elements_uses_64_bit_indexing():
     pu.assert_close(pu.widen(pu.to_host(gv[repeats - 1], BF16), BF16), pu.widen(gin_o, BF16), BF16, "gelu grad_in (large)")
 
 
+# ------------------------------------------------------------------ SiLU with the 4-bit stash
+@pytest.mark.parametrize("dt", [F32, BF16])
+@pytest.mark.parametrize("rows,L", [(5, 1), (7, 3), (33, 65), (451, 197), (1001, 64), (137, 1024), (41, 3072),
+                                    (11, 4096), (9, 5120), (3, 8191), (2, 40000)])
+def test_silu(rows, L, dt):
+    n = rows * L
+    x = synth.to_io(synth.gelu_preact(9, ("silu", rows, L, dt), n) * np.float32(2.2), dt)
+    g = synth.to_io(synth.normal(9, ("silug", rows, L, dt), n), dt)
+    for inplace in (False, True):
+        y_o, codes_o, meta_o = o.silu_fwd(x, L, dt, threads=THREADS)
+        y_g, codes_g, meta_g = pu.gpu_fwd("silu", x, L, dt, inplace=inplace)
+        assert np.array_equal(codes_g, codes_o), "SiLU codes differ from the oracle's"
+        assert np.array_equal(meta_g.view(np.uint32), meta_o.view(np.uint32))
+        pu.assert_close(pu.widen(y_g, dt), pu.widen(y_o, dt), dt, "silu y")
+        gin_o = o.silu_bwd(g, codes_o, meta_o, L, dt, threads=THREADS)
+        gin_g = pu.gpu_bwd("silu", g, codes_o, meta_o, L, dt, inplace=inplace)
+        pu.assert_close(pu.widen(gin_g, dt), pu.widen(gin_o, dt), dt, "silu grad_in")
+    plan = binding.s2a_describe_plan(binding.SILU_FWD, n, L, dt)
+    assert plan.startswith("tile") == (L % (4 if dt == F32 else 8) == 0 and rows >= 2 and L <= 8192), plan
+
+
 # ------------------------------------------------------------------ per-tensor range variant
 @pytest.mark.parametrize("dt", [F32, BF16])
 @pytest.mark.parametrize("rows,L,scale", [(3, 5, 0.3), (1, 1, 1.0), (7, 197, 0.2), (300, 66, 0.4), (64, 3072, 0.25),
