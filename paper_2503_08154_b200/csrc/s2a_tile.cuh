@@ -1003,7 +1003,7 @@ struct PairGeom {
 
 template <int DT, int UNIT_, int LCT>
 struct PairSoftmaxFwd {
-  static constexpr int kMaxRegs = 104;
+  static constexpr int kMaxRegs = 96;  // 4 CTAs of 160 threads per SM
   static constexpr int kKernel = kSoftmaxFwd;
   static constexpr int UNIT = UNIT_;
   using P = P2<DT>;
@@ -1096,7 +1096,7 @@ struct PairSoftmaxFwd {
 // and the exponent's argument is one fused multiply-add.
 template <int UNIT_, int LCT>
 struct PairSoftmaxFwd<kBF16, UNIT_, LCT> {
-  static constexpr int kMaxRegs = 104;
+  static constexpr int kMaxRegs = 96;  // 4 CTAs of 160 threads per SM
   static constexpr int kKernel = kSoftmaxFwd;
   static constexpr int UNIT = UNIT_;
   using G = PairGeom<UNIT_, LCT>;
@@ -1115,96 +1115,133 @@ struct PairSoftmaxFwd<kBF16, UNIT_, LCT> {
   static __device__ __forceinline__ float lo(uint32_t w) { return __uint_as_float(w << 16); }
   static __device__ __forceinline__ float hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
-  // An inactive unit (no row pair left in this round) runs on row 0 and stores nothing, so
-  // that every lane takes part in the shuffles without per-element guards.
+  // The two rows of a pair are worked on TOGETHER, phase by phase, so that each row's
+  // shuffle and special-function latencies hide behind the other row's arithmetic.  HP = 0
+  // is the row that starts on an even element (the high half of its last word is the next
+  // row's), HP = 1 the one that starts on an odd element (the low half of its first word is
+  // the previous row's).  An inactive unit (no pair left in this round) runs on rows 0 and 1
+  // and stores nothing, so that every lane takes part in the shuffles.
+  struct Regs {
+    uint32_t w[G::ITERS];      // input words, later y as written
+    float e[G::ITERS][2];
+  };
   template <int HP>
-  static __device__ __forceinline__ void row(Unit<UNIT_>& u, const StagePtrs& p, uint32_t r, bool active) {
+  static __device__ __forceinline__ bool drop_lo(int i, int ul) { return HP == 1 && i == 0 && ul == 0; }
+  template <int HP>
+  static __device__ __forceinline__ bool drop_hi(int i, int ul) { return HP == 0 && i == G::LAST_I && ul == G::LAST_UL; }
+
+  template <int HP>
+  static __device__ __forceinline__ float load_max(Regs& R, const uint32_t* words, int ul) {
     constexpr uint32_t kNegInf2 = 0xFF80FF80u;
-    const uint32_t a0 = (r * (uint32_t)LCT) >> 1;
-    const int ul = u.ul;
-    const uint32_t* words = (const uint32_t*)p.data + a0 + ul;
-    uint32_t raw[G::ITERS];
     uint32_t mx2 = kNegInf2;
 #pragma unroll
     for (int i = 0; i < G::ITERS; ++i) {
       uint32_t w = kNegInf2;
       if (G::has(i, ul)) w = words[UNIT_ * i];
-      if (HP == 1 && i == 0 && ul == 0) w = (w & 0xffff0000u) | 0xFF80u;                     // foreign low half
-      if (HP == 0 && i == G::LAST_I && ul == G::LAST_UL) w = (w & 0x0000ffffu) | 0xFF800000u;  // foreign high half
-      raw[i] = w;
+      if (drop_lo<HP>(i, ul)) w = (w & 0xffff0000u) | 0xFF80u;      // foreign low half
+      if (drop_hi<HP>(i, ul)) w = (w & 0x0000ffffu) | 0xFF800000u;  // foreign high half
+      R.w[i] = w;
       mx2 = max2(mx2, w);
     }
-    const float m = u.template reduce<kOpMax>(fmaxf(lo(mx2), hi(mx2)));
+    return fmaxf(lo(mx2), hi(mx2));
+  }
+
+  static __device__ __forceinline__ float exp_sum(Regs& R, float m) {
     constexpr float kLog2e = 1.4426950408889634f;
     const float nm = -m * kLog2e;
-    float e[G::ITERS][2];
     float z = 0.0f;
 #pragma unroll
     for (int i = 0; i < G::ITERS; ++i) {
-      e[i][0] = ex2_approx(fmaf(lo(raw[i]), kLog2e, nm));  // foreign / absent: 2^-inf = 0
-      e[i][1] = ex2_approx(fmaf(hi(raw[i]), kLog2e, nm));
-      z += e[i][0];
-      z += e[i][1];
+      R.e[i][0] = ex2_approx(fmaf(lo(R.w[i]), kLog2e, nm));  // foreign / absent: 2^-inf = 0
+      R.e[i][1] = ex2_approx(fmaf(hi(R.w[i]), kLog2e, nm));
+      z += R.e[i][0];
+      z += R.e[i][1];
     }
-    z = u.template reduce<kOpSum>(z);
-    const float rz = __fdiv_rn(1.0f, z);
-    uint32_t mn2 = 0x7F807F80u;
-    mx2 = kNegInf2;
-    uint32_t* out = (uint32_t*)p.data + a0 + ul;
+    return z;
+  }
+
+  template <int HP>
+  static __device__ __forceinline__ void scale_store(Regs& R, float rz, uint32_t* out, int ul, bool active,
+                                                     float& mn, float& mx) {
+    uint32_t mn2 = 0x7F807F80u, mx2 = 0xFF80FF80u;
 #pragma unroll
     for (int i = 0; i < G::ITERS; ++i) {
-      __nv_bfloat162 b = __floats2bfloat162_rn(e[i][0] * rz, e[i][1] * rz);
+      __nv_bfloat162 b = __floats2bfloat162_rn(R.e[i][0] * rz, R.e[i][1] * rz);
       const uint32_t w = *(uint32_t*)&b;  // y as written
-      raw[i] = w;
-      const bool drop_lo = HP == 1 && i == 0 && ul == 0;
-      const bool drop_hi = HP == 0 && i == G::LAST_I && ul == G::LAST_UL;
+      R.w[i] = w;
       if (G::has(i, ul)) {
         uint32_t wm = w;  // for min/max a foreign half is replaced by its neighbour
-        if (drop_lo) wm = (w & 0xffff0000u) | (w >> 16);
-        if (drop_hi) wm = (w & 0x0000ffffu) | (w << 16);
+        if (drop_lo<HP>(i, ul)) wm = (w & 0xffff0000u) | (w >> 16);
+        if (drop_hi<HP>(i, ul)) wm = (w & 0x0000ffffu) | (w << 16);
         mn2 = min2(mn2, wm);
         mx2 = max2(mx2, wm);
         if (active) {
-          if (drop_lo) *((uint16_t*)(out + UNIT_ * i) + 1) = (uint16_t)(w >> 16);
-          else if (drop_hi) *(uint16_t*)(out + UNIT_ * i) = (uint16_t)w;
+          if (drop_lo<HP>(i, ul)) *((uint16_t*)(out + UNIT_ * i) + 1) = (uint16_t)(w >> 16);
+          else if (drop_hi<HP>(i, ul)) *(uint16_t*)(out + UNIT_ * i) = (uint16_t)w;
           else out[UNIT_ * i] = w;
         }
       }
     }
-    float mn = fminf(lo(mn2), hi(mn2)), mx = fmaxf(lo(mx2), hi(mx2));
-    reduce_minmax_bf16<UNIT_>(mn, mx);
-    const QRange q = make_qrange(mn, mx);
-    if (active && ul == 0) { p.meta[2 * r] = q.mn; p.meta[2 * r + 1] = q.s; }
-    unsigned char* cb = p.codes + a0 + ul;
-#pragma unroll
-    for (int i = 0; i < G::ITERS; ++i) {
-      if (active && G::has(i, ul)) {
-        const bool drop_lo = HP == 1 && i == 0 && ul == 0;
-        const bool drop_hi = HP == 0 && i == G::LAST_I && ul == G::LAST_UL;
-        CodePacker<2> pk;
-        pk.init();
-        pk.add(0, drop_lo ? q.mn : lo(raw[i]), q);
-        pk.add(1, drop_hi ? q.mn : hi(raw[i]), q);  // a dropped element codes as 0
-        uint32_t byte = pk.acc & 0xFFu;
-        if (drop_lo) byte |= cb[UNIT_ * i] & 0x0Fu;  // low nibble: the previous row's
-        cb[UNIT_ * i] = (unsigned char)byte;
-      }
-    }
+    mn = fminf(lo(mn2), hi(mn2));
+    mx = fmaxf(lo(mx2), hi(mx2));
+  }
+
+  // Code byte of word i of a row (a foreign half codes as 0).
+  template <int HP>
+  static __device__ __forceinline__ uint32_t code_byte(const Regs& R, int i, int ul, const QRange& q) {
+    CodePacker<2> pk;
+    pk.init();
+    pk.add(0, drop_lo<HP>(i, ul) ? q.mn : lo(R.w[i]), q);
+    pk.add(1, drop_hi<HP>(i, ul) ? q.mn : hi(R.w[i]), q);
+    return pk.acc & 0xFFu;
   }
 
   static __device__ __forceinline__ void group(Unit<UNIT_>& u, State&, const StagePtrs& p, float*, uint32_t grp,
                                                bool active, uint32_t) {
     const uint32_t r = active ? 2 * grp : 0;
-    row<0>(u, p, r, active);
-    u.sync();  // the odd row reads the shared word and code byte the even row left
-    row<1>(u, p, r + 1, active);
-    u.sync();
+    const int ul = u.ul;
+    const uint32_t a0 = (r * (uint32_t)LCT) >> 1, a1 = ((r + 1) * (uint32_t)LCT) >> 1;  // a1 = a0 + NACC - 1
+    Regs A, B;
+    float mA = load_max<0>(A, (const uint32_t*)p.data + a0 + ul, ul);
+    float mB = load_max<1>(B, (const uint32_t*)p.data + a1 + ul, ul);
+    mA = u.template reduce<kOpMax>(mA);
+    mB = u.template reduce<kOpMax>(mB);
+    float zA = exp_sum(A, mA);
+    float zB = exp_sum(B, mB);
+    zA = u.template reduce<kOpSum>(zA);
+    zB = u.template reduce<kOpSum>(zB);
+    float mnA, mxA, mnB, mxB;
+    scale_store<0>(A, __fdiv_rn(1.0f, zA), (uint32_t*)p.data + a0 + ul, ul, active, mnA, mxA);
+    scale_store<1>(B, __fdiv_rn(1.0f, zB), (uint32_t*)p.data + a1 + ul, ul, active, mnB, mxB);
+    reduce_minmax_bf16<UNIT_>(mnA, mxA);
+    reduce_minmax_bf16<UNIT_>(mnB, mxB);
+    const QRange qA = make_qrange(mnA, mxA), qB = make_qrange(mnB, mxB);
+    if (active && ul == 0) {
+      p.meta[2 * r] = qA.mn; p.meta[2 * r + 1] = qA.s;
+      p.meta[2 * r + 2] = qB.mn; p.meta[2 * r + 3] = qB.s;
+    }
+    // The byte the two rows share: row A's last element is its low nibble, row B's first
+    // its high nibble.  A's nibble travels by shuffle to the lane that owns B's first word.
+    const uint32_t a_last = code_byte<0>(A, G::LAST_I, ul, qA);
+    const uint32_t shared_lo = __shfl_sync(0xffffffffu, a_last, (threadIdx.x & 31 & ~(UNIT_ - 1)) | G::LAST_UL);
+    unsigned char* cA = p.codes + a0 + ul;
+    unsigned char* cB = p.codes + a1 + ul;
+#pragma unroll
+    for (int i = 0; i < G::ITERS; ++i) {
+      if (active && G::has(i, ul)) {
+        if (!(i == G::LAST_I && ul == G::LAST_UL)) cA[UNIT_ * i] = (unsigned char)code_byte<0>(A, i, ul, qA);
+        uint32_t b = code_byte<1>(B, i, ul, qB);
+        if (i == 0 && ul == 0) b |= shared_lo & 0x0Fu;
+        cB[UNIT_ * i] = (unsigned char)b;
+      }
+    }
+    u.sync();  // orders this pair's shared-memory writes before the unit's next pair
   }
 };
 
 template <int DT, int UNIT_, int LCT>
 struct PairSoftmaxBwd {
-  static constexpr int kMaxRegs = 104;
+  static constexpr int kMaxRegs = 96;  // 4 CTAs of 160 threads per SM
   static constexpr int kKernel = kSoftmaxBwd;
   static constexpr int UNIT = UNIT_;
   using P = P2<DT>;
