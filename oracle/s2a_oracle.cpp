@@ -447,6 +447,47 @@ int s2a_oracle_relu_bwd(const void* g, const uint8_t* mask, void* gin, size_t n,
   return 0;
 }
 
+// ---- Channel Average Pooling (Eq. 5): y_k = (1/r) sum_{j<r} x_{k r + j} along the channel
+// axis of an [n_rows, channels] tensor; backward: dL/dx_{k r + j} = (1/r) dL/dy_k.
+int s2a_oracle_cap_fwd(const void* x, void* y, size_t n_rows, size_t channels, size_t r, int dt) {
+  if (r == 0 || channels % r != 0) return 2;
+  const size_t out_ch = channels / r;
+  for (size_t row = 0; row < n_rows; ++row)
+    for (size_t k = 0; k < out_ch; ++k) {
+      double sum = 0.0;
+      for (size_t j = 0; j < r; ++j) sum += load_elem(x, row * channels + k * r + j, dt);
+      store_elem(y, row * out_ch + k, dt, sum / (double)r);
+    }
+  return 0;
+}
+
+int s2a_oracle_cap_bwd(const void* g, void* gin, size_t n_rows, size_t channels, size_t r, int dt) {
+  if (r == 0 || channels % r != 0) return 2;
+  const size_t out_ch = channels / r;
+  for (size_t row = 0; row < n_rows; ++row)
+    for (size_t k = 0; k < out_ch; ++k) {
+      double v = load_elem(g, row * out_ch + k, dt) / (double)r;
+      for (size_t j = 0; j < r; ++j) store_elem(gin, row * channels + k * r + j, dt, v);
+    }
+  return 0;
+}
+
+// ---- Low-Rank Prompt, forward (Eq. 3): y = x + A B with A [tokens, rank], B [rank, channels]
+// (binary32 parameters), the same prompt added to every sample of the batch.  Backward to
+// the activation (Eq. 4) is the identity and needs no kernel.
+int s2a_oracle_lrp_fwd(const void* x, const float* A, const float* B, void* y, size_t batch, size_t tokens,
+                       size_t channels, size_t rank, int dt) {
+  for (size_t b = 0; b < batch; ++b)
+    for (size_t t = 0; t < tokens; ++t)
+      for (size_t c = 0; c < channels; ++c) {
+        double p = 0.0;
+        for (size_t k = 0; k < rank; ++k) p += (double)A[t * rank + k] * (double)B[k * channels + c];
+        size_t e = (b * tokens + t) * channels + c;
+        store_elem(y, e, dt, load_elem(x, e, dt) + p);
+      }
+  return 0;
+}
+
 // Number of hardware threads the row-parallel driver can use.
 int s2a_oracle_hardware_threads() {
   unsigned h = std::thread::hardware_concurrency();

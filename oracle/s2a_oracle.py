@@ -82,6 +82,12 @@ def lib() -> ctypes.CDLL:
         L.s2a_oracle_relu_fwd.restype = i32
         L.s2a_oracle_relu_bwd.argtypes = [vp, vp, vp, sz, i32]
         L.s2a_oracle_relu_bwd.restype = i32
+        L.s2a_oracle_cap_fwd.argtypes = [vp, vp, sz, sz, sz, i32]
+        L.s2a_oracle_cap_fwd.restype = i32
+        L.s2a_oracle_cap_bwd.argtypes = [vp, vp, sz, sz, sz, i32]
+        L.s2a_oracle_cap_bwd.restype = i32
+        L.s2a_oracle_lrp_fwd.argtypes = [vp, vp, vp, vp, sz, sz, sz, sz, i32]
+        L.s2a_oracle_lrp_fwd.restype = i32
         L.s2a_oracle_hardware_threads.argtypes = []
         L.s2a_oracle_hardware_threads.restype = i32
         _lib = L
@@ -270,6 +276,36 @@ def relu_bwd(g, mask, dt: int):
     gin = np.empty_like(g)
     lib().s2a_oracle_relu_bwd(_ptr(g), _ptr(mask), _ptr(gin), g.size, dt)
     return gin
+
+
+def cap_fwd(x, n_rows: int, channels: int, r: int, dt: int):
+    """Channel Average Pooling (Eq. 5): [n_rows, channels] -> [n_rows, channels / r]."""
+    x = _check_io(x, dt).reshape(-1)
+    assert x.size == n_rows * channels
+    y = np.empty(n_rows * (channels // r if r else 0), dtype=x.dtype)
+    if lib().s2a_oracle_cap_fwd(_ptr(x), _ptr(y), n_rows, channels, r, dt) != 0:
+        raise ValueError("oracle rejected the shape")
+    return y
+
+
+def cap_bwd(g, n_rows: int, channels: int, r: int, dt: int):
+    g = _check_io(g, dt).reshape(-1)
+    assert g.size == n_rows * (channels // r)
+    gin = np.empty(n_rows * channels, dtype=g.dtype)
+    if lib().s2a_oracle_cap_bwd(_ptr(g), _ptr(gin), n_rows, channels, r, dt) != 0:
+        raise ValueError("oracle rejected the shape")
+    return gin
+
+
+def lrp_fwd(x, A, B, batch: int, tokens: int, channels: int, rank: int, dt: int):
+    """Low-Rank Prompt (Eq. 3): y[b] = x[b] + A @ B for every sample b."""
+    x = _check_io(x, dt).reshape(-1)
+    A = np.ascontiguousarray(A, dtype=np.float32)
+    B = np.ascontiguousarray(B, dtype=np.float32)
+    assert x.size == batch * tokens * channels and A.size == tokens * rank and B.size == rank * channels
+    y = np.empty_like(x)
+    lib().s2a_oracle_lrp_fwd(_ptr(x), _ptr(A), _ptr(B), _ptr(y), batch, tokens, channels, rank, dt)
+    return y
 
 
 def quantize_tensor(v, row_len: int, dt: int, clip_to_2: bool = False, threads: int = 1):

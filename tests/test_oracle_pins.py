@@ -452,6 +452,41 @@ def test_relu_mask_against_numpy(dt, n):
     assert np.allclose(fd[far], bits[far])
 
 
+# ------------------------------------------------------------------ CAP (Eq. 5) and LRP (Eq. 3)
+@pytest.mark.parametrize("dt", [F32, BF16])
+@pytest.mark.parametrize("rows,ch,r", [(3, 8, 8), (5, 24, 3), (4, 768, 8), (2, 10, 1)])
+def test_cap_against_numpy_mean_and_finite_differences(dt, rows, ch, r):
+    x = synth.to_io(synth.normal(21, ("cap", rows, ch, r), rows * ch), dt)
+    xw = o.widen(x, dt).reshape(rows, ch // r, r)
+    y = o.widen(o.cap_fwd(x, rows, ch, r, dt), dt).reshape(rows, ch // r)
+    tol = 2.0 ** -24 if dt == F32 else 2.0 ** -8
+    assert np.all(np.abs(y - xw.mean(axis=2)) <= tol * np.abs(xw.mean(axis=2)) + 1e-40)
+    g = synth.to_io(synth.normal(21, ("capg", rows, ch, r), rows * ch // r), dt)
+    gw = o.widen(g, dt).reshape(rows, ch // r)
+    gin = o.widen(o.cap_bwd(g, rows, ch, r, dt), dt).reshape(rows, ch // r, r)
+    want = np.repeat((gw / r)[:, :, None], r, axis=2)          # the gradient of a mean: g / r to every input
+    assert np.all(np.abs(gin - want) <= tol * np.abs(want) + 1e-40)
+    # vector-Jacobian identity: <g, CAP(x)> = <CAP^T(g), x>
+    assert float((gw * xw.mean(axis=2)).sum()) == pytest.approx(float((want * xw).sum()), rel=1e-9, abs=1e-12)
+    with pytest.raises(ValueError):
+        o.cap_fwd(x, rows, ch, ch + 1, dt)
+
+
+@pytest.mark.parametrize("dt", [F32, BF16])
+def test_lrp_against_numpy_matmul(dt):
+    batch, tokens, ch, rank = 3, 7, 16, 5
+    x = synth.to_io(synth.normal(22, "lrpx", batch * tokens * ch), dt)
+    A = synth.normal(22, "lrpa", tokens * rank).reshape(tokens, rank)
+    B = synth.normal(22, "lrpb", rank * ch).reshape(rank, ch)
+    y = o.widen(o.lrp_fwd(x, A, B, batch, tokens, ch, rank, dt), dt).reshape(batch, tokens, ch)
+    want = o.widen(x, dt).reshape(batch, tokens, ch) + (A.astype(np.float64) @ B.astype(np.float64))[None]
+    tol = 2.0 ** -24 if dt == F32 else 2.0 ** -8
+    assert np.all(np.abs(y - want) <= tol * np.abs(want) + 1e-40)
+    # A = 0 (the paper's initialisation) leaves the activation unchanged
+    y0 = o.lrp_fwd(x, np.zeros_like(A), B, batch, tokens, ch, rank, dt)
+    assert np.array_equal(y0, x)
+
+
 # ------------------------------------------------------------------ memory accounting
 def test_stash_size_and_the_papers_memory_delta():
     # 0.5 B per element, against the 4 B of the 32-bit activation the paper replaces
