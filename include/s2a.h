@@ -192,6 +192,28 @@ int s2a_relu_fwd(const void* x, void* y, uint8_t* mask, size_t n_elems, int dt, 
 int s2a_relu_bwd(const void* grad_out, const uint8_t* mask, void* grad_in, size_t n_elems, int dt,
                  void* cuda_stream);
 
+/* Channel Average Pooling (Eq. 5), the parameter-free connector of the side branch.
+ * x is [n_rows, channels], y is [n_rows, channels / r]: y_k = (1/r) * sum_{j<r} x_{k r + j};
+ * the sum runs in index order in binary32.  No activation is kept for backward (the
+ * gradient needs only r).  channels must be a multiple of r (else S2A_ERR_SHAPE); x and y
+ * 16-byte aligned.
+ */
+int s2a_cap_fwd(const void* x, void* y, size_t n_rows, size_t channels, size_t r, int dt, void* cuda_stream);
+
+/* Backward of Eq. 5: grad_in_{k r + j} = grad_out_k / r.  grad_out is [n_rows, channels / r],
+ * grad_in is [n_rows, channels].
+ */
+int s2a_cap_bwd(const void* grad_out, void* grad_in, size_t n_rows, size_t channels, size_t r, int dt,
+                void* cuda_stream);
+
+/* Low-Rank Prompt forward (Eq. 3): y[b] = x[b] + A B for every sample b of a
+ * [batch, tokens, channels] activation, with A [tokens, rank] and B [rank, channels] in
+ * binary32 (device pointers).  The product is accumulated in binary32, k in order.  The
+ * gradient to the activation (Eq. 4) is grad_out itself and needs no call.  y may alias x.
+ */
+int s2a_lrp_fwd(const void* x, const float* A, const float* B, void* y, size_t batch, size_t tokens,
+                size_t channels, size_t rank, int dt, void* cuda_stream);
+
 /* The pipelined kernels wait on shared-memory barriers with an iteration limit; a
  * wait that runs out records a bit in a per-device word and the kernel returns early.
  * This call copies that word of the CURRENT device into *flags (0 = no kernel ever gave

@@ -110,6 +110,48 @@ def _time_tensor_range(rows: int, L: int, dtype, seed: int):
     return alg / t / 1e9
 
 
+def _time_side(seed: int):
+    """CAP (r = 8) and the LRP add on the ViT-B/16 batch-64 token stream [64*197, 768] ... [.., 3072]."""
+    out = []
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    for dtype in (torch.bfloat16, torch.float32):
+        item = 2 if dtype == torch.bfloat16 else 4
+        rows, ch, r = 64 * 197 * 4, 3072, 8
+        xs = [torch.randn(rows * ch, device="cuda", generator=g).to(dtype) for _ in range(3)]
+        ys = [torch.empty(rows * ch // r, device="cuda", dtype=dtype) for _ in range(3)]
+
+        def timed(fn, iters=30):
+            for i in range(3):
+                fn(i)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for i in range(iters):
+                fn(i % 3)
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) * 1e-3 / iters
+
+        t_f = timed(lambda i: binding.s2a_cap_fwd(xs[i], ys[i], rows, ch, r))
+        t_b = timed(lambda i: binding.s2a_cap_bwd(ys[i], xs[i], rows, ch, r))
+        alg = rows * ch * item * (1 + 1.0 / r)
+        out.append({"kernel_pair": "cap", "rows": rows, "channels": ch, "r": r,
+                    "io_dtype": "bf16" if dtype == torch.bfloat16 else "f32",
+                    "fwd_GBps": round(alg / t_f / 1e9, 1), "bwd_GBps": round(alg / t_b / 1e9, 1),
+                    "note": "algorithmic bytes = n*itemsize*(1 + 1/r) per kernel"})
+        batch, tokens, chn, rank = 256, 197, 768, 30
+        A = torch.randn(tokens * rank, device="cuda", generator=g)
+        B = torch.randn(rank * chn, device="cuda", generator=g)
+        xl = [torch.randn(batch * tokens * chn, device="cuda", generator=g).to(dtype) for _ in range(3)]
+        yl = [torch.empty_like(x) for x in xl]
+        t = timed(lambda i: binding.s2a_lrp_fwd(xl[i], A, B, yl[i], batch, tokens, chn, rank))
+        out.append({"kernel": "lrp_fwd", "batch": batch, "tokens": tokens, "channels": chn, "rank": rank,
+                    "io_dtype": "bf16" if dtype == torch.bfloat16 else "f32",
+                    "GBps": round(2 * batch * tokens * chn * item / t / 1e9, 1),
+                    "note": "algorithmic bytes = 2*n*itemsize (A and B stay in cache)"})
+    return out
+
+
 def cases(quick: bool):
     out = []
     for n in ((1e6, 1e8) if quick else (1e6, 1e7, 1e8, 1e9, 2e9)):
@@ -132,6 +174,8 @@ def main():
     ap.add_argument("--quick", action="store_true")
     ap.add_argument("--seeds", type=int, default=5)
     args = ap.parse_args()
+    for line in _time_side(0):
+        print(json.dumps(line), flush=True)
     for n in ((10**6, 10**8) if args.quick else (10**6, 10**7, 10**8, 10**9, 2 * 10**9)):
         for dtype in (torch.bfloat16, torch.float32):
             res = []

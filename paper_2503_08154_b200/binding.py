@@ -25,7 +25,7 @@ EXPORTS = (
     "s2a_mask_bytes", "s2a_relu_fwd", "s2a_relu_bwd",
     "s2a_tensor_range_scratch_bytes", "s2a_gelu_fwd_tensor_range",
     "s2a_tensor_range_static_max_elems", "s2a_gelu_fwd_tensor_range_static",
-    "s2a_silu_fwd", "s2a_silu_bwd",
+    "s2a_silu_fwd", "s2a_silu_bwd", "s2a_cap_fwd", "s2a_cap_bwd", "s2a_lrp_fwd",
 )
 
 _lib = None
@@ -66,6 +66,13 @@ def lib() -> ctypes.CDLL:
         L.s2a_gelu_fwd_tensor_range_static.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_size_t,
                                                        c.c_size_t, c.c_int, c.c_void_p]
         L.s2a_gelu_fwd_tensor_range_static.restype = c.c_int
+        for name in ("s2a_cap_fwd", "s2a_cap_bwd"):
+            f = getattr(L, name)
+            f.argtypes = [c.c_void_p, c.c_void_p, c.c_size_t, c.c_size_t, c.c_size_t, c.c_int, c.c_void_p]
+            f.restype = c.c_int
+        L.s2a_lrp_fwd.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_size_t, c.c_size_t, c.c_size_t,
+                                  c.c_size_t, c.c_int, c.c_void_p]
+        L.s2a_lrp_fwd.restype = c.c_int
         L.s2a_mask_bytes.argtypes = [c.c_size_t]
         L.s2a_mask_bytes.restype = c.c_size_t
         for name in ("s2a_relu_fwd", "s2a_relu_bwd"):
@@ -214,6 +221,32 @@ def s2a_gelu_fwd_tensor_range_static(x, y, codes, meta, row_len: int) -> None:
         raise S2AError("codes/meta buffers are too small")
     check(lib().s2a_gelu_fwd_tensor_range_static(x.data_ptr(), y.data_ptr(), codes.data_ptr(), meta.data_ptr(),
                                                  n, row_len, dtype_code(x), _stream_ptr()))
+
+
+def s2a_cap_fwd(x, y, n_rows: int, channels: int, r: int) -> None:
+    _dev(x, "x"), _dev(y, "y")
+    if x.numel() != n_rows * channels or r <= 0 or y.numel() * r != x.numel() or y.dtype != x.dtype:
+        raise S2AError("x must be [n_rows, channels] and y [n_rows, channels / r] of the same dtype")
+    check(lib().s2a_cap_fwd(x.data_ptr(), y.data_ptr(), n_rows, channels, r, dtype_code(x), _stream_ptr()))
+
+
+def s2a_cap_bwd(grad_out, grad_in, n_rows: int, channels: int, r: int) -> None:
+    _dev(grad_out, "grad_out"), _dev(grad_in, "grad_in")
+    if grad_in.numel() != n_rows * channels or r <= 0 or grad_out.numel() * r != grad_in.numel() \
+            or grad_in.dtype != grad_out.dtype:
+        raise S2AError("grad_out must be [n_rows, channels / r] and grad_in [n_rows, channels]")
+    check(lib().s2a_cap_bwd(grad_out.data_ptr(), grad_in.data_ptr(), n_rows, channels, r, dtype_code(grad_out),
+                            _stream_ptr()))
+
+
+def s2a_lrp_fwd(x, A, B, y, batch: int, tokens: int, channels: int, rank: int) -> None:
+    _dev(x, "x"), _dev(y, "y"), _dev(A, "A"), _dev(B, "B")
+    if x.numel() != batch * tokens * channels or y.numel() != x.numel() or y.dtype != x.dtype:
+        raise S2AError("x and y must be [batch, tokens, channels] of the same dtype")
+    if A.dtype != torch.float32 or B.dtype != torch.float32 or A.numel() != tokens * rank or B.numel() != rank * channels:
+        raise S2AError("A must be float32 [tokens, rank] and B float32 [rank, channels]")
+    check(lib().s2a_lrp_fwd(x.data_ptr(), A.data_ptr(), B.data_ptr(), y.data_ptr(), batch, tokens, channels, rank,
+                            dtype_code(x), _stream_ptr()))
 
 
 def mask_bytes(n_elems: int) -> int:

@@ -93,6 +93,38 @@ int s2a_softmax_bwd(const void* grad_out, const uint8_t* codes, const float* met
              const_cast<float*>(meta), n_elems, row_len, dt, cuda_stream);
 }
 
+static int run_cap(bool fwd, const void* in, void* out, size_t n_rows, size_t channels, size_t r, int dt,
+                   void* stream) {
+  if (dt != S2A_F32 && dt != S2A_BF16) return S2A_ERR_DTYPE;
+  if (r == 0 || r > 0x7fffffffull || channels % r != 0) return S2A_ERR_SHAPE;
+  if (n_rows * channels == 0) return S2A_OK;
+  if (!in || !out) return S2A_ERR_NULL;
+  if (misaligned(in, 16) || misaligned(out, 16)) return S2A_ERR_ALIGN;
+  return launch_cap(fwd, dt, in, out, n_rows * (channels / r), (uint32_t)r, (cudaStream_t)stream) == cudaSuccess
+             ? S2A_OK : S2A_ERR_CUDA;
+}
+
+int s2a_cap_fwd(const void* x, void* y, size_t n_rows, size_t channels, size_t r, int dt, void* cuda_stream) {
+  return run_cap(true, x, y, n_rows, channels, r, dt, cuda_stream);
+}
+
+int s2a_cap_bwd(const void* grad_out, void* grad_in, size_t n_rows, size_t channels, size_t r, int dt,
+                void* cuda_stream) {
+  return run_cap(false, grad_out, grad_in, n_rows, channels, r, dt, cuda_stream);
+}
+
+int s2a_lrp_fwd(const void* x, const float* A, const float* B, void* y, size_t batch, size_t tokens,
+                size_t channels, size_t rank, int dt, void* cuda_stream) {
+  if (dt != S2A_F32 && dt != S2A_BF16) return S2A_ERR_DTYPE;
+  if (batch > 0xffffffffull || tokens > 0xffffffffull || channels > 0xffffffffull || rank > 0xffffffffull)
+    return S2A_ERR_SHAPE;
+  if (batch * tokens * channels == 0) return S2A_OK;
+  if (!x || !y || (rank > 0 && (!A || !B))) return S2A_ERR_NULL;
+  if (misaligned(x, 16) || misaligned(y, 16) || misaligned(A, 4) || misaligned(B, 4)) return S2A_ERR_ALIGN;
+  return launch_lrp_fwd(dt, x, A, B, y, (uint32_t)batch, (uint32_t)tokens, (uint32_t)channels, (uint32_t)rank,
+                        (cudaStream_t)cuda_stream) == cudaSuccess ? S2A_OK : S2A_ERR_CUDA;
+}
+
 int s2a_silu_fwd(const void* x, void* y, uint8_t* codes, float* meta, size_t n_elems, size_t row_len, int dt,
                  void* cuda_stream) {
   return run(kSiluFwd, x, y, codes, meta, n_elems, row_len, dt, cuda_stream);

@@ -44,6 +44,12 @@ uint64_t tensor_range_static_max_elems();
 cudaError_t launch_gelu_fwd_tensor_range_static(int dt, const void* x, void* y, uint8_t* codes, float* meta,
                                                 uint64_t n, uint64_t n_rows, cudaStream_t st);
 
+// Channel Average Pooling (flat: n_out outputs, each the mean of r consecutive inputs; the
+// backward spreads g / r) and the Low-Rank Prompt add.
+cudaError_t launch_cap(bool fwd, int dt, const void* in, void* out, uint64_t n_out, uint32_t r, cudaStream_t st);
+cudaError_t launch_lrp_fwd(int dt, const void* x, const float* A, const float* B, void* y, uint32_t batch,
+                           uint32_t tokens, uint32_t channels, uint32_t rank, cudaStream_t st);
+
 // ---------------------------------------------------------------- pipelined tiles
 // A tile is `tile_rows` consecutive rows whose flat element span starts and ends on a
 // multiple of 32 elements, so that its data and its code bytes can move with 16-byte

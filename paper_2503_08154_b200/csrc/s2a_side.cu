@@ -1,0 +1,177 @@
+// The activation-free pieces next to the stash path (Section 3.1): Channel Average Pooling
+// forward/backward (Eq. 5) and the Low-Rank Prompt add (Eq. 3).  Plain memory-bound
+// kernels: grid-stride, 16-byte accesses where the shape allows, scalar otherwise.
+#include "s2a_common.cuh"
+#include "s2a_launch.h"
+
+namespace s2a {
+namespace {
+
+constexpr int kThreads = 256;
+
+int grid_for(uint64_t work_items) {
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  uint64_t want = (work_items + kThreads - 1) / kThreads;
+  const uint64_t cap = (uint64_t)sms * 8;
+  return (int)(want < 1 ? 1 : (want < cap ? want : cap));
+}
+
+__device__ __forceinline__ void widen8(const uint4& r, float* v) {
+  const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    v[2 * k] = __uint_as_float(w[k] << 16);
+    v[2 * k + 1] = __uint_as_float(w[k] & 0xffff0000u);
+  }
+}
+__device__ __forceinline__ uint4 narrow8(const float* v) {
+  uint32_t w[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    __nv_bfloat162 b = __floats2bfloat162_rn(v[2 * k], v[2 * k + 1]);
+    w[k] = *(uint32_t*)&b;
+  }
+  return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// ---- CAP.  channels % r == 0, so groups of r consecutive elements never straddle a row and
+// the tensor can be treated as flat: y[i] = mean(x[i r .. i r + r - 1]).  The sum runs in
+// index order in binary32.  R8 = true is the paper's r = 8 with one (bfloat16) or two
+// (binary32) 16-byte loads per output.
+template <int DT, bool R8>
+__global__ void __launch_bounds__(kThreads) cap_fwd_kernel(const void* xv, void* yv, uint64_t n_out, uint32_t r) {
+  using T = typename Io<DT>::T;
+  const T* x = (const T*)xv;
+  T* y = (T*)yv;
+  const uint64_t stride = (uint64_t)gridDim.x * kThreads;
+  for (uint64_t i = (uint64_t)blockIdx.x * kThreads + threadIdx.x; i < n_out; i += stride) {
+    float sum = 0.0f;
+    if (R8) {
+      float v[8];
+      if (DT == kBF16) {
+        widen8(((const uint4*)xv)[i], v);
+      } else {
+        const float4 a = ((const float4*)xv)[2 * i], b = ((const float4*)xv)[2 * i + 1];
+        v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+      }
+#pragma unroll
+      for (int j = 0; j < 8; ++j) sum += v[j];
+      y[i] = Io<DT>::narrow(sum * 0.125f);
+    } else {
+      for (uint32_t j = 0; j < r; ++j) sum += Io<DT>::widen(x[i * r + j]);
+      y[i] = Io<DT>::narrow(__fdiv_rn(sum, (float)r));
+    }
+  }
+}
+
+template <int DT, bool R8>
+__global__ void __launch_bounds__(kThreads) cap_bwd_kernel(const void* gv, void* ov, uint64_t n_out, uint32_t r) {
+  using T = typename Io<DT>::T;
+  const T* g = (const T*)gv;
+  T* out = (T*)ov;
+  const uint64_t stride = (uint64_t)gridDim.x * kThreads;
+  for (uint64_t i = (uint64_t)blockIdx.x * kThreads + threadIdx.x; i < n_out; i += stride) {
+    const float gi = Io<DT>::widen(g[i]);
+    if (R8) {
+      const float v = gi * 0.125f;
+      if (DT == kBF16) {
+        float vv[8] = {v, v, v, v, v, v, v, v};
+        ((uint4*)ov)[i] = narrow8(vv);
+      } else {
+        ((float4*)ov)[2 * i] = make_float4(v, v, v, v);
+        ((float4*)ov)[2 * i + 1] = make_float4(v, v, v, v);
+      }
+    } else {
+      const T v = Io<DT>::narrow(__fdiv_rn(gi, (float)r));
+      for (uint32_t j = 0; j < r; ++j) out[i * r + j] = v;
+    }
+  }
+}
+
+// ---- LRP forward: y[b, t, c] = x[b, t, c] + sum_k A[t, k] B[k, c].  A thread owns 8
+// consecutive channels of one token: it forms its 8 prompt values once (binary32, k in
+// order) and then streams over its share of the batch.  VEC = false is the scalar form
+// for channel counts that are not a multiple of 8.
+template <int DT, bool VEC>
+__global__ void __launch_bounds__(kThreads) lrp_fwd_kernel(const void* xv, const float* A, const float* B, void* yv,
+                                                           uint32_t batch, uint32_t tokens, uint32_t channels,
+                                                           uint32_t rank) {
+  using T = typename Io<DT>::T;
+  constexpr int W = VEC ? 8 : 1;
+  const uint32_t cgroups = channels / W;
+  const uint64_t items = (uint64_t)tokens * cgroups;
+  const uint64_t item = (uint64_t)blockIdx.x * kThreads + threadIdx.x;
+  if (item >= items) return;
+  const uint32_t t = (uint32_t)(item / cgroups), c0 = (uint32_t)(item % cgroups) * W;
+  float p[W];
+#pragma unroll
+  for (int w = 0; w < W; ++w) p[w] = 0.0f;
+  for (uint32_t k = 0; k < rank; ++k) {
+    const float a = A[(uint64_t)t * rank + k];
+#pragma unroll
+    for (int w = 0; w < W; ++w) p[w] = fmaf(a, B[(uint64_t)k * channels + c0 + w], p[w]);
+  }
+  const uint64_t sample = (uint64_t)tokens * channels;
+  for (uint32_t b = blockIdx.y; b < batch; b += gridDim.y) {
+    const uint64_t e = (uint64_t)b * sample + (uint64_t)t * channels + c0;
+    if (VEC) {
+      float v[8];
+      if (DT == kBF16) {
+        widen8(*(const uint4*)((const T*)xv + e), v);
+      } else {
+        const float4 a = *(const float4*)((const T*)xv + e), b2 = *(const float4*)((const T*)xv + e + 4);
+        v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b2.x; v[5] = b2.y; v[6] = b2.z; v[7] = b2.w;
+      }
+#pragma unroll
+      for (int w = 0; w < 8; ++w) v[w] += p[w];
+      if (DT == kBF16) {
+        *(uint4*)((T*)yv + e) = narrow8(v);
+      } else {
+        *(float4*)((T*)yv + e) = make_float4(v[0], v[1], v[2], v[3]);
+        *(float4*)((T*)yv + e + 4) = make_float4(v[4], v[5], v[6], v[7]);
+      }
+    } else {
+      ((T*)yv)[e] = Io<DT>::narrow(Io<DT>::widen(((const T*)xv)[e]) + p[0]);
+    }
+  }
+}
+
+}  // namespace
+
+template <int DT>
+void launch_cap_dt(bool fwd, bool r8, int grid, const void* in, void* out, uint64_t n_out, uint32_t r, cudaStream_t st) {
+  if (fwd) {
+    if (r8) cap_fwd_kernel<DT, true><<<grid, kThreads, 0, st>>>(in, out, n_out, r);
+    else cap_fwd_kernel<DT, false><<<grid, kThreads, 0, st>>>(in, out, n_out, r);
+  } else {
+    if (r8) cap_bwd_kernel<DT, true><<<grid, kThreads, 0, st>>>(in, out, n_out, r);
+    else cap_bwd_kernel<DT, false><<<grid, kThreads, 0, st>>>(in, out, n_out, r);
+  }
+}
+
+cudaError_t launch_cap(bool fwd, int dt, const void* in, void* out, uint64_t n_out, uint32_t r, cudaStream_t st) {
+  if (n_out == 0) return cudaSuccess;
+  const int grid = grid_for(n_out);
+  if (dt == kF32) launch_cap_dt<kF32>(fwd, r == 8, grid, in, out, n_out, r, st);
+  else launch_cap_dt<kBF16>(fwd, r == 8, grid, in, out, n_out, r, st);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_lrp_fwd(int dt, const void* x, const float* A, const float* B, void* y, uint32_t batch,
+                           uint32_t tokens, uint32_t channels, uint32_t rank, cudaStream_t st) {
+  if ((uint64_t)batch * tokens * channels == 0) return cudaSuccess;
+  const bool vec = channels % 8 == 0;
+  const uint64_t items = (uint64_t)tokens * (vec ? channels / 8 : channels);
+  dim3 grid((unsigned)((items + kThreads - 1) / kThreads), batch < 8 ? batch : 8);
+  if (dt == kF32) {
+    if (vec) lrp_fwd_kernel<kF32, true><<<grid, kThreads, 0, st>>>(x, A, B, y, batch, tokens, channels, rank);
+    else lrp_fwd_kernel<kF32, false><<<grid, kThreads, 0, st>>>(x, A, B, y, batch, tokens, channels, rank);
+  } else {
+    if (vec) lrp_fwd_kernel<kBF16, true><<<grid, kThreads, 0, st>>>(x, A, B, y, batch, tokens, channels, rank);
+    else lrp_fwd_kernel<kBF16, false><<<grid, kThreads, 0, st>>>(x, A, B, y, batch, tokens, channels, rank);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace s2a

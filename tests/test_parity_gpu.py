@@ -269,6 +269,47 @@ def test_silu(rows, L, dt):
     assert plan.startswith("tile") == (L % (4 if dt == F32 else 8) == 0 and rows >= 2 and L <= 8192), plan
 
 
+# ------------------------------------------------------------------ CAP (Eq. 5) and LRP add (Eq. 3)
+@pytest.mark.parametrize("dt", [F32, BF16])
+@pytest.mark.parametrize("rows,ch,r", [(3, 8, 8), (5, 24, 3), (12608, 768, 8), (1000, 96, 4), (7, 10, 1), (64, 1024, 16)])
+def test_cap(rows, ch, r, dt):
+    x = synth.to_io(synth.normal(3, ("cap", rows, ch, r, dt), rows * ch), dt)
+    g = synth.to_io(synth.normal(3, ("capg", rows, ch, r, dt), rows * ch // r), dt)
+    y_o = o.cap_fwd(x, rows, ch, r, dt)
+    gin_o = o.cap_bwd(g, rows, ch, r, dt)
+    item = synth.io_itemsize(dt)
+    tdt = pu.torch_dtype(dt)
+    yg, og = pu.Guarded(rows * ch // r * item), pu.Guarded(rows * ch * item)
+    binding.s2a_cap_fwd(pu.to_device(x, dt), yg.view(tdt), rows, ch, r)
+    binding.s2a_cap_bwd(pu.to_device(g, dt), og.view(tdt), rows, ch, r)
+    torch.cuda.synchronize()
+    yg.check("cap y"), og.check("cap grad_in")
+    mean_abs = np.abs(pu.widen(x, dt)).reshape(-1, r).mean(axis=1)        # size of the summed terms
+    pu.assert_close(pu.widen(pu.to_host(yg.view(tdt), dt), dt), pu.widen(y_o, dt), dt, "cap y",
+                    extra_mag=mean_abs * (1.0 if dt == F32 else 2.0 ** -12))
+    pu.assert_close(pu.widen(pu.to_host(og.view(tdt), dt), dt), pu.widen(gin_o, dt), dt, "cap grad_in")
+
+
+@pytest.mark.parametrize("dt", [F32, BF16])
+@pytest.mark.parametrize("batch,tokens,ch,rank", [(3, 7, 16, 5), (64, 197, 768, 30), (2, 5, 12, 3), (9, 50, 1024, 30)])
+def test_lrp_add(batch, tokens, ch, rank, dt):
+    n = batch * tokens * ch
+    x = synth.to_io(synth.normal(4, ("lrp", batch, tokens, ch, dt), n), dt)
+    A = synth.normal(4, ("lrpA", tokens, rank), tokens * rank)
+    B = synth.normal(4, ("lrpB", rank, ch), rank * ch)
+    y_o = o.lrp_fwd(x, A, B, batch, tokens, ch, rank, dt)
+    tdt = pu.torch_dtype(dt)
+    yg = pu.Guarded(n * synth.io_itemsize(dt))
+    binding.s2a_lrp_fwd(pu.to_device(x, dt), torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda(), yg.view(tdt),
+                        batch, tokens, ch, rank)
+    torch.cuda.synchronize()
+    yg.check("lrp y")
+    terms = np.abs(A.reshape(tokens, rank).astype(np.float64)) @ np.abs(B.reshape(rank, ch).astype(np.float64))
+    mag = np.broadcast_to(terms[None], (batch, tokens, ch)).reshape(-1) + np.abs(pu.widen(x, dt))
+    pu.assert_close(pu.widen(pu.to_host(yg.view(tdt), dt), dt), pu.widen(y_o, dt), dt, "lrp y",
+                    extra_mag=mag * (4.0 if dt == F32 else 2.0 ** -12))
+
+
 # ------------------------------------------------------------------ per-tensor range variant
 @pytest.mark.parametrize("dt", [F32, BF16])
 @pytest.mark.parametrize("rows,L,scale", [(3, 5, 0.3), (1, 1, 1.0), (7, 197, 0.2), (300, 66, 0.4), (64, 3072, 0.25),
