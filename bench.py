@@ -410,23 +410,39 @@ def run_ours(args, shape, blocks, rank, world):
         hy_g = torch.empty(shape.gelu_elems * item, dtype=torch.uint8).pin_memory()
         hy_s = torch.empty(shape.softmax_elems * item, dtype=torch.uint8).pin_memory() if has_softmax else None
 
+        # Host->device copies, kernels and device->host copies run on three streams chained
+        # by events, so that the two PCIe directions and the kernels overlap; every step
+        # still moves all of its inputs in and all of its results out.
+        s_in, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+
+        def staged(copies_in, launch, copies_out):
+            with torch.cuda.stream(s_in):
+                for dst, src in copies_in:
+                    dst.copy_(dview(src), non_blocking=True)
+                ready = torch.cuda.Event()
+                ready.record(s_in)
+            stream.wait_event(ready)
+            launch()
+            done = torch.cuda.Event()
+            done.record(stream)
+            s_out.wait_event(done)
+            with torch.cuda.stream(s_out):
+                for dst, src in copies_out:
+                    dst.copy_(src.view(torch.uint8), non_blocking=True)
+
         def e2e_step():
+            s_in.wait_stream(stream)  # last step's kernels have finished with the input buffers
             for B, (gx, gg, sx, sg) in zip(blks, host):
                 if has_softmax:
-                    B.sx.copy_(dview(sx), non_blocking=True)
-                    binding.s2a_softmax_fwd(B.sx, B.sy, B.scodes, B.smeta, Ls)
-                    hy_s.copy_(B.sy.view(torch.uint8), non_blocking=True)
-                B.gx.copy_(dview(gx), non_blocking=True)
-                binding.s2a_gelu_fwd(B.gx, B.gy, B.gcodes, B.gmeta, Lg)
-                hy_g.copy_(B.gy.view(torch.uint8), non_blocking=True)
+                    staged([(B.sx, sx)], lambda: binding.s2a_softmax_fwd(B.sx, B.sy, B.scodes, B.smeta, Ls),
+                           [(hy_s, B.sy)])
+                staged([(B.gx, gx)], lambda: binding.s2a_gelu_fwd(B.gx, B.gy, B.gcodes, B.gmeta, Lg), [(hy_g, B.gy)])
             for B, (gx, gg, sx, sg) in zip(reversed(blks), reversed(host)):
-                B.gg.copy_(dview(gg), non_blocking=True)
-                binding.s2a_gelu_bwd(B.gg, B.gcodes, B.gmeta, B.gin, Lg)
-                hy_g.copy_(B.gin.view(torch.uint8), non_blocking=True)
+                staged([(B.gg, gg)], lambda: binding.s2a_gelu_bwd(B.gg, B.gcodes, B.gmeta, B.gin, Lg), [(hy_g, B.gin)])
                 if has_softmax:
-                    B.sg.copy_(dview(sg), non_blocking=True)
-                    binding.s2a_softmax_bwd(B.sg, B.scodes, B.smeta, B.sin, Ls)
-                    hy_s.copy_(B.sin.view(torch.uint8), non_blocking=True)
+                    staged([(B.sg, sg)], lambda: binding.s2a_softmax_bwd(B.sg, B.scodes, B.smeta, B.sin, Ls),
+                           [(hy_s, B.sin)])
+            stream.wait_stream(s_out)  # the step ends when its last result is on the host
 
         e2e_step()
         barrier()
