@@ -385,6 +385,74 @@ def test_relu_mask(n, dt):
     assert binding.mask_bytes(n) == (n + 7) // 8
 
 
+def test_softmax_ten_million_rows_of_197():
+    """The largest softmax case of the bandwidth sweep (1e7 rows of 197, 1.97e9 bfloat16
+    elements, beyond 2^32 bytes per tensor): a seeded block of rows repeated down the tensor;
+    every repeat must be identical and the first and last are compared with the oracle."""
+    L, block_rows, repeats = 197, 4000, 2500
+    n = L * block_rows * repeats
+    free, _ = torch.cuda.mem_get_info()
+    if free < 2.7 * 2 * n:
+        pytest.skip("not enough free device memory")
+    x, g = _softmax_inputs(block_rows, L, BF16, seed=8)
+    y_o, codes_o, meta_o = o.softmax_fwd(x, L, BF16, threads=THREADS)
+    xd = pu.to_device(x, BF16).repeat(repeats)
+    yd = torch.empty_like(xd)
+    codes, meta = binding.alloc_stash(n, L, xd.device)
+    binding.s2a_softmax_fwd(xd, yd, codes, meta, L)
+    torch.cuda.synchronize()
+    assert binding.s2a_device_error() == 0
+    yv, cv, mv = yd.view(repeats, -1), codes.view(repeats, -1), meta.view(repeats, -1)
+    assert bool((yv == yv[0]).all()) and bool((cv == cv[0]).all()) and bool((mv == mv[0]).all())
+    for rep in (0, repeats - 1):
+        y_g = pu.to_host(yv[rep], BF16)
+        pu.assert_close(pu.widen(y_g, BF16), pu.widen(y_o, BF16), BF16, "softmax y (large)")
+        q_np, meta_np = pu.numpy_quantize(synth.io_to_f32(y_g, BF16), L)
+        assert np.array_equal(pu.unpack_np(cv[rep].cpu().numpy(), block_rows * L).reshape(block_rows, L), q_np)
+        assert np.array_equal(mv[rep].cpu().numpy().view(np.uint32), meta_np.view(np.uint32))
+    del yd, yv, xd
+    # backward from the oracle's stash, repeated the same way
+    cd = torch.from_numpy(codes_o).cuda().repeat(repeats)
+    md = torch.from_numpy(meta_o).cuda().repeat(repeats)
+    gd = pu.to_device(g, BF16).repeat(repeats)
+    gin = torch.empty_like(gd)
+    binding.s2a_softmax_bwd(gd, cd, md, gin, L)
+    torch.cuda.synchronize()
+    assert binding.s2a_device_error() == 0
+    gv = gin.view(repeats, -1)
+    assert bool((gv == gv[0]).all())
+    gin_o = o.softmax_bwd(g, codes_o, meta_o, L, BF16, threads=THREADS)
+    q_o = pu.unpack_np(codes_o, block_rows * L).reshape(block_rows, L)
+    yh = q_o.astype(np.float64) * meta_o[1::2, None].astype(np.float64) + meta_o[0::2, None].astype(np.float64)
+    M = yh * (np.abs(pu.widen(g, BF16).reshape(block_rows, L)) * yh).sum(axis=1, keepdims=True)
+    pu.assert_close(pu.widen(pu.to_host(gv[repeats - 1], BF16), BF16), pu.widen(gin_o, BF16), BF16,
+                    "softmax grad_in (large)", extra_mag=M)
+
+
+def test_metadata_that_is_only_8_byte_aligned_takes_the_row_path_and_matches():
+    """The pipelined path moves metadata with 16-byte bulk copies; a metadata pointer that is
+    only 8-byte aligned (allowed by the ABI) must be served by the row-at-a-time path with
+    the same results."""
+    rows, L, dt = 256, 3072, BF16
+    x, g = _gelu_inputs(rows, L, dt, seed=12)
+    y_o, codes_o, meta_o = o.gelu_fwd(x, L, dt, threads=THREADS)
+    xd = pu.to_device(x, dt)
+    yd = torch.empty_like(xd)
+    codes = torch.empty(binding.codes_bytes(rows * L), dtype=torch.uint8, device="cuda")
+    meta_big = torch.full((2 * rows + 4,), -7.0, dtype=torch.float32, device="cuda")
+    meta = meta_big[2:2 + 2 * rows]                       # 8 bytes past a 16-byte boundary
+    assert meta.data_ptr() % 16 == 8
+    binding.s2a_gelu_fwd(xd, yd, codes, meta, L)
+    gin = torch.empty_like(xd)
+    binding.s2a_gelu_bwd(pu.to_device(g, dt), codes, meta, gin, L)
+    torch.cuda.synchronize()
+    assert np.array_equal(codes.cpu().numpy(), codes_o) and np.array_equal(meta.cpu().numpy(), meta_o)
+    assert meta_big[:2].tolist() == [-7.0, -7.0] and meta_big[-2:].tolist() == [-7.0, -7.0]
+    pu.assert_close(pu.widen(pu.to_host(yd, dt), dt), pu.widen(y_o, dt), dt, "gelu y (row path)")
+    gin_o = o.gelu_bwd(g, codes_o, meta_o, L, dt, threads=THREADS)
+    pu.assert_close(pu.widen(pu.to_host(gin, dt), dt), pu.widen(gin_o, dt), dt, "gelu grad_in (row path)")
+
+
 def test_stash_bytes_are_half_a_byte_per_element_plus_row_metadata():
     for sh in (synth.VIT_B16_B64, synth.VIT_L16_B64, synth.VIT_H14_B32):
         total = 0
