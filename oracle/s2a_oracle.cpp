@@ -135,7 +135,7 @@ void softmax_vjp_row(const double* y, const double* g, double* gin, size_t n) {
 // Multiplying by inv = 15/d (rather than dividing by the rounded s) keeps the exact
 // tie at the centre of a [-2, 2] row (v = 0, t = 7.5) a tie.  A constant row
 // (d == 0) gets all-zero codes and s = 0, so that dequantisation returns mn.
-void quantize_row(const float* v, size_t n, uint8_t* q, float* mn_out, float* s_out) {
+void quantize_row_levels(const float* v, size_t n, int levels, uint8_t* q, float* mn_out, float* s_out) {
   float mn = v[0], mx = v[0];
   for (size_t i = 1; i < n; ++i) {
     mn = std::min(mn, v[i]);
@@ -148,16 +148,20 @@ void quantize_row(const float* v, size_t n, uint8_t* q, float* mn_out, float* s_
     *s_out = 0.0f;
     return;
   }
-  float s = d / (float)kLevels;
-  float inv = (float)kLevels / d;
+  float s = d / (float)levels;
+  float inv = (float)levels / d;
   for (size_t i = 0; i < n; ++i) {
     float t = (v[i] - mn) * inv;
     float r = std::nearbyintf(t);  // ties-to-even under the default rounding mode
     if (r < 0.0f) r = 0.0f;
-    if (r > (float)kLevels) r = (float)kLevels;
+    if (r > (float)levels) r = (float)levels;
     q[i] = (uint8_t)r;
   }
   *s_out = s;
+}
+
+void quantize_row(const float* v, size_t n, uint8_t* q, float* mn_out, float* s_out) {
+  quantize_row_levels(v, n, kLevels, q, mn_out, s_out);
 }
 
 // Eq. 8 evaluated as printed, in binary64: q = round((v - min) / s), s = (max-min)/15.
@@ -194,6 +198,26 @@ void unpack_codes(const uint8_t* bytes, size_t n, uint8_t* q) {
     q[e] = (e & 1) ? (uint8_t)(b >> 4) : (uint8_t)(b & 0xF);
   }
 }
+
+// General bit width N in {1, 2, 4, 8} (Eq. 8 is stated for any N): element e owns bits
+// [(e N) mod 8, (e N) mod 8 + N) of byte (e N) / 8, least significant first -- for N = 4
+// this is the nibble layout above.
+void pack_codes_bits(const uint8_t* q, size_t n, int bits, uint8_t* bytes) {
+  for (size_t b = 0; b < (n * bits + 7) / 8; ++b) bytes[b] = 0;
+  for (size_t e = 0; e < n; ++e) {
+    size_t bit = e * (size_t)bits;
+    bytes[bit >> 3] |= (uint8_t)((q[e] & ((1u << bits) - 1u)) << (bit & 7));
+  }
+}
+
+void unpack_codes_bits(const uint8_t* bytes, size_t n, int bits, uint8_t* q) {
+  for (size_t e = 0; e < n; ++e) {
+    size_t bit = e * (size_t)bits;
+    q[e] = (uint8_t)((bytes[bit >> 3] >> (bit & 7)) & ((1u << bits) - 1u));
+  }
+}
+
+bool bad_bits(int bits) { return bits != 1 && bits != 2 && bits != 4 && bits != 8; }
 
 // Eq. 9: v_hat = q * s + min, in binary64 from the stored binary32 (min, s).
 double dequantize(uint8_t q, float mn, float s) { return (double)q * (double)s + (double)mn; }
@@ -401,6 +425,67 @@ int s2a_oracle_softmax_bwd(const void* g, const uint8_t* codes, const float* met
     for (size_t i = 0; i < L; ++i) store_elem(gin, r * L + i, dt, out[i]);
   });
   return 0;
+}
+
+// ---- The four kernels at a general bit width N (Eq. 8 with 2^N - 1 levels); N = 4
+// reproduces the functions above bit for bit.  kind: 0 GELU, 1 softmax.
+int s2a_oracle_fwd_bits(int kind, const void* x, void* y, uint8_t* codes, float* meta, size_t n, size_t L,
+                        int bits, int dt) {
+  if (n == 0) return 0;
+  if (bad_shape(n, L) || bad_bits(bits)) return 2;
+  const int levels = (1 << bits) - 1;
+  std::vector<uint8_t> q(n);
+  for (size_t r = 0; r < n / L; ++r) {
+    std::vector<float> v(L);
+    if (kind == 0) {
+      for (size_t i = 0; i < L; ++i) {
+        double xi = load_elem(x, r * L + i, dt);
+        v[i] = (float)std::min(std::max(xi, -2.0), 2.0);
+        store_elem(y, r * L + i, dt, gelu(xi));
+      }
+    } else {
+      std::vector<double> xr(L), yr(L);
+      for (size_t i = 0; i < L; ++i) xr[i] = load_elem(x, r * L + i, dt);
+      softmax_row(xr.data(), yr.data(), L);
+      for (size_t i = 0; i < L; ++i) v[i] = store_elem(y, r * L + i, dt, yr[i]);
+    }
+    quantize_row_levels(v.data(), L, levels, &q[r * L], &meta[2 * r], &meta[2 * r + 1]);
+  }
+  pack_codes_bits(q.data(), n, bits, codes);
+  return 0;
+}
+
+int s2a_oracle_bwd_bits(int kind, const void* g, const uint8_t* codes, const float* meta, void* gin, size_t n,
+                        size_t L, int bits, int dt) {
+  if (n == 0) return 0;
+  if (bad_shape(n, L) || bad_bits(bits)) return 2;
+  std::vector<uint8_t> q(n);
+  unpack_codes_bits(codes, n, bits, q.data());
+  for (size_t r = 0; r < n / L; ++r) {
+    float mn = meta[2 * r], s = meta[2 * r + 1];
+    if (kind == 0) {
+      for (size_t i = 0; i < L; ++i)
+        store_elem(gin, r * L + i, dt,
+                   load_elem(g, r * L + i, dt) * gelu_grad_sine(dequantize(q[r * L + i], mn, s)));
+    } else {
+      std::vector<double> yh(L), gr(L), out(L);
+      for (size_t i = 0; i < L; ++i) {
+        yh[i] = dequantize(q[r * L + i], mn, s);
+        gr[i] = load_elem(g, r * L + i, dt);
+      }
+      softmax_vjp_row(yh.data(), gr.data(), out.data(), L);
+      for (size_t i = 0; i < L; ++i) store_elem(gin, r * L + i, dt, out[i]);
+    }
+  }
+  return 0;
+}
+
+void s2a_oracle_quantize_row_levels(const float* v, size_t n, int levels, uint8_t* q, float* mn, float* s) {
+  quantize_row_levels(v, n, levels, q, mn, s);
+}
+void s2a_oracle_pack_bits(const uint8_t* q, size_t n, int bits, uint8_t* bytes) { pack_codes_bits(q, n, bits, bytes); }
+void s2a_oracle_unpack_bits(const uint8_t* bytes, size_t n, int bits, uint8_t* q) {
+  unpack_codes_bits(bytes, n, bits, q);
 }
 
 // ---- Quantise an already materialised tensor row by row (Eq. 8 + packing); lets a

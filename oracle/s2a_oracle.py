@@ -76,6 +76,16 @@ def lib() -> ctypes.CDLL:
             getattr(L, name).restype = i32
         L.s2a_oracle_gelu_fwd_tensor_range.argtypes = [vp, vp, vp, vp, sz, sz, i32]
         L.s2a_oracle_gelu_fwd_tensor_range.restype = i32
+        L.s2a_oracle_fwd_bits.argtypes = [i32, vp, vp, vp, vp, sz, sz, i32, i32]
+        L.s2a_oracle_fwd_bits.restype = i32
+        L.s2a_oracle_bwd_bits.argtypes = [i32, vp, vp, vp, vp, sz, sz, i32, i32]
+        L.s2a_oracle_bwd_bits.restype = i32
+        L.s2a_oracle_quantize_row_levels.argtypes = [vp, sz, i32, vp, vp, vp]
+        L.s2a_oracle_quantize_row_levels.restype = None
+        L.s2a_oracle_pack_bits.argtypes = [vp, sz, i32, vp]
+        L.s2a_oracle_pack_bits.restype = None
+        L.s2a_oracle_unpack_bits.argtypes = [vp, sz, i32, vp]
+        L.s2a_oracle_unpack_bits.restype = None
         L.s2a_oracle_quantize_tensor.argtypes = [vp, vp, vp, sz, sz, i32, i32, i32]
         L.s2a_oracle_quantize_tensor.restype = i32
         L.s2a_oracle_relu_fwd.argtypes = [vp, vp, vp, sz, i32]
@@ -306,6 +316,59 @@ def lrp_fwd(x, A, B, batch: int, tokens: int, channels: int, rank: int, dt: int)
     y = np.empty_like(x)
     lib().s2a_oracle_lrp_fwd(_ptr(x), _ptr(A), _ptr(B), _ptr(y), batch, tokens, channels, rank, dt)
     return y
+
+
+def codes_bytes_bits(n: int, bits: int) -> int:
+    return (n * bits + 7) // 8
+
+
+def quantize_row_levels(v, levels: int):
+    v = np.ascontiguousarray(v, dtype=np.float32)
+    q = np.empty(v.size, dtype=np.uint8)
+    mn = np.empty(1, dtype=np.float32)
+    s = np.empty(1, dtype=np.float32)
+    lib().s2a_oracle_quantize_row_levels(_ptr(v), v.size, levels, _ptr(q), _ptr(mn), _ptr(s))
+    return q, np.float32(mn[0]), np.float32(s[0])
+
+
+def pack_bits(q, bits: int) -> np.ndarray:
+    q = np.ascontiguousarray(q, dtype=np.uint8)
+    out = np.empty(codes_bytes_bits(q.size, bits), dtype=np.uint8)
+    lib().s2a_oracle_pack_bits(_ptr(q), q.size, bits, _ptr(out))
+    return out
+
+
+def unpack_bits(b, n: int, bits: int) -> np.ndarray:
+    b = np.ascontiguousarray(b, dtype=np.uint8)
+    out = np.empty(n, dtype=np.uint8)
+    lib().s2a_oracle_unpack_bits(_ptr(b), n, bits, _ptr(out))
+    return out
+
+
+def fwd_bits(kind: str, x, row_len: int, bits: int, dt: int):
+    """GELU ('gelu') or softmax ('softmax') forward with an N-bit stash; returns (y, codes, meta)."""
+    x = _check_io(x, dt).reshape(-1)
+    n = x.size
+    y = np.empty_like(x)
+    codes = np.zeros(codes_bytes_bits(n, bits), dtype=np.uint8)
+    meta = np.zeros(2 * (n // row_len if row_len else 0), dtype=np.float32)
+    rc = lib().s2a_oracle_fwd_bits(0 if kind == "gelu" else 1, _ptr(x), _ptr(y), _ptr(codes), _ptr(meta), n,
+                                   row_len, bits, dt)
+    if rc != 0:
+        raise ValueError("oracle rejected the shape or the bit width")
+    return y, codes, meta
+
+
+def bwd_bits(kind: str, g, codes, meta, row_len: int, bits: int, dt: int):
+    g = _check_io(g, dt).reshape(-1)
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    meta = np.ascontiguousarray(meta, dtype=np.float32)
+    gin = np.empty_like(g)
+    rc = lib().s2a_oracle_bwd_bits(0 if kind == "gelu" else 1, _ptr(g), _ptr(codes), _ptr(meta), _ptr(gin), g.size,
+                                   row_len, bits, dt)
+    if rc != 0:
+        raise ValueError("oracle rejected the shape or the bit width")
+    return gin
 
 
 def quantize_tensor(v, row_len: int, dt: int, clip_to_2: bool = False, threads: int = 1):

@@ -380,6 +380,94 @@ def test_gelu_tensor_range_reading(dt):
     assert np.all(np.abs(gin - wantg) <= tol * np.abs(wantg) + 1e-40)
 
 
+# ------------------------------------------------------------------ general bit width (Eq. 8)
+def _exact_codes_levels(v, levels):
+    fr = [Fraction(float(x)) for x in v]
+    mn, mx = min(fr), max(fr)
+    if mx == mn:
+        return [0] * len(fr), [False] * len(fr)
+    codes, ties = [], []
+    for x in fr:
+        t = (x - mn) * levels / (mx - mn)
+        fl = t.numerator // t.denominator
+        rem = t - fl
+        if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and fl % 2 == 1):
+            fl += 1
+        codes.append(int(fl))
+        ties.append(abs(rem - Fraction(1, 2)) < Fraction(1, 10 ** 5))
+    return codes, ties
+
+
+@pytest.mark.parametrize("bits", [1, 2, 4, 8])
+def test_general_bit_width_quantiser_and_packing(bits):
+    levels = 2 ** bits - 1
+    g = np.random.default_rng(bits)
+    for _ in range(40):
+        v = (g.standard_normal(int(g.integers(2, 50))) * 10.0 ** g.uniform(-2, 1)).astype(np.float32)
+        q, mn, s = o.quantize_row_levels(v, levels)
+        want, tie = _exact_codes_levels(v, levels)
+        ok = ~np.array(tie)
+        assert np.array_equal(q[ok], np.array(want)[ok])
+        assert q.max() == levels and q.min() == 0 and mn == v.min()
+        assert float(s) == float(np.float32(np.float32(v.max() - v.min()) / np.float32(levels)))
+    q = g.integers(0, levels + 1, 1003).astype(np.uint8)
+    packed = o.pack_bits(q, bits)
+    assert packed.size == (1003 * bits + 7) // 8
+    # little-endian bit order: numpy's unpackbits recovers the codes
+    bitsarr = np.unpackbits(packed, bitorder="little")[:1003 * bits].reshape(1003, bits)
+    assert np.array_equal((bitsarr * (1 << np.arange(bits))).sum(axis=1), q)
+    assert np.array_equal(o.unpack_bits(packed, 1003, bits), q)
+    if bits == 4:
+        assert np.array_equal(packed, o.pack(q))          # the 4-bit layout is the nibble layout
+
+
+@pytest.mark.parametrize("dt", [F32, BF16])
+@pytest.mark.parametrize("kind,rows,L", [("gelu", 5, 197), ("softmax", 6, 65), ("gelu", 3, 64), ("softmax", 2, 1024)])
+def test_tensor_path_at_other_bit_widths(kind, rows, L, dt):
+    n = rows * L
+    if kind == "gelu":
+        x = synth.to_io(synth.gelu_preact(31, (kind, rows, L), n), dt)
+    else:
+        x = synth.to_io(synth.softmax_logits(31, (kind, rows, L), rows, L), dt)
+    gout = synth.to_io(synth.normal(31, ("g", kind, rows, L), n), dt)
+    # N = 4 is the existing path, bit for bit
+    four = o.fwd_bits(kind, x, L, 4, dt)
+    ref = o.gelu_fwd(x, L, dt) if kind == "gelu" else o.softmax_fwd(x, L, dt)
+    for a, b in zip(four, ref):
+        assert np.array_equal(a, b)
+    ref_b = (o.gelu_bwd if kind == "gelu" else o.softmax_bwd)(gout, ref[1], ref[2], L, dt)
+    assert np.array_equal(o.bwd_bits(kind, gout, four[1], four[2], L, 4, dt), ref_b)
+    prev_err = None
+    for bits in (2, 4, 8):
+        y, codes, meta = o.fwd_bits(kind, x, L, bits, dt)
+        assert np.array_equal(y, ref[0]) and codes.size == (n * bits + 7) // 8
+        q = o.unpack_bits(codes, n, bits).reshape(rows, L)
+        v = (np.clip(o.widen(x, dt), -2, 2) if kind == "gelu" else o.widen(y, dt)).reshape(rows, L)
+        for r in range(rows):
+            want, tie = _exact_codes_levels(v[r].astype(np.float32), 2 ** bits - 1)
+            ok = ~np.array(tie)
+            assert np.array_equal(q[r][ok], np.array(want)[ok])
+        vh = q.astype(np.float64) * meta[1::2, None].astype(np.float64) + meta[0::2, None].astype(np.float64)
+        err = np.abs(vh - v).max()
+        assert err <= 0.5 * float(meta[1::2].max()) * (1 + 1e-5)
+        if prev_err is not None:
+            assert err < prev_err                          # more bits, smaller reconstruction error
+        prev_err = err
+        gin = o.widen(o.bwd_bits(kind, gout, codes, meta, L, bits, dt), dt).reshape(rows, L)
+        gw = o.widen(gout, dt).reshape(rows, L)
+        if kind == "gelu":
+            want_g = gw * (sp.expit(A * vh) + B * np.sin(W * vh))
+            scale = 0.0
+        else:
+            dot = (gw * vh).sum(axis=1, keepdims=True)
+            want_g = vh * (gw - dot)
+            scale = vh * (np.abs(gw) * vh).sum(axis=1, keepdims=True)
+        tol = 2.0 ** -23 if dt == F32 else 2.0 ** -8
+        assert np.all(np.abs(gin - want_g) <= tol * (np.abs(want_g) + scale) + 1e-40)
+    with pytest.raises(ValueError):
+        o.fwd_bits(kind, x, L, 3, dt)
+
+
 # ------------------------------------------------------------------ SiLU / Swish
 def test_silu_closed_forms_and_derivative():
     assert o.silu(0.0) == 0.0 and o.silu_grad(0.0) == 0.5
