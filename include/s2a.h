@@ -192,6 +192,24 @@ int s2a_relu_fwd(const void* x, void* y, uint8_t* mask, size_t n_elems, int dt, 
 int s2a_relu_bwd(const void* grad_out, const uint8_t* mask, void* grad_in, size_t n_elems, int dt,
                  void* cuda_stream);
 
+/* Eq. 8 is stated for a general bit width N; these are the four kernels with N = `bits`.
+ * bits = 4 is exactly s2a_gelu_fwd / _bwd / s2a_softmax_fwd / _bwd (same kernels, same
+ * speed).  bits = 2 and bits = 8 use 3 and 255 quantisation levels, pack 4 codes or 1 code
+ * per byte (element e owns bits [(e N) mod 8, (e N) mod 8 + N) of byte (e N) / 8, least
+ * significant first) and run on the row-at-a-time path only, i.e. well below the bandwidth
+ * of the 4-bit kernels.  codes: s2a_codes_bytes_bits(n_elems, bits) bytes.  Any other
+ * `bits` returns S2A_ERR_SHAPE.  Everything else as for the 4-bit entry points.
+ */
+size_t s2a_codes_bytes_bits(size_t n_elems, int bits);
+int s2a_gelu_fwd_bits(const void* x, void* y, uint8_t* codes, float* meta, size_t n_elems, size_t row_len,
+                      int bits, int dt, void* cuda_stream);
+int s2a_gelu_bwd_bits(const void* grad_out, const uint8_t* codes, const float* meta, void* grad_in, size_t n_elems,
+                      size_t row_len, int bits, int dt, void* cuda_stream);
+int s2a_softmax_fwd_bits(const void* x, void* y, uint8_t* codes, float* meta, size_t n_elems, size_t row_len,
+                         int bits, int dt, void* cuda_stream);
+int s2a_softmax_bwd_bits(const void* grad_out, const uint8_t* codes, const float* meta, void* grad_in,
+                         size_t n_elems, size_t row_len, int bits, int dt, void* cuda_stream);
+
 /* Channel Average Pooling (Eq. 5), the parameter-free connector of the side branch.
  * x is [n_rows, channels], y is [n_rows, channels / r]: y_k = (1/r) * sum_{j<r} x_{k r + j};
  * the sum runs in index order in binary32.  No activation is kept for backward (the

@@ -152,6 +152,36 @@ def _time_side(seed: int):
     return out
 
 
+def _time_bits(seed: int):
+    """The 2-bit and 8-bit forms (row-at-a-time path) on one ViT-B/16 block, bfloat16."""
+    out = []
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    for kind, rows, L in (("gelu", 12608, 3072), ("softmax", 151296, 197)):
+        n = rows * L
+        xs = [torch.randn(n, device="cuda", generator=g).to(torch.bfloat16) for _ in range(3)]
+        ys = [torch.empty_like(x) for x in xs]
+        for bits in (2, 8):
+            codes = [torch.empty(binding.codes_bytes_bits(n, bits), dtype=torch.uint8, device="cuda") for _ in range(3)]
+            meta = [torch.empty(2 * rows, dtype=torch.float32, device="cuda") for _ in range(3)]
+            res = {}
+            for name, fn in (("fwd", lambda i: binding.s2a_fwd_bits(kind, xs[i], ys[i], codes[i], meta[i], L, bits)),
+                             ("bwd", lambda i: binding.s2a_bwd_bits(kind, xs[i], codes[i], meta[i], ys[i], L, bits))):
+                for i in range(3):
+                    fn(i)
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for i in range(12):
+                    fn(i % 3)
+                e1.record()
+                torch.cuda.synchronize()
+                res[name] = (4 * n + n * bits // 8 + 8 * rows) / (e0.elapsed_time(e1) * 1e-3 / 12) / 1e9
+            out.append({"kernel_pair": kind + "_bits", "bits": bits, "rows": rows, "row_len": L, "io_dtype": "bf16",
+                        "fwd_GBps": round(res["fwd"], 1), "bwd_GBps": round(res["bwd"], 1),
+                        "note": "row-at-a-time path; algorithmic bytes = 4*n + n*bits/8 + 8*rows"})
+    return out
+
+
 def cases(quick: bool):
     out = []
     for n in ((1e6, 1e8) if quick else (1e6, 1e7, 1e8, 1e9, 2e9)):
@@ -175,6 +205,8 @@ def main():
     ap.add_argument("--seeds", type=int, default=5)
     args = ap.parse_args()
     for line in _time_side(0):
+        print(json.dumps(line), flush=True)
+    for line in _time_bits(0):
         print(json.dumps(line), flush=True)
     for n in ((10**6, 10**8) if args.quick else (10**6, 10**7, 10**8, 10**9, 2 * 10**9)):
         for dtype in (torch.bfloat16, torch.float32):

@@ -26,6 +26,7 @@ EXPORTS = (
     "s2a_tensor_range_scratch_bytes", "s2a_gelu_fwd_tensor_range",
     "s2a_tensor_range_static_max_elems", "s2a_gelu_fwd_tensor_range_static",
     "s2a_silu_fwd", "s2a_silu_bwd", "s2a_cap_fwd", "s2a_cap_bwd", "s2a_lrp_fwd",
+    "s2a_codes_bytes_bits", "s2a_gelu_fwd_bits", "s2a_gelu_bwd_bits", "s2a_softmax_fwd_bits", "s2a_softmax_bwd_bits",
 )
 
 _lib = None
@@ -73,6 +74,13 @@ def lib() -> ctypes.CDLL:
         L.s2a_lrp_fwd.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_size_t, c.c_size_t, c.c_size_t,
                                   c.c_size_t, c.c_int, c.c_void_p]
         L.s2a_lrp_fwd.restype = c.c_int
+        L.s2a_codes_bytes_bits.argtypes = [c.c_size_t, c.c_int]
+        L.s2a_codes_bytes_bits.restype = c.c_size_t
+        for name in ("s2a_gelu_fwd_bits", "s2a_gelu_bwd_bits", "s2a_softmax_fwd_bits", "s2a_softmax_bwd_bits"):
+            f = getattr(L, name)
+            f.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_size_t, c.c_size_t, c.c_int, c.c_int,
+                          c.c_void_p]
+            f.restype = c.c_int
         L.s2a_mask_bytes.argtypes = [c.c_size_t]
         L.s2a_mask_bytes.restype = c.c_size_t
         for name in ("s2a_relu_fwd", "s2a_relu_bwd"):
@@ -247,6 +255,34 @@ def s2a_lrp_fwd(x, A, B, y, batch: int, tokens: int, channels: int, rank: int) -
         raise S2AError("A must be float32 [tokens, rank] and B float32 [rank, channels]")
     check(lib().s2a_lrp_fwd(x.data_ptr(), A.data_ptr(), B.data_ptr(), y.data_ptr(), batch, tokens, channels, rank,
                             dtype_code(x), _stream_ptr()))
+
+
+def codes_bytes_bits(n_elems: int, bits: int) -> int:
+    return int(lib().s2a_codes_bytes_bits(n_elems, bits))
+
+
+def _call_bits(name, a, b, c_, d, n, row_len, bits, dt_code):
+    check(getattr(lib(), name)(a.data_ptr(), b.data_ptr(), c_.data_ptr(), d.data_ptr(), n, row_len, bits, dt_code,
+                               _stream_ptr()))
+
+
+def s2a_fwd_bits(kind: str, x, y, codes, meta, row_len: int, bits: int) -> None:
+    """s2a_gelu_fwd_bits / s2a_softmax_fwd_bits (kind = 'gelu' or 'softmax')."""
+    _dev(x, "x"), _dev(y, "y"), _dev(codes, "codes"), _dev(meta, "meta")
+    n = x.numel()
+    if y.numel() != n or y.dtype != x.dtype or codes.dtype != torch.uint8 or meta.dtype != torch.float32:
+        raise S2AError("y must match x; codes must be uint8 and meta float32")
+    if codes.numel() < codes_bytes_bits(n, bits) or (row_len > 0 and meta.numel() * 4 < meta_bytes(n, row_len)):
+        raise S2AError("codes/meta buffers are too small")
+    _call_bits("s2a_%s_fwd_bits" % kind, x, y, codes, meta, n, row_len, bits, dtype_code(x))
+
+
+def s2a_bwd_bits(kind: str, grad_out, codes, meta, grad_in, row_len: int, bits: int) -> None:
+    _dev(grad_out, "grad_out"), _dev(grad_in, "grad_in"), _dev(codes, "codes"), _dev(meta, "meta")
+    n = grad_out.numel()
+    if grad_in.numel() != n or grad_in.dtype != grad_out.dtype:
+        raise S2AError("grad_in must match grad_out in size and dtype")
+    _call_bits("s2a_%s_bwd_bits" % kind, grad_out, codes, meta, grad_in, n, row_len, bits, dtype_code(grad_out))
 
 
 def mask_bytes(n_elems: int) -> int:

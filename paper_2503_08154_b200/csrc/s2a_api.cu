@@ -181,6 +181,40 @@ int s2a_relu_bwd(const void* grad_out, const uint8_t* mask, void* grad_in, size_
   return run_relu(false, grad_out, grad_in, const_cast<uint8_t*>(mask), n_elems, dt, cuda_stream);
 }
 
+size_t s2a_codes_bytes_bits(size_t n_elems, int bits) {
+  return (bits == 2 || bits == 4 || bits == 8) ? (n_elems * (size_t)bits + 7) / 8 : 0;
+}
+
+// General code width: 4 goes to the ordinary entry points; 2 and 8 run row at a time.
+static int run_bits(int kernel, const void* in, void* out, uint8_t* codes, float* meta, size_t n, size_t row_len,
+                    int bits, int dt, void* stream) {
+  if (bits == 4) return run(kernel, in, out, codes, meta, n, row_len, dt, stream);
+  if (bits != 2 && bits != 8) return S2A_ERR_SHAPE;
+  int rc = check_args(in, out, codes, meta, n, row_len, dt);
+  if (rc != S2A_OK || n == 0) return rc;
+  RowwiseArgs ra{in, out, codes, meta, 0, n / row_len, (uint32_t)row_len};
+  return launch_rowwise(kernel, dt, ra, (cudaStream_t)stream, bits) == cudaSuccess ? S2A_OK : S2A_ERR_CUDA;
+}
+
+int s2a_gelu_fwd_bits(const void* x, void* y, uint8_t* codes, float* meta, size_t n_elems, size_t row_len,
+                      int bits, int dt, void* cuda_stream) {
+  return run_bits(kGeluFwd, x, y, codes, meta, n_elems, row_len, bits, dt, cuda_stream);
+}
+int s2a_gelu_bwd_bits(const void* grad_out, const uint8_t* codes, const float* meta, void* grad_in, size_t n_elems,
+                      size_t row_len, int bits, int dt, void* cuda_stream) {
+  return run_bits(kGeluBwd, grad_out, grad_in, const_cast<uint8_t*>(codes), const_cast<float*>(meta), n_elems,
+                  row_len, bits, dt, cuda_stream);
+}
+int s2a_softmax_fwd_bits(const void* x, void* y, uint8_t* codes, float* meta, size_t n_elems, size_t row_len,
+                         int bits, int dt, void* cuda_stream) {
+  return run_bits(kSoftmaxFwd, x, y, codes, meta, n_elems, row_len, bits, dt, cuda_stream);
+}
+int s2a_softmax_bwd_bits(const void* grad_out, const uint8_t* codes, const float* meta, void* grad_in,
+                         size_t n_elems, size_t row_len, int bits, int dt, void* cuda_stream) {
+  return run_bits(kSoftmaxBwd, grad_out, grad_in, const_cast<uint8_t*>(codes), const_cast<float*>(meta), n_elems,
+                  row_len, bits, dt, cuda_stream);
+}
+
 int s2a_device_error(unsigned int* flags, int clear) {
   if (!flags) return S2A_ERR_NULL;
   return read_error_word(flags, clear != 0) == cudaSuccess ? S2A_OK : S2A_ERR_CUDA;

@@ -45,7 +45,7 @@ struct QRange {
   float s;    // (max - min) / 15, 0 for a constant row
 };
 
-__device__ __forceinline__ QRange make_qrange(float mn, float mx) {
+__device__ __forceinline__ QRange make_qrange(float mn, float mx, float levels = kLevels) {
   QRange q;
   q.mn = mn;
   float d = __fsub_rn(mx, mn);
@@ -53,17 +53,17 @@ __device__ __forceinline__ QRange make_qrange(float mn, float mx) {
     q.inv = 0.0f;
     q.s = 0.0f;
   } else {
-    q.inv = __fdiv_rn(kLevels, d);
-    q.s = __fdiv_rn(d, kLevels);
+    q.inv = __fdiv_rn(levels, d);
+    q.s = __fdiv_rn(d, levels);
   }
   return q;
 }
 
 // For v inside [min, max] the scaled value lies in [0, 15 + 2^-20], so adding
 // 1.5 * 2^23 rounds it half-to-even into the low mantissa bits without a clamp.
-__device__ __forceinline__ uint32_t quant_code(float v, const QRange& q) {
+__device__ __forceinline__ uint32_t quant_code(float v, const QRange& q, uint32_t mask = 0xFu) {
   float t = __fmul_rn(__fsub_rn(v, q.mn), q.inv);
-  return __float_as_uint(__fadd_rn(t, 12582912.0f)) & 0xFu;
+  return __float_as_uint(__fadd_rn(t, 12582912.0f)) & mask;
 }
 
 // Eq. 9 in binary32: one rounding of the exact code * s + min.

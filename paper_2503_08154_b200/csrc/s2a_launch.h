@@ -27,7 +27,9 @@ struct RowwiseArgs {
   uint32_t row_len;
 };
 
-cudaError_t launch_rowwise(int kernel, int dt, const RowwiseArgs& a, cudaStream_t st);
+// bits: the code width (4 by default; 2 and 8 for the four kernels of the paper).  row0 * row_len
+// must be a multiple of 8 / bits.
+cudaError_t launch_rowwise(int kernel, int dt, const RowwiseArgs& a, cudaStream_t st, int bits = 4);
 
 // ReLU with its 1-bit mask: in = x (forward) or grad_out (backward), out = y or grad_in.
 cudaError_t launch_relu(bool fwd, int dt, const void* in, void* out, uint8_t* mask, uint64_t n, cudaStream_t st);

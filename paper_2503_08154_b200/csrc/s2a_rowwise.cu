@@ -40,24 +40,35 @@ __device__ __forceinline__ float block_reduce(float v, BlockScratch& sc, int slo
   return r;
 }
 
-__device__ __forceinline__ uint32_t nibble_at(const uint8_t* codes, uint64_t e) {
-  uint32_t b = codes[e >> 1];
-  return (e & 1) ? (b >> 4) : (b & 0xFu);
+// The N-bit code of flat element e: bits [(e N) mod 8, +N) of byte (e N) / 8.
+template <int NBITS>
+__device__ __forceinline__ uint32_t code_at(const uint8_t* codes, uint64_t e) {
+  constexpr uint32_t EPB = 8 / NBITS;
+  const uint32_t b = codes[e / EPB];
+  return (b >> ((uint32_t)(e % EPB) * NBITS)) & ((1u << NBITS) - 1u);
 }
 
-template <int KERNEL, int DT>
+// NBITS is the code width of Eq. 8 (4 in the paper; 2 and 8 are the general-N form).  A
+// CTA owns the smallest group of rows that ends on a whole code byte: 8 / NBITS elements
+// share a byte, so up to 4 rows when NBITS = 2 and row_len is odd.
+template <int KERNEL, int DT, int NBITS>
 __global__ void __launch_bounds__(kThreads) rowwise_kernel(RowwiseArgs a) {
   using T = typename Io<DT>::T;
   constexpr int ACT = act_of(KERNEL);
   constexpr float kActClip = Act<ACT>::kClipOf;
+  constexpr uint32_t EPB = 8 / NBITS;                 // elements per code byte
+  constexpr uint32_t kMask = (1u << NBITS) - 1u;
+  constexpr float kLevelsN = (float)((1 << NBITS) - 1);
+  constexpr int kTab = 1 << NBITS;
   __shared__ BlockScratch sc;
-  __shared__ float row_mn[2], row_inv[2], row_s[2], row_aux[2];
-  __shared__ float dtab[2][16];
+  __shared__ float row_mn[4], row_inv[4], row_s[4], row_aux[4];
+  __shared__ float dtab[is_act_bwd(KERNEL) ? 4 : 1][is_act_bwd(KERNEL) ? kTab : 1];
 
   const T* in = (const T*)a.in;
   T* out = (T*)a.out;
   const uint32_t L = a.row_len;
-  const uint32_t P = (L & 1u) ? 2u : 1u;
+  uint32_t P = 1;                                     // rows per group: P * L is a multiple of EPB
+  while ((P * (uint64_t)L) % EPB != 0) P *= 2;
   const uint64_t n_groups = (a.n_rows + P - 1) / P;
   const int tid = threadIdx.x;
 
@@ -65,7 +76,7 @@ __global__ void __launch_bounds__(kThreads) rowwise_kernel(RowwiseArgs a) {
     const uint64_t r0 = a.row0 + g * P;
     const uint64_t rows_left = a.row0 + a.n_rows - r0;
     const uint32_t rows_here = rows_left < P ? (uint32_t)rows_left : P;
-    const uint64_t e0 = r0 * L;  // even by construction
+    const uint64_t e0 = r0 * L;  // a multiple of EPB by construction
     const uint64_t cnt = (uint64_t)rows_here * L;
 
     // ---- per-row statistics ---------------------------------------------------
@@ -81,7 +92,7 @@ __global__ void __launch_bounds__(kThreads) rowwise_kernel(RowwiseArgs a) {
         mn = block_reduce<1>(mn, sc, 0);
         mx = block_reduce<0>(mx, sc, 1);
         // min/max of the clipped row = clipped min/max of the row (the clip is monotone)
-        QRange q = make_qrange(fminf(fmaxf(mn, -kActClip), kActClip), fminf(fmaxf(mx, -kActClip), kActClip));
+        QRange q = make_qrange(fminf(fmaxf(mn, -kActClip), kActClip), fminf(fmaxf(mx, -kActClip), kActClip), kLevelsN);
         if (tid == 0) { row_mn[h] = q.mn; row_inv[h] = q.inv; row_s[h] = q.s; }
       } else if (KERNEL == kSoftmaxFwd) {
         float m = -INFINITY;
@@ -102,16 +113,16 @@ __global__ void __launch_bounds__(kThreads) rowwise_kernel(RowwiseArgs a) {
         }
         mn = block_reduce<1>(mn, sc, 0);
         mx = block_reduce<0>(mx, sc, 1);
-        QRange q = make_qrange(mn, mx);
+        QRange q = make_qrange(mn, mx, kLevelsN);
         if (tid == 0) { row_mn[h] = q.mn; row_inv[h] = q.inv; row_s[h] = q.s; }
       } else if (is_act_bwd(KERNEL)) {
         const float mn = a.meta[2 * (r0 + h)], s = a.meta[2 * (r0 + h) + 1];
-        if (tid < 16) dtab[h][tid] = (float)act_derivative<ACT>((uint32_t)tid, mn, s);
+        if (tid < kTab) dtab[h][tid] = (float)act_derivative<ACT>((uint32_t)tid, mn, s);
       } else {  // kSoftmaxBwd
         const float mn = a.meta[2 * (r0 + h)], s = a.meta[2 * (r0 + h) + 1];
         float dot = 0.0f;
         for (uint32_t i = tid; i < L; i += kThreads) {
-          float yh = dequant(nibble_at(a.codes, base + i), mn, s);
+          float yh = dequant(code_at<NBITS>(a.codes, base + i), mn, s);
           dot = fmaf(Io<DT>::widen(in[base + i]), yh, dot);
         }
         dot = block_reduce<2>(dot, sc, 0);
@@ -125,57 +136,69 @@ __global__ void __launch_bounds__(kThreads) rowwise_kernel(RowwiseArgs a) {
       a.meta[2 * (r0 + tid) + 1] = row_s[tid];
     }
 
-    // ---- element pass, one code byte (two flat-adjacent elements) per step --------
-    const uint64_t n_bytes = (cnt + 1) >> 1;
+    // ---- element pass, one code byte (EPB flat-adjacent elements) per step ----------
+    const uint64_t n_bytes = (cnt + EPB - 1) / EPB;
     for (uint64_t b = tid; b < n_bytes; b += kThreads) {
       uint32_t byte = 0;
-      if (!is_fwd(KERNEL)) byte = a.codes[(e0 >> 1) + b];
+      if (!is_fwd(KERNEL)) byte = a.codes[e0 / EPB + b];
 #pragma unroll
-      for (int k = 0; k < 2; ++k) {
-        const uint64_t rel = 2 * b + k;
+      for (uint32_t k = 0; k < EPB; ++k) {
+        const uint64_t rel = EPB * b + k;
         if (rel < cnt) {
-          const uint32_t h = rel >= L ? 1u : 0u;
+          const uint32_t h = (uint32_t)(rel / L);
           const uint64_t e = e0 + rel;
           if (is_act_fwd(KERNEL)) {
             float x = Io<DT>::widen(in[e]);
             QRange q{row_mn[h], row_inv[h], row_s[h]};
-            byte |= quant_code(fminf(fmaxf(x, -kActClip), kActClip), q) << (4 * k);
+            byte |= quant_code(fminf(fmaxf(x, -kActClip), kActClip), q, kMask) << (NBITS * k);
             out[e] = Io<DT>::narrow(act_value<ACT>(x));
           } else if (KERNEL == kSoftmaxFwd) {
             QRange q{row_mn[h], row_inv[h], row_s[h]};
-            byte |= quant_code(Io<DT>::widen(out[e]), q) << (4 * k);
+            byte |= quant_code(Io<DT>::widen(out[e]), q, kMask) << (NBITS * k);
           } else if (is_act_bwd(KERNEL)) {
-            uint32_t code = (byte >> (4 * k)) & 0xFu;
+            uint32_t code = (byte >> (NBITS * k)) & kMask;
             out[e] = Io<DT>::narrow(Io<DT>::widen(in[e]) * dtab[h][code]);
           } else {
-            uint32_t code = (byte >> (4 * k)) & 0xFu;
+            uint32_t code = (byte >> (NBITS * k)) & kMask;
             float yh = dequant(code, row_mn[h], row_s[h]);
             out[e] = Io<DT>::narrow(yh * (Io<DT>::widen(in[e]) - row_aux[h]));
           }
         }
       }
-      if (is_fwd(KERNEL)) a.codes[(e0 >> 1) + b] = (uint8_t)byte;
+      if (is_fwd(KERNEL)) a.codes[e0 / EPB + b] = (uint8_t)byte;
     }
     __syncthreads();  // shared statistics are reused by the next group
   }
 }
 
-template <int KERNEL, int DT>
+template <int KERNEL, int DT, int NBITS>
 cudaError_t launch_one(const RowwiseArgs& a, cudaStream_t st) {
-  const uint32_t P = (a.row_len & 1u) ? 2u : 1u;
+  uint32_t P = 1;
+  while ((P * (uint64_t)a.row_len) % (8 / NBITS) != 0) P *= 2;
   uint64_t groups = (a.n_rows + P - 1) / P;
   unsigned grid = (unsigned)(groups < (1ull << 20) ? groups : (1ull << 20));
-  rowwise_kernel<KERNEL, DT><<<grid, kThreads, 0, st>>>(a);
+  rowwise_kernel<KERNEL, DT, NBITS><<<grid, kThreads, 0, st>>>(a);
   return cudaGetLastError();
+}
+
+template <int KERNEL, int DT>
+cudaError_t launch_bits(int bits, const RowwiseArgs& a, cudaStream_t st) {
+  if (bits == 4) return launch_one<KERNEL, DT, 4>(a, st);
+  if (KERNEL <= kSoftmaxBwd) {  // the general-N form exists for the four kernels of the paper
+    constexpr int K = KERNEL <= kSoftmaxBwd ? KERNEL : kGeluFwd;
+    if (bits == 2) return launch_one<K, DT, 2>(a, st);
+    if (bits == 8) return launch_one<K, DT, 8>(a, st);
+  }
+  return cudaErrorInvalidValue;
 }
 
 }  // namespace
 
-cudaError_t launch_rowwise(int kernel, int dt, const RowwiseArgs& a, cudaStream_t st) {
+cudaError_t launch_rowwise(int kernel, int dt, const RowwiseArgs& a, cudaStream_t st, int bits) {
   if (a.n_rows == 0) return cudaSuccess;
 #define S2A_CASE(K) \
   case K:           \
-    return dt == kF32 ? launch_one<K, kF32>(a, st) : launch_one<K, kBF16>(a, st);
+    return dt == kF32 ? launch_bits<K, kF32>(bits, a, st) : launch_bits<K, kBF16>(bits, a, st);
   switch (kernel) {
     S2A_CASE(kGeluFwd)
     S2A_CASE(kGeluBwd)

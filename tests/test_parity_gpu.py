@@ -269,6 +269,73 @@ def test_silu(rows, L, dt):
     assert plan.startswith("tile") == (L % (4 if dt == F32 else 8) == 0 and rows >= 2 and L <= 8192), plan
 
 
+# ------------------------------------------------------------------ other bit widths (Eq. 8, general N)
+@pytest.mark.parametrize("dt", [F32, BF16])
+@pytest.mark.parametrize("bits", [2, 4, 8])
+@pytest.mark.parametrize("kind,rows,L", [("gelu", 7, 3), ("gelu", 41, 197), ("gelu", 24, 3072), ("gelu", 5, 1),
+                                         ("softmax", 9, 65), ("softmax", 300, 197), ("softmax", 12, 1024),
+                                         ("softmax", 3, 2), ("softmax", 131, 257)])
+def test_other_bit_widths(kind, rows, L, bits, dt):
+    n = rows * L
+    if kind == "gelu":
+        x, g = _gelu_inputs(rows, L, dt, seed=20 + bits)
+    else:
+        x, g = _softmax_inputs(rows, L, dt, seed=20 + bits)
+    y_o, codes_o, meta_o = o.fwd_bits(kind, x, L, bits, dt)
+    item = synth.io_itemsize(dt)
+    tdt = pu.torch_dtype(dt)
+    yg, cg, mg = pu.Guarded(n * item), pu.Guarded(binding.codes_bytes_bits(n, bits)), pu.Guarded(binding.meta_bytes(n, L))
+    binding.s2a_fwd_bits(kind, pu.to_device(x, dt), yg.view(tdt), cg.view(torch.uint8), mg.view(torch.float32), L, bits)
+    og = pu.Guarded(n * item)
+    binding.s2a_bwd_bits(kind, pu.to_device(g, dt), torch.from_numpy(codes_o).cuda(), torch.from_numpy(meta_o).cuda(),
+                         og.view(tdt), L, bits)
+    torch.cuda.synchronize()
+    for buf, what in ((yg, "y"), (cg, "codes"), (mg, "meta"), (og, "grad_in")):
+        buf.check("%s bits=%d %s" % (kind, bits, what))
+    assert binding.codes_bytes_bits(n, bits) == (n * bits + 7) // 8
+    y_g = pu.to_host(yg.view(tdt), dt)
+    codes_g = cg.view(torch.uint8).cpu().numpy()
+    meta_g = mg.view(torch.float32).cpu().numpy()
+    q_g = o.unpack_bits(codes_g, n, bits).reshape(rows, L)
+    q_o = o.unpack_bits(codes_o, n, bits).reshape(rows, L)
+    xw = pu.widen(x, dt).reshape(rows, L)
+    if kind == "gelu":
+        assert np.array_equal(codes_g, codes_o) and np.array_equal(meta_g.view(np.uint32), meta_o.view(np.uint32))
+        pu.assert_close(pu.widen(y_g, dt), pu.widen(y_o, dt), dt, "gelu y")
+        mag = None
+    else:
+        gap = (xw.max(axis=1, keepdims=True) - xw) * 2.0 ** -24
+        pu.assert_close(pu.widen(y_g, dt), pu.widen(y_o, dt), dt, "softmax y", extra_rtol=gap)
+        # codes are Q_N(y as written): an independent numpy evaluation, zero tolerance
+        v = synth.io_to_f32(y_g, dt).reshape(rows, L)
+        mn, mx = v.min(axis=1, keepdims=True), v.max(axis=1, keepdims=True)
+        d = (mx - mn).astype(np.float32)
+        levels = np.float32(2 ** bits - 1)
+        with np.errstate(divide="ignore", invalid="ignore"):
+            inv = np.where(d == 0, np.float32(0), levels / d).astype(np.float32)
+        q_np = np.rint(((v - mn).astype(np.float32) * inv).astype(np.float32)).astype(np.uint8)
+        assert np.array_equal(q_g, q_np)
+        diff = q_g != q_o
+        assert diff.mean() <= 0.02 and (not diff.any() or np.abs(q_g.astype(int) - q_o.astype(int)).max() <= 1)
+        yh = q_o.astype(np.float64) * meta_o[1::2, None].astype(np.float64) + meta_o[0::2, None].astype(np.float64)
+        mag = yh * (np.abs(pu.widen(g, dt).reshape(rows, L)) * yh).sum(axis=1, keepdims=True)
+    gin_o = o.bwd_bits(kind, g, codes_o, meta_o, L, bits, dt)
+    pu.assert_close(pu.widen(pu.to_host(og.view(tdt), dt), dt), pu.widen(gin_o, dt), dt, "grad_in", extra_mag=mag)
+    if bits == 4:   # the same bytes as the 4-bit entry points
+        y4, c4, m4 = pu.gpu_fwd(kind, x, L, dt)
+        assert np.array_equal(c4, codes_g) and np.array_equal(m4, meta_g) and np.array_equal(y4, y_g)
+
+
+def test_other_bit_widths_reject_unsupported_values():
+    L = binding.lib()
+    x = torch.zeros(64, device="cuda")
+    codes, meta = binding.alloc_stash(64 * 2, 8, "cuda")
+    s = torch.cuda.current_stream().cuda_stream
+    for bits in (0, 1, 3, 16):
+        assert L.s2a_gelu_fwd_bits(x.data_ptr(), x.data_ptr(), codes.data_ptr(), meta.data_ptr(), 64, 8, bits, 0, s) == 2
+        assert binding.codes_bytes_bits(64, bits) == 0
+
+
 # ------------------------------------------------------------------ CAP (Eq. 5) and LRP add (Eq. 3)
 @pytest.mark.parametrize("dt", [F32, BF16])
 @pytest.mark.parametrize("rows,ch,r", [(3, 8, 8), (5, 24, 3), (12608, 768, 8), (1000, 96, 4), (7, 10, 1), (64, 1024, 16)])
