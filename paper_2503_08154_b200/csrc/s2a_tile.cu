@@ -139,7 +139,11 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L) {
   warps = (uint32_t)env_int("S2A_WARPS", (int)warps);
   if (warps < 1 || warps > 16 || (warps * 32) % unit != 0) return p;
   const uint32_t n_units = warps * 32 / unit;
-  const uint32_t G = (!vec16 && (L & 1u)) ? 2u : 1u;
+  uint32_t G = (!vec16 && (L & 1u)) ? 2u : 1u;  // rows a unit takes per round
+  if (variant == kVariantStream && kernel == kSoftmaxFwd) {
+    const uint32_t held = iters * epa;            // elements a lane keeps per row
+    G = held <= 8 ? 4u : (held <= 16 ? 2u : 1u);  // as StreamSoftmaxFwd::RPU
+  }
 
   // tile rows: a multiple of r_min that gives every unit a row (pair) per round, within
   // the stage budget; prefer ~16 KiB of data per tile
@@ -152,7 +156,7 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L) {
     while (rows % (n_units * G) != 0 && (uint64_t)(rows + r_min) * L * esize <= kMaxStageBytes) rows += r_min;
   }
   rows = (uint32_t)env_int("S2A_TILE_ROWS", (int)rows);
-  if (rows == 0 || rows % r_min != 0 || (uint64_t)rows * L * esize > kMaxStageBytes) return p;
+  if (rows == 0 || rows % r_min != 0 || rows % G != 0 || (uint64_t)rows * L * esize > kMaxStageBytes) return p;
 
   const uint32_t data_bytes = rows * L * esize;
   const uint32_t code_bytes = rows * L / 2;

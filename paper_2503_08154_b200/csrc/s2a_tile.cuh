@@ -826,7 +826,10 @@ struct StreamActBwd {
 template <int DT, int UNIT_, int NVL> using StreamGeluBwd = StreamActBwd<DT, UNIT_, NVL, kActGelu>;
 template <int DT, int UNIT_, int NVL> using StreamSiluBwd = StreamActBwd<DT, UNIT_, NVL, kActSilu>;
 
-// Softmax forward on 16-byte vectors, NV vectors per lane kept in registers.
+// Softmax forward on 16-byte vectors, NV vectors per lane kept in registers.  Short rows
+// leave a lane with little work between the four row reductions, so a unit takes RPU rows
+// at a time and walks them phase by phase: each row's shuffle latency hides behind the
+// other rows' arithmetic.
 template <int DT, int UNIT_, int NV>
 struct StreamSoftmaxFwd {
   static constexpr int kMaxRegs = NV * V16<DT>::EPA >= 32 ? 128 : 80;
@@ -834,75 +837,100 @@ struct StreamSoftmaxFwd {
   static constexpr int UNIT = UNIT_;
   using V = V16<DT>;
   static constexpr int EPA = V::EPA;
+  static constexpr int RPU = NV * EPA <= 8 ? 4 : (NV * EPA <= 16 ? 2 : 1);  // rows per unit per round
   struct State {};
   static __device__ __forceinline__ void init(State&) {}
-  static __device__ __forceinline__ uint32_t rows_per_group(uint32_t) { return 1u; }
+  static __device__ __forceinline__ uint32_t rows_per_group(uint32_t) { return RPU; }
 
-  static __device__ __forceinline__ void group(Unit<UNIT_>& u, State&, const StagePtrs& p, float*, uint32_t r,
+  static __device__ __forceinline__ void group(Unit<UNIT_>& u, State&, const StagePtrs& p, float*, uint32_t grp,
                                                bool active, uint32_t L) {
     const uint32_t nv = active ? L / EPA : 0u;
-    unsigned char* row = p.data + (size_t)r * L * Io<DT>::kBytes;
-    unsigned char* crow = p.codes + (size_t)r * (L / 2);
-    float e[NV][EPA];
-    float m = -INFINITY;
+    const uint32_t r0 = grp * RPU;
+    float e[RPU][NV][EPA];
+    float m[RPU], z[RPU], mn[RPU], mx[RPU];
 #pragma unroll
-    for (int i = 0; i < NV; ++i) {
-      const uint32_t j = u.ul + UNIT_ * i;
-      if (j < nv) {
-        V::widen(*(const typename V::Raw*)(row + j * 16u), e[i]);
+    for (int rr = 0; rr < RPU; ++rr) {
+      const unsigned char* row = p.data + (size_t)(r0 + rr) * L * Io<DT>::kBytes;
+      m[rr] = -INFINITY;
 #pragma unroll
-        for (int k = 0; k < EPA; ++k) m = fmaxf(m, e[i][k]);
-      } else {
+      for (int i = 0; i < NV; ++i) {
+        const uint32_t j = u.ul + UNIT_ * i;
+        if (j < nv) {
+          V::widen(*(const typename V::Raw*)(row + j * 16u), e[rr][i]);
 #pragma unroll
-        for (int k = 0; k < EPA; ++k) e[i][k] = -INFINITY;
+          for (int k = 0; k < EPA; ++k) m[rr] = fmaxf(m[rr], e[rr][i][k]);
+        } else {
+#pragma unroll
+          for (int k = 0; k < EPA; ++k) e[rr][i][k] = -INFINITY;
+        }
       }
     }
-    m = u.template reduce<kOpMax>(m);
-    if (!active) m = 0.0f;
-    float z = 0.0f;
+#pragma unroll
+    for (int rr = 0; rr < RPU; ++rr) {
+      m[rr] = u.template reduce<kOpMax>(m[rr]);
+      if (!active) m[rr] = 0.0f;
+    }
     constexpr float kLog2e = 1.4426950408889634f;
-    const float nm = -m * kLog2e;
 #pragma unroll
-    for (int i = 0; i < NV; ++i)
+    for (int rr = 0; rr < RPU; ++rr) {
+      const float nm = -m[rr] * kLog2e;
+      z[rr] = 0.0f;
 #pragma unroll
-      for (int k = 0; k < EPA; ++k) {
-        // bfloat16: the exponent's argument is one fused multiply-add (the result is rounded to 8 bits)
-        e[i][k] = DT == kBF16 ? ex2_approx(fmaf(e[i][k], kLog2e, nm)) : exp_eval<DT>(e[i][k] - m);
-        z += e[i][k];
+      for (int i = 0; i < NV; ++i)
+#pragma unroll
+        for (int k = 0; k < EPA; ++k) {
+          // bfloat16: the exponent's argument is one fused multiply-add (the result is rounded to 8 bits)
+          e[rr][i][k] = DT == kBF16 ? ex2_approx(fmaf(e[rr][i][k], kLog2e, nm)) : exp_eval<DT>(e[rr][i][k] - m[rr]);
+          z[rr] += e[rr][i][k];
+        }
+    }
+#pragma unroll
+    for (int rr = 0; rr < RPU; ++rr) z[rr] = u.template reduce<kOpSum>(z[rr]);
+#pragma unroll
+    for (int rr = 0; rr < RPU; ++rr) {
+      unsigned char* row = p.data + (size_t)(r0 + rr) * L * Io<DT>::kBytes;
+      const float rz = __fdiv_rn(1.0f, active ? z[rr] : 1.0f);
+      typename V::MinMax mm;
+      mm.init();
+#pragma unroll
+      for (int i = 0; i < NV; ++i) {
+        const uint32_t j = u.ul + UNIT_ * i;
+        if (j < nv) {
+#pragma unroll
+          for (int k = 0; k < EPA; ++k) e[rr][i][k] *= rz;
+          const typename V::Raw yw = V::narrow(e[rr][i]);  // e now holds y as written
+          *(typename V::Raw*)(row + j * 16u) = yw;
+          mm.add(yw);
+        }
       }
-    z = u.template reduce<kOpSum>(z);
-    const float rz = __fdiv_rn(1.0f, active ? z : 1.0f);
-    typename V::MinMax mm;
-    mm.init();
+      mn[rr] = mm.lo();
+      mx[rr] = mm.hi();
+    }
 #pragma unroll
-    for (int i = 0; i < NV; ++i) {
-      const uint32_t j = u.ul + UNIT_ * i;
-      if (j < nv) {
-#pragma unroll
-        for (int k = 0; k < EPA; ++k) e[i][k] *= rz;
-        const typename V::Raw yw = V::narrow(e[i]);  // e now holds y as written
-        *(typename V::Raw*)(row + j * 16u) = yw;
-        mm.add(yw);
+    for (int rr = 0; rr < RPU; ++rr) {
+      if (DT == kBF16) {
+        reduce_minmax_bf16<UNIT_>(mn[rr], mx[rr]);
+      } else {
+        mn[rr] = u.template reduce<kOpMin>(mn[rr]);
+        mx[rr] = u.template reduce<kOpMax>(mx[rr]);
       }
     }
-    float mn = mm.lo(), mx = mm.hi();
-    if (DT == kBF16) {
-      reduce_minmax_bf16<UNIT_>(mn, mx);
-    } else {
-      mn = u.template reduce<kOpMin>(mn);
-      mx = u.template reduce<kOpMax>(mx);
-    }
-    const QRange q = make_qrange(mn, mx);
-    if (active && u.ul == 0) { p.meta[2 * r] = q.mn; p.meta[2 * r + 1] = q.s; }
 #pragma unroll
-    for (int i = 0; i < NV; ++i) {
-      const uint32_t j = u.ul + UNIT_ * i;
-      if (j < nv) {
-        CodePacker<EPA> pk;
-        pk.init();
+    for (int rr = 0; rr < RPU; ++rr) {
+      const uint32_t r = r0 + rr;
+      unsigned char* crow = p.codes + (size_t)r * (L / 2);
+      const QRange q = make_qrange(mn[rr], mx[rr]);
+      if (active && u.ul == 0) { p.meta[2 * r] = q.mn; p.meta[2 * r + 1] = q.s; }
 #pragma unroll
-        for (int k = 0; k < EPA; ++k) pk.add(k, e[i][k], q);
-        V::store_codes(crow, j, pk.acc);
+      for (int i = 0; i < NV; ++i) {
+        const uint32_t j = u.ul + UNIT_ * i;
+        if (j < nv) {
+          CodePacker<EPA> pk;
+          pk.init();
+#pragma unroll
+          for (int k = 0; k < EPA; ++k) pk.add(k, e[rr][i][k], q);
+          V::store_codes(crow, j, pk.acc);
+        }
       }
     }
   }
