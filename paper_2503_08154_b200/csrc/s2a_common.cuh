@@ -101,6 +101,28 @@ __device__ __forceinline__ float act_value(float x) {
 }
 __device__ __forceinline__ float gelu_value(float x) { return act_value<kActGelu>(x); }
 
+// Fast forms for bfloat16 outputs (the result is rounded to 8 bits): one special-function
+// exponential and one reciprocal.
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float rcp_approx(float x) {
+  float y;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+template <int DT, int ACT = kActGelu>
+__device__ __forceinline__ float gelu_eval(float x) {
+  if (DT == kF32) return act_value<ACT>(x);
+  // y = x / (1 + 2^(-1.702 log2(e) x)).  For x < -52 the power overflows and y becomes
+  // -0 instead of a value below 2^-120: the bfloat16 path flushes such results.
+  constexpr float c = -Act<ACT>::kSlopeOf * 1.4426950408889634f;
+  return x * rcp_approx(1.0f + ex2_approx(c * x));
+}
+
 // The derivative used by the backward pass at a dequantised x_hat = code * s + min, in
 // binary64: Eq. 12 for GELU, the exact derivative for SiLU.
 template <int ACT>

@@ -163,7 +163,13 @@ cudaError_t launch_lrp_fwd(int dt, const void* x, const float* A, const float* B
   if ((uint64_t)batch * tokens * channels == 0) return cudaSuccess;
   const bool vec = channels % 8 == 0;
   const uint64_t items = (uint64_t)tokens * (vec ? channels / 8 : channels);
-  dim3 grid((unsigned)((items + kThreads - 1) / kThreads), batch < 8 ? batch : 8);
+  // enough threads to fill the machine: the batch is split over gridDim.y (each split forms
+  // its prompt values again, 30 multiply-adds per element of one sample)
+  uint64_t splits = (148ull * 2048 + items - 1) / items;
+  if (splits > batch) splits = batch;
+  if (splits > 64) splits = 64;
+  if (splits < 1) splits = 1;
+  dim3 grid((unsigned)((items + kThreads - 1) / kThreads), (unsigned)splits);
   if (dt == kF32) {
     if (vec) lrp_fwd_kernel<kF32, true><<<grid, kThreads, 0, st>>>(x, A, B, y, batch, tokens, channels, rank);
     else lrp_fwd_kernel<kF32, false><<<grid, kThreads, 0, st>>>(x, A, B, y, batch, tokens, channels, rank);

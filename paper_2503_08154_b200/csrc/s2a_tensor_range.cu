@@ -124,7 +124,7 @@ __global__ void __launch_bounds__(kThreads) fixed_range_fwd(const void* x, void*
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
       bits |= quant_code(fminf(fmaxf(v[k], -kClip), kClip), q) << (4 * k);
-      v[k] = gelu_value(v[k]);
+      v[k] = gelu_eval<DT>(v[k]);
     }
     store8<DT>(y, o, v);
     ((uint32_t*)codes)[o] = bits;
@@ -134,7 +134,7 @@ __global__ void __launch_bounds__(kThreads) fixed_range_fwd(const void* x, void*
     for (uint64_t e = n8 << 3; e < n; ++e) {
       const float xe = Io<DT>::widen(((const T*)x)[e]);
       bits |= quant_code(fminf(fmaxf(xe, -kClip), kClip), q) << (4 * (e & 7u));
-      ((T*)y)[e] = Io<DT>::narrow(gelu_value(xe));
+      ((T*)y)[e] = Io<DT>::narrow(gelu_eval<DT>(xe));
     }
     for (uint64_t b = n8 * 4; b < (n + 1) / 2; ++b) codes[b] = (uint8_t)(bits >> (8 * (b - n8 * 4)));
   }
