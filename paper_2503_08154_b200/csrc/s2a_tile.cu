@@ -206,7 +206,8 @@ cudaError_t launch_tile(int kernel, int dt, const TilePlan& p, const TileArgs& a
   ka.out = (unsigned char*)a.out;
   ka.codes = a.codes;
   ka.meta = (unsigned char*)a.meta;
-  ka.n_tiles = a.n_tiles;
+  ka.tiles_per_cta = a.n_tiles / p.grid;
+  ka.tiles_extra = (uint32_t)(a.n_tiles % p.grid);
   ka.row_len = a.row_len;
   ka.tile_rows = p.tile_rows;
   const uint32_t esize = dt == kF32 ? 4u : 2u;

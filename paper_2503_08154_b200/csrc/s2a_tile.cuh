@@ -40,7 +40,8 @@ struct TileKernelArgs {
   unsigned char* out;
   unsigned char* codes;
   unsigned char* meta;
-  uint64_t n_tiles;
+  uint64_t tiles_per_cta;  // n_tiles / grid; the first tiles_extra CTAs take one more
+  uint32_t tiles_extra;    // n_tiles % grid
   uint32_t row_len;
   uint32_t tile_rows;
   uint32_t data_bytes;   // per tile
@@ -85,6 +86,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // warps it is waiting for).
 template <int SLEEP_NS = 0>
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned int* err, unsigned err_bit) {
+#pragma unroll 1
   for (uint32_t i = 0; i < kSpinLimit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
@@ -1320,8 +1322,11 @@ __global__ void __maxnreg__(WORK::kMaxRegs) tile_kernel(TileKernelArgs a) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_cwarps = (blockDim.x >> 5) - 1;
   const uint32_t S = a.stages;
-  const uint64_t my_tiles =
-      a.n_tiles > blockIdx.x ? (a.n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+  // Tiles go round-robin over the CTAs.  Stage and phase of a tile are carried along the
+  // loops (a 64-bit division is a long instruction sequence), and the loops of the frame
+  // stay rolled: the four kernels of a training step should fit the instruction cache
+  // together.
+  const uint64_t my_tiles = a.tiles_per_cta + (blockIdx.x < a.tiles_extra ? 1u : 0u);
 
   if (threadIdx.x == 0) {
     for (uint32_t s = 0; s < S; ++s) {
@@ -1342,11 +1347,10 @@ __global__ void __maxnreg__(WORK::kMaxRegs) tile_kernel(TileKernelArgs a) {
   if (warp == n_cwarps) {
     // ------------------------------------------------------------ copy warp
     if (lane != 0) return;
-    auto stage_ptr = [&](uint64_t it) { return smem + kHeaderBytes + (size_t)(it % S) * a.stage_bytes; };
-    auto issue_load = [&](uint64_t it) {
+    auto issue_load = [&](uint64_t it, uint32_t s) {
       const uint64_t t = blockIdx.x + it * gridDim.x;
-      unsigned char* st = stage_ptr(it);
-      uint64_t* bar = &full[it % S];
+      unsigned char* st = smem + kHeaderBytes + (size_t)s * a.stage_bytes;
+      uint64_t* bar = &full[s];
       const uint32_t bytes = kFwd ? a.data_bytes : a.data_bytes + a.code_bytes + a.meta_bytes;
       mbar_arrive_expect_tx(bar, bytes);
       bulk_load(st, a.in + t * a.data_bytes, a.data_bytes, bar);
@@ -1355,15 +1359,18 @@ __global__ void __maxnreg__(WORK::kMaxRegs) tile_kernel(TileKernelArgs a) {
         bulk_load(st + a.meta_off, a.meta + t * a.meta_bytes, a.meta_bytes, bar);
       }
     };
-    const uint64_t pre = my_tiles < S ? my_tiles : S;
-    for (uint64_t it = 0; it < pre; ++it) issue_load(it);
+    const uint32_t pre = my_tiles < S ? (uint32_t)my_tiles : S;
+#pragma unroll 1
+    for (uint32_t s = 0; s < pre; ++s) issue_load(s, s);
     uint64_t issued = pre;
     uint64_t it = 0;
+    uint32_t s = 0, phase = 0;  // stage and phase of tile `it`
     bool ok = true;
+#pragma unroll 1
     for (; it < my_tiles; ++it) {
-      if (!mbar_wait<200>(&done[it % S], (uint32_t)((it / S) & 1), a.error_word, kErrDrainWait)) { ok = false; break; }
+      if (!mbar_wait<200>(&done[s], phase, a.error_word, kErrDrainWait)) { ok = false; break; }
       const uint64_t t = blockIdx.x + it * gridDim.x;
-      unsigned char* st = stage_ptr(it);
+      unsigned char* st = smem + kHeaderBytes + (size_t)s * a.stage_bytes;
       bulk_store(a.out + t * a.data_bytes, st, a.data_bytes);
       if (kFwd) {
         bulk_store(a.codes + t * a.code_bytes, st + a.code_off, a.code_bytes);
@@ -1371,16 +1378,20 @@ __global__ void __maxnreg__(WORK::kMaxRegs) tile_kernel(TileKernelArgs a) {
       }
       bulk_commit();
       if (issued < my_tiles) {
-        bulk_wait_read<0>();  // the stores of this tile have left shared memory
-        issue_load(issued);   // == it + S: refills the stage just drained
+        bulk_wait_read<0>();    // the stores of this tile have left shared memory
+        issue_load(issued, s);  // tile it + S refills the stage just drained
         ++issued;
       }
+      if (++s == S) { s = 0; phase ^= 1u; }
     }
     bulk_wait_all();
     if (!ok) {
       // wind down: let every load already issued land before shared memory is released
-      for (uint64_t j = it; j < issued; ++j)
-        mbar_wait(&full[j % S], (uint32_t)((j / S) & 1), a.error_word, kErrLoadWait);
+#pragma unroll 1
+      for (uint64_t j = it; j < issued; ++j) {
+        mbar_wait(&full[s], phase, a.error_word, kErrLoadWait);
+        if (++s == S) { s = 0; phase ^= 1u; }
+      }
     }
     return;
   }
@@ -1402,9 +1413,10 @@ __global__ void __maxnreg__(WORK::kMaxRegs) tile_kernel(TileKernelArgs a) {
   const uint32_t n_groups = a.tile_rows / WORK::rows_per_group(L);
   const uint32_t rounds = (n_groups + n_units - 1) / n_units;
 
+  uint32_t s = 0, phase = 0;  // stage and phase of tile `it`
+#pragma unroll 1
   for (uint64_t it = 0; it < my_tiles; ++it) {
-    const uint32_t s = (uint32_t)(it % S);
-    bool ok = mbar_wait(&full[s], (uint32_t)((it / S) & 1), a.error_word, kErrLoadWait);
+    bool ok = mbar_wait(&full[s], phase, a.error_word, kErrLoadWait);
     ok = __all_sync(0xffffffffu, ok);
     if (UNIT > 32) {
       if (!ok && lane == 0) *(volatile int*)abort_flag = 1;
@@ -1431,6 +1443,7 @@ __global__ void __maxnreg__(WORK::kMaxRegs) tile_kernel(TileKernelArgs a) {
     fence_proxy_async();  // this thread's shared-memory writes -> visible to the copy engine
     __syncwarp();
     if (lane == 0) mbar_arrive(&done[s]);
+    if (++s == S) { s = 0; phase ^= 1u; }
   }
 }
 
