@@ -27,6 +27,8 @@ namespace s2a {
 namespace {
 
 constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr uint32_t kSuspendNs = 100000;             // longest sleep inside one try
+constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s: a wait this long has failed
 constexpr int kMaxStages = 8;
 constexpr int kHeaderBytes = 4096;  // barriers, reduction scratch, derivative tables
 constexpr int kRedOffset = 256;     // float[2 slots][16 units][4 warps]  (multi-warp units)
@@ -81,15 +83,34 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait for the phase with the given parity to complete.  SLEEP_NS > 0 backs off
-// between tries (used by the copy lane, which would otherwise take issue slots from the
-// warps it is waiting for).
-template <int SLEEP_NS = 0>
+// The same test, but the warp may sleep in hardware for up to `ns` nanoseconds and is woken
+// when the phase completes: a waiting warp then takes no issue slots from the warps it is
+// waiting for (a polling loop of the copy lane was a fifth of all instructions issued).
+__device__ __forceinline__ bool mbar_try_wait_suspend(uint64_t* bar, uint32_t parity, uint32_t ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(ns)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait for the phase with the given parity to complete: gives up after
+// kWaitLimitNs of wall time or kSpinLimit tries, whichever comes first, and records why.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned int* err, unsigned err_bit) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_timer_ns();
 #pragma unroll 1
   for (uint32_t i = 0; i < kSpinLimit; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
+    if (mbar_try_wait_suspend(bar, parity, kSuspendNs)) return true;
+    if (global_timer_ns() - t0 > kWaitLimitNs) break;
   }
   atomicOr(err, err_bit);
   return false;
@@ -1368,7 +1389,7 @@ __global__ void __maxnreg__(WORK::kMaxRegs) tile_kernel(TileKernelArgs a) {
     bool ok = true;
 #pragma unroll 1
     for (; it < my_tiles; ++it) {
-      if (!mbar_wait<200>(&done[s], phase, a.error_word, kErrDrainWait)) { ok = false; break; }
+      if (!mbar_wait(&done[s], phase, a.error_word, kErrDrainWait)) { ok = false; break; }
       const uint64_t t = blockIdx.x + it * gridDim.x;
       unsigned char* st = smem + kHeaderBytes + (size_t)s * a.stage_bytes;
       bulk_store(a.out + t * a.data_bytes, st, a.data_bytes);
