@@ -95,16 +95,17 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L) {
       if ((per >= 3 && per <= 6) || per == 8 || per == 10) iters = per;
     }
   } else if (vec16 && !force_generic) {
-    // softmax on 16-byte vectors: up to 32 (at most 64) elements per lane in registers
+    // softmax on 16-byte vectors: up to 32 (at most 64) elements per lane in registers; rows
+    // too long for a warp go to units of two or four warps
     const uint32_t cap = 32u / epa, cap2 = 64u / epa;
-    const uint32_t units[3] = {8, 16, 32};
-    for (int k = 0; k < 3 && unit == 0; ++k)
+    const uint32_t units[5] = {8, 16, 32, 64, 128};
+    for (int k = 0; k < 5 && unit == 0; ++k)
       if ((n_acc + units[k] - 1) / units[k] <= cap) unit = units[k];
-    if (unit == 0 && (n_acc + 31) / 32 <= cap2) unit = 32;
-    if (env_unit == 8 || env_unit == 16 || env_unit == 32) unit = (uint32_t)env_unit;
+    if (unit == 0 && (n_acc + 127) / 128 <= cap2) unit = 128;
+    if (env_unit == 8 || env_unit == 16 || env_unit == 32 || env_unit == 64 || env_unit == 128) unit = (uint32_t)env_unit;
     if (unit != 0 && (n_acc + unit - 1) / unit <= cap2) {
       variant = kVariantStream;
-      iters = 1;
+      iters = unit >= 64 ? 4 : 1;
       while (iters < (n_acc + unit - 1) / unit) iters *= 2;
     } else {
       unit = 0;
@@ -133,6 +134,12 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L) {
   }
 
   uint32_t warps = unit == 128 ? 8u : 4u;
+  if (variant == kVariantStream && !is_gelu) {
+    // A softmax row is a chain of dependent phases (reduce, evaluate, reduce, ...).  With few
+    // elements per lane, or the cheaper bfloat16 arithmetic, four warps leave the SM waiting
+    // on shuffles; binary32 rows with 32 elements per lane run best with four (measured).
+    warps = (dt == kBF16 || iters * epa <= 16) ? 8u : 4u;
+  }
   int ctas_per_sm = 2;
   if (variant == kVariantStream && is_gelu) ctas_per_sm = 4;
   if (variant == kVariantPairFixed) ctas_per_sm = 4;
@@ -172,6 +179,13 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L) {
   // (measured: 50.5 KB and 52.5 KB requests in alternation cost 3.7 us per launch).
   ctas_per_sm = env_int("S2A_CTAS_PER_SM", ctas_per_sm);
   if (ctas_per_sm != 1 && ctas_per_sm != 2 && ctas_per_sm != 4) ctas_per_sm = 2;
+  {
+    // registers bound the residency too: the kernels' register caps, by variant
+    uint32_t regs = 128;
+    if (variant == kVariantStream) regs = is_gelu ? 64u : (uint32_t)softmax_stream_regs(dt, (int)(iters * epa));
+    if (variant == kVariantPairFixed) regs = 96;
+    while (ctas_per_sm > 1 && (uint64_t)regs * (warps + 1) * 32 * (uint32_t)ctas_per_sm > 65536) ctas_per_sm /= 2;
+  }
   const int env_stages = env_int("S2A_STAGES", 0);
   uint32_t stages = 0, smem = 0;
   for (int c = ctas_per_sm; c >= 1 && stages == 0; c /= 2) {

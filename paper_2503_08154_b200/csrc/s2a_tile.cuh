@@ -828,13 +828,19 @@ struct StreamActBwd {
 template <int DT, int UNIT_, int NVL> using StreamGeluBwd = StreamActBwd<DT, UNIT_, NVL, kActGelu>;
 template <int DT, int UNIT_, int NVL> using StreamSiluBwd = StreamActBwd<DT, UNIT_, NVL, kActSilu>;
 
+// Register cap of the streamed softmax kernels by elements held per lane (the planner
+// derives the CTAs that fit an SM from the same number).
+constexpr int softmax_stream_regs(int dt, int held) {
+  return held >= 64 ? 128 : (held >= 32 ? (dt == kBF16 ? 112 : 128) : 80);
+}
+
 // Softmax forward on 16-byte vectors, NV vectors per lane kept in registers.  Short rows
 // leave a lane with little work between the four row reductions, so a unit takes RPU rows
 // at a time and walks them phase by phase: each row's shuffle latency hides behind the
 // other rows' arithmetic.
 template <int DT, int UNIT_, int NV>
 struct StreamSoftmaxFwd {
-  static constexpr int kMaxRegs = NV * V16<DT>::EPA >= 32 ? 128 : 80;
+  static constexpr int kMaxRegs = softmax_stream_regs(DT, NV * V16<DT>::EPA);
   static constexpr int kKernel = kSoftmaxFwd;
   static constexpr int UNIT = UNIT_;
   using V = V16<DT>;
@@ -910,7 +916,7 @@ struct StreamSoftmaxFwd {
     }
 #pragma unroll
     for (int rr = 0; rr < RPU; ++rr) {
-      if (DT == kBF16) {
+      if constexpr (DT == kBF16 && UNIT_ <= 32) {
         reduce_minmax_bf16<UNIT_>(mn[rr], mx[rr]);
       } else {
         mn[rr] = u.template reduce<kOpMin>(mn[rr]);
@@ -940,7 +946,7 @@ struct StreamSoftmaxFwd {
 
 template <int DT, int UNIT_, int NV>
 struct StreamSoftmaxBwd {
-  static constexpr int kMaxRegs = NV * V16<DT>::EPA >= 32 ? 128 : 80;
+  static constexpr int kMaxRegs = softmax_stream_regs(DT, NV * V16<DT>::EPA);
   static constexpr int kKernel = kSoftmaxBwd;
   static constexpr int UNIT = UNIT_;
   using V = V16<DT>;
@@ -1540,12 +1546,26 @@ cudaError_t launch_softmax_nv(const TilePlan& p, const TileKernelArgs& ka, cudaS
   return cudaErrorInvalidValue;
 }
 
+// Multi-warp units take the long rows: 4 or 8 vectors per lane (16 for binary32 at 8192).
+template <template <int, int, int> class WORK, int DT, int UNIT>
+cudaError_t launch_softmax_wide(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
+  switch (p.iters) {
+    case 4: return launch_work<WORK<DT, UNIT, 4>>(p, ka, st);
+    case 8: return launch_work<WORK<DT, UNIT, 8>>(p, ka, st);
+    case 16:
+      if (DT == kF32 && UNIT == 128) return launch_work<WORK<DT, UNIT, DT == kF32 ? 16 : 8>>(p, ka, st);
+  }
+  return cudaErrorInvalidValue;
+}
+
 template <template <int, int, int> class WORK, int DT>
 cudaError_t launch_softmax_stream(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
   switch (p.unit_lanes) {
     case 8: return launch_softmax_nv<WORK, DT, 8>(p, ka, st);
     case 16: return launch_softmax_nv<WORK, DT, 16>(p, ka, st);
     case 32: return launch_softmax_nv<WORK, DT, 32>(p, ka, st);
+    case 64: return launch_softmax_wide<WORK, DT, 64>(p, ka, st);
+    case 128: return launch_softmax_wide<WORK, DT, 128>(p, ka, st);
   }
   return cudaErrorInvalidValue;
 }
