@@ -185,15 +185,29 @@ size_t s2a_codes_bytes_bits(size_t n_elems, int bits) {
   return (bits == 2 || bits == 4 || bits == 8) ? (n_elems * (size_t)bits + 7) / 8 : 0;
 }
 
-// General code width: 4 goes to the ordinary entry points; 2 and 8 run row at a time.
+// General code width: 4 goes to the ordinary entry points.  At 2 and 8 bits the GELU
+// kernels have a pipelined form for rows of whole 16-byte vectors; everything else, and
+// the rows left over, run row at a time.
 static int run_bits(int kernel, const void* in, void* out, uint8_t* codes, float* meta, size_t n, size_t row_len,
                     int bits, int dt, void* stream) {
   if (bits == 4) return run(kernel, in, out, codes, meta, n, row_len, dt, stream);
   if (bits != 2 && bits != 8) return S2A_ERR_SHAPE;
   int rc = check_args(in, out, codes, meta, n, row_len, dt);
   if (rc != S2A_OK || n == 0) return rc;
-  RowwiseArgs ra{in, out, codes, meta, 0, n / row_len, (uint32_t)row_len};
-  return launch_rowwise(kernel, dt, ra, (cudaStream_t)stream, bits) == cudaSuccess ? S2A_OK : S2A_ERR_CUDA;
+  cudaStream_t st = (cudaStream_t)stream;
+  const uint64_t n_rows = n / row_len;
+  uint64_t done_rows = 0;
+  TilePlan p = plan_tile(kernel, dt, n_rows, (uint32_t)row_len, bits);
+  if (p.tile_rows != 0 && p.n_tiles != 0 && !misaligned(meta, 16)) {
+    TileArgs ta{in, out, codes, meta, (uint32_t)row_len, p.n_tiles};
+    if (launch_tile(kernel, dt, p, ta, st) != cudaSuccess) return S2A_ERR_CUDA;
+    done_rows = p.n_tiles * p.tile_rows;
+  }
+  if (done_rows < n_rows) {
+    RowwiseArgs ra{in, out, codes, meta, done_rows, n_rows - done_rows, (uint32_t)row_len};
+    if (launch_rowwise(kernel, dt, ra, st, bits) != cudaSuccess) return S2A_ERR_CUDA;
+  }
+  return S2A_OK;
 }
 
 int s2a_gelu_fwd_bits(const void* x, void* y, uint8_t* codes, float* meta, size_t n_elems, size_t row_len,

@@ -54,8 +54,8 @@ cudaError_t launch_lrp_fwd(int dt, const void* x, const float* A, const float* B
 
 // ---------------------------------------------------------------- pipelined tiles
 // A tile is `tile_rows` consecutive rows whose flat element span starts and ends on a
-// multiple of 32 elements, so that its data and its code bytes can move with 16-byte
-// bulk copies.  A plan with tile_rows == 0 means "no pipelined path for this shape".
+// multiple of 32 elements (128 / bits in general), so that its data and its code bytes can
+// move with 16-byte bulk copies.  A plan with tile_rows == 0 means "no pipelined path for this shape".
 enum { kVariantGeneric = 0, kVariantStream = 1, kVariantPairFixed = 2 };
 
 struct TilePlan {
@@ -70,6 +70,7 @@ struct TilePlan {
   uint32_t grid;        // CTAs launched
   uint64_t n_tiles;     // full tiles covered; remaining rows go to the row-at-a-time path
   uint32_t overlap_launch;  // 1: launched with programmatic stream serialization
+  uint32_t bits;        // code width of Eq. 8: 4, or 2 / 8 (GELU rows of whole 16-byte vectors)
 };
 
 struct TileArgs {
@@ -82,7 +83,7 @@ struct TileArgs {
 };
 
 // Chooses the launch shape for (kernel, dt, row_len, n_rows) on the current device.
-TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t row_len);
+TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t row_len, int bits = 4);
 cudaError_t launch_tile(int kernel, int dt, const TilePlan& p, const TileArgs& a, cudaStream_t st);
 
 // Reads (and optionally clears) the per-device error word the pipelined kernels set

@@ -14,6 +14,7 @@ cudaError_t launch_tile_softmax_fwd(int dt, const TilePlan& p, const void* kerne
 cudaError_t launch_tile_softmax_bwd(int dt, const TilePlan& p, const void* kernel_args, cudaStream_t st);
 cudaError_t launch_tile_silu_fwd(int dt, const TilePlan& p, const void* kernel_args, cudaStream_t st);
 cudaError_t launch_tile_silu_bwd(int dt, const TilePlan& p, const void* kernel_args, cudaStream_t st);
+cudaError_t launch_tile_bits(int kernel, int dt, const TilePlan& p, const void* kernel_args, cudaStream_t st);
 
 namespace {
 
@@ -63,8 +64,10 @@ unsigned int* error_word_address() {
 // Launch-shape policy.  Environment overrides (for tuning sweeps): S2A_PATH=rowwise
 // disables this path; S2A_UNIT, S2A_TILE_ROWS, S2A_WARPS, S2A_STAGES, S2A_CTAS_PER_SM,
 // S2A_VARIANT=generic, S2A_FIXED=0, S2A_PDL=0.
-TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L) {
+TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
   TilePlan p{};
+  p.bits = (uint32_t)bits;
+  if (bits != 4 && bits != 2 && bits != 8) return p;
   const char* path = getenv("S2A_PATH");
   if (path && path[0] == 'r') return p;
   const char* var = getenv("S2A_VARIANT");
@@ -76,14 +79,22 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L) {
   const bool vec16 = (L % vec) == 0;
   const uint32_t epa = vec16 ? vec : 2u;
   const uint32_t n_acc = vec16 ? L / vec : (L + 1) / 2;  // accesses covering one row
-  // rows per tile: the tile's element count must be a multiple of 32, its row count even
-  uint32_t r_min = 32u / gcd_u32(L, 32u);
+  // rows per tile: the tile's code bytes must be a multiple of 16 (its element count a
+  // multiple of 32 at 4 bits), its row count even
+  const uint32_t epc = 128u / (uint32_t)bits;  // elements per 16 code bytes
+  uint32_t r_min = epc / gcd_u32(L, epc);
   if (r_min < 2) r_min = 2;
   if ((uint64_t)r_min * L * esize > kMaxStageBytes) return p;
 
   uint32_t variant = kVariantGeneric, unit = 0, iters = 0;
   const int env_unit = env_int("S2A_UNIT", 0);
-  if (vec16 && !force_generic && is_gelu) {
+  if (bits != 4) {
+    // other code widths: GELU rows of whole vectors, long enough for a two-warp unit
+    if (!(kernel == kGeluFwd || kernel == kGeluBwd) || !vec16 || n_acc < 128) return p;
+    variant = kVariantStream;
+    unit = (dt == kF32 && n_acc >= 512) ? 128u : 64u;
+    if (env_unit == 64 || env_unit == 128) unit = (uint32_t)env_unit;
+  } else if (vec16 && !force_generic && is_gelu) {
     // streamed: nothing held in registers; a warp per row unless the row is short
     variant = kVariantStream;
     unit = n_acc >= 256 ? 64u : (n_acc >= 32 ? 32u : (n_acc >= 16 ? 16u : 8u));
@@ -166,7 +177,7 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L) {
   if (rows == 0 || rows % r_min != 0 || rows % G != 0 || (uint64_t)rows * L * esize > kMaxStageBytes) return p;
 
   const uint32_t data_bytes = rows * L * esize;
-  const uint32_t code_bytes = rows * L / 2;
+  const uint32_t code_bytes = (uint32_t)((uint64_t)rows * L * (uint32_t)bits / 8);
   const uint32_t meta_bytes = rows * 8;
   const uint32_t code_off = align_up(data_bytes, 128);
   const uint32_t meta_off = code_off + align_up(code_bytes, 128);
@@ -190,7 +201,8 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L) {
   uint32_t stages = 0, smem = 0;
   for (int c = ctas_per_sm; c >= 1 && stages == 0; c /= 2) {
     const uint32_t budget = kMaxSmem / (uint32_t)c - 1024;  // 1 KiB per CTA is the system's
-    uint32_t fit = budget > kHeaderBytes ? (budget - kHeaderBytes) / stage_bytes : 0;
+    const uint32_t fixed = kHeaderBytes + (bits == 8 ? n_units * 1024u : 0u);  // + 256-entry tables
+    uint32_t fit = budget > fixed ? (budget - fixed) / stage_bytes : 0;
     if (fit > 4) fit = 4;
     if (env_stages > 0 && (uint32_t)env_stages <= fit) fit = (uint32_t)env_stages;
     if (fit >= 2) { stages = fit; ctas_per_sm = c; smem = budget; }
@@ -226,12 +238,13 @@ cudaError_t launch_tile(int kernel, int dt, const TilePlan& p, const TileArgs& a
   ka.tile_rows = p.tile_rows;
   const uint32_t esize = dt == kF32 ? 4u : 2u;
   ka.data_bytes = p.tile_rows * a.row_len * esize;
-  ka.code_bytes = p.tile_rows * a.row_len / 2;
+  ka.code_bytes = (uint32_t)((uint64_t)p.tile_rows * a.row_len * p.bits / 8);
   ka.meta_bytes = p.tile_rows * 8;
   ka.code_off = align_up(ka.data_bytes, 128);
   ka.meta_off = ka.code_off + align_up(ka.code_bytes, 128);
   ka.stage_bytes = ka.meta_off + align_up(ka.meta_bytes, 128);
   ka.stages = p.stages;
+  ka.tab_off = p.bits == 8 ? kHeaderBytes + p.stages * ka.stage_bytes : 0u;
   {
     // spreading needs every warp's units to find a group in every round
     const uint32_t upw = p.unit_lanes < 32 ? 32 / p.unit_lanes : 1;
@@ -241,6 +254,7 @@ cudaError_t launch_tile(int kernel, int dt, const TilePlan& p, const TileArgs& a
   }
   ka.error_word = error_word_address();
   if (!ka.error_word) return cudaErrorInvalidDevice;
+  if (p.bits != 4) return launch_tile_bits(kernel, dt, p, &ka, st);
   switch (kernel) {
     case kGeluFwd: return launch_tile_gelu_fwd(dt, p, &ka, st);
     case kGeluBwd: return launch_tile_gelu_bwd(dt, p, &ka, st);

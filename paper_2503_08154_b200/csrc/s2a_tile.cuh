@@ -23,6 +23,8 @@
 #include "s2a_common.cuh"
 #include "s2a_launch.h"
 
+#include <type_traits>
+
 namespace s2a {
 namespace {
 
@@ -54,6 +56,7 @@ struct TileKernelArgs {
   uint32_t stage_bytes;
   uint32_t stages;
   uint32_t spread_units;     // 1: sub-warp units of a warp take groups a fixed stride apart
+  uint32_t tab_off;          // byte offset of the wide derivative tables (8-bit codes), else 0
   unsigned int* error_word;  // device address of the per-device error word
 };
 
@@ -828,6 +831,169 @@ struct StreamActBwd {
 template <int DT, int UNIT_, int NVL> using StreamGeluBwd = StreamActBwd<DT, UNIT_, NVL, kActGelu>;
 template <int DT, int UNIT_, int NVL> using StreamSiluBwd = StreamActBwd<DT, UNIT_, NVL, kActSilu>;
 
+// ---------------------------------------------------------------- Eq. 8 at 2 and 8 bits
+// The streamed GELU kernels for code widths other than 4 (rows of whole 16-byte vectors,
+// units of two or four warps).  A vector of EPA elements owns EPA * NBITS / 8 code bytes.
+template <int N, int NBITS>
+struct CodePackerBits {
+  static constexpr int PER = 32 / NBITS;            // codes per 32-bit word
+  static constexpr int W = (N + PER - 1) / PER;
+  uint32_t acc[W];
+  __device__ __forceinline__ void init() {
+#pragma unroll
+    for (int w = 0; w < W; ++w) {
+      uint32_t ones = 0;
+#pragma unroll
+      for (int k = 0; k < PER; ++k)
+        if (w * PER + k < N) ones |= 1u << (NBITS * k);
+      acc[w] = 0u - kMagicBits * ones;
+    }
+  }
+  __device__ __forceinline__ void add(int k, float v, const QRange& q) {
+    const float t = __fmul_rn(__fsub_rn(v, q.mn), q.inv);
+    acc[k / PER] += __float_as_uint(__fadd_rn(t, 12582912.0f)) << (NBITS * (k % PER));
+  }
+};
+
+template <int DT, int NBITS>
+struct CodeIo {
+  static constexpr int EPA = V16<DT>::EPA;
+  static constexpr int BYTES = EPA * NBITS / 8;     // 1, 2, 4 or 8 code bytes per vector
+  static constexpr int W = (BYTES + 3) / 4;
+  static __device__ __forceinline__ void store(unsigned char* c, uint32_t j, const uint32_t* w) {
+    if (BYTES == 1) c[j] = (unsigned char)w[0];
+    if (BYTES == 2) *(uint16_t*)(c + j * 2u) = (uint16_t)w[0];
+    if (BYTES == 4) *(uint32_t*)(c + j * 4u) = w[0];
+    if (BYTES == 8) *(uint2*)(c + j * 8u) = make_uint2(w[0], w[W - 1]);
+  }
+  static __device__ __forceinline__ void load(const unsigned char* c, uint32_t j, uint32_t* w) {
+    if (BYTES == 1) w[0] = c[j];
+    if (BYTES == 2) w[0] = *(const uint16_t*)(c + j * 2u);
+    if (BYTES == 4) w[0] = *(const uint32_t*)(c + j * 4u);
+    if (BYTES == 8) {
+      const uint2 t = *(const uint2*)(c + j * 8u);
+      w[0] = t.x;
+      w[W - 1] = t.y;
+    }
+  }
+};
+
+template <int DT, int UNIT_, int ACT, int NBITS>
+struct StreamActFwdBits {
+  static_assert(UNIT_ >= 64 && (NBITS == 2 || NBITS == 8), "multi-warp units, 2 or 8 bits");
+  static constexpr int kMaxRegs = 64;
+  static constexpr int kKernel = ACT == kActGelu ? kGeluFwd : kSiluFwd;
+  static constexpr float kActClip = Act<ACT>::kClipOf;
+  static constexpr int UNIT = UNIT_;
+  using V = V16<DT>;
+  using C = CodeIo<DT, NBITS>;
+  struct State {};
+  static __device__ __forceinline__ void init(State&) {}
+  static __device__ __forceinline__ uint32_t rows_per_group(uint32_t) { return 1u; }
+
+  static __device__ __forceinline__ void group(Unit<UNIT_>& u, State&, const StagePtrs& p, float*, uint32_t r,
+                                               bool active, uint32_t L) {
+    if (!active) return;  // whole warps leave together
+    const uint32_t nv = L / V::EPA;
+    unsigned char* row = p.data + (size_t)r * L * Io<DT>::kBytes;
+    unsigned char* crow = p.codes + (size_t)r * (L / V::EPA) * C::BYTES;
+    typename V::MinMax mm;
+    mm.init();
+#pragma unroll 4
+    for (uint32_t j = u.ul; j < nv; j += UNIT_) mm.add(*(const typename V::Raw*)(row + j * 16u));
+    const float mn = u.template reduce<kOpMin>(mm.lo());
+    const float mx = u.template reduce<kOpMax>(mm.hi());
+    const QRange q = make_qrange(fminf(fmaxf(mn, -kActClip), kActClip), fminf(fmaxf(mx, -kActClip), kActClip),
+                                 (float)((1 << NBITS) - 1));
+    if (u.ul == 0) { p.meta[2 * r] = q.mn; p.meta[2 * r + 1] = q.s; }
+#pragma unroll 2
+    for (uint32_t j = u.ul; j < nv; j += UNIT_) {
+      float v[V::EPA];
+      V::widen(*(const typename V::Raw*)(row + j * 16u), v);
+      CodePackerBits<V::EPA, NBITS> pk;
+      pk.init();
+#pragma unroll
+      for (int k = 0; k < V::EPA; ++k) {
+        pk.add(k, fminf(fmaxf(v[k], -kActClip), kActClip), q);
+        v[k] = gelu_eval<DT, ACT>(v[k]);
+      }
+      *(typename V::Raw*)(row + j * 16u) = V::narrow(v);
+      C::store(crow, j, pk.acc);
+    }
+  }
+};
+
+// Backward: the 2^NBITS derivative values of a row.  Four values sit one per lane (eight
+// times over) and are fetched with a shuffle; 256 values go to a table of the unit's own
+// in shared memory.  Either is kept while (min, s) repeat from row to row.
+template <int DT, int UNIT_, int ACT, int NBITS>
+struct StreamActBwdBits {
+  static_assert(UNIT_ >= 64 && (NBITS == 2 || NBITS == 8), "multi-warp units, 2 or 8 bits");
+  static constexpr int kMaxRegs = 64;
+  static constexpr int kKernel = ACT == kActGelu ? kGeluBwd : kSiluBwd;
+  static constexpr int UNIT = UNIT_;
+  static constexpr int kTabFloats = NBITS == 8 ? 256 : 16;
+  using V = V16<DT>;
+  using C = CodeIo<DT, NBITS>;
+  struct State {
+    float tab_mn, tab_s, d;
+  };
+  static __device__ __forceinline__ void init(State& st) {
+    st.tab_mn = __int_as_float(0x7fc00000);  // NaN: nothing cached yet
+    st.tab_s = st.tab_mn;
+    st.d = 0.0f;
+  }
+  static __device__ __forceinline__ uint32_t rows_per_group(uint32_t) { return 1u; }
+
+  static __device__ __forceinline__ void group(Unit<UNIT_>& u, State& st, const StagePtrs& p, float* tab,
+                                               uint32_t r, bool active, uint32_t L) {
+    if (!active) return;  // whole warps leave together
+    const float mn = p.meta[2 * r];
+    const float s = p.meta[2 * r + 1];
+    if (mn != st.tab_mn || s != st.tab_s) {  // the same decision in every lane of the unit
+      if (NBITS == 2) {
+        st.d = (float)act_derivative<ACT>((uint32_t)(u.ul & 3), mn, s);
+      } else {
+        u.sync();  // the previous row's reads of the table are over
+        for (int c = u.ul; c < 256; c += UNIT_) tab[c] = (float)act_derivative<ACT>((uint32_t)c, mn, s);
+        u.sync();
+      }
+      st.tab_mn = mn;
+      st.tab_s = s;
+    }
+    const uint32_t nv = L / V::EPA;
+    unsigned char* row = p.data + (size_t)r * L * Io<DT>::kBytes;
+    const unsigned char* crow = p.codes + (size_t)r * (L / V::EPA) * C::BYTES;
+    // every lane runs the same number of rounds so that the shuffles stay warp-wide
+    const uint32_t rounds = (nv + UNIT_ - 1) / UNIT_;
+#pragma unroll 2
+    for (uint32_t it = 0; it < rounds; ++it) {
+      const uint32_t j = it * UNIT_ + u.ul;
+      const bool ok = j < nv;
+      float v[V::EPA];
+      uint32_t w[C::W] = {};
+      if (ok) {
+        V::widen(*(const typename V::Raw*)(row + j * 16u), v);
+        C::load(crow, j, w);
+      }
+#pragma unroll
+      for (int k = 0; k < V::EPA; ++k) {
+        constexpr int PER = 32 / NBITS;
+        const uint32_t code = w[k / PER] >> (NBITS * (k % PER));
+        float d;
+        if (NBITS == 2) d = __shfl_sync(0xffffffffu, st.d, (int)code);  // lane = code mod 4 (+4, +8, ...)
+        else d = tab[code & 0xFFu];
+        v[k] *= d;
+      }
+      if (ok) *(typename V::Raw*)(row + j * 16u) = V::narrow(v);
+    }
+  }
+};
+
+// Floats of derivative table a policy wants per unit (16 unless it says otherwise).
+template <class W, class = void> struct TabFloats { static constexpr int value = 16; };
+template <class W> struct TabFloats<W, std::void_t<decltype(W::kTabFloats)>> { static constexpr int value = W::kTabFloats; };
+
 // Register cap of the streamed softmax kernels by elements held per lane (the planner
 // derives the CTAs that fit an SM from the same number).
 constexpr int softmax_stream_regs(int dt, int held) {
@@ -1432,7 +1598,8 @@ __global__ void __maxnreg__(WORK::kMaxRegs) tile_kernel(TileKernelArgs a) {
   u.phase = 0;
   const uint32_t n_units = (uint32_t)(n_cwarps * 32 / UNIT);
   int* abort_flag = (int*)(smem + kFlagOffset) + (UNIT > 32 ? u.uid : 0);
-  float* tab = (float*)(smem + kTabOffset) + u.uid * 16;
+  float* tab = TabFloats<WORK>::value == 16 ? (float*)(smem + kTabOffset) + u.uid * 16
+                                            : (float*)(smem + a.tab_off) + u.uid * TabFloats<WORK>::value;
   typename WORK::State state;
   WORK::init(state);
 
@@ -1625,6 +1792,27 @@ cudaError_t launch_variant(const TilePlan& p, const TileKernelArgs& ka, cudaStre
     return cudaErrorInvalidValue;
   }
   return launch_generic<KERNEL, DT>(p, ka, st);
+}
+
+// The 2- and 8-bit GELU kernels (their own translation unit instantiates this).
+template <int KERNEL, int DT, int NBITS>
+cudaError_t launch_bits_unit(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
+  if constexpr (KERNEL == kGeluFwd) {
+    if (p.unit_lanes == 64) return launch_work<StreamActFwdBits<DT, 64, kActGelu, NBITS>>(p, ka, st);
+    if (p.unit_lanes == 128) return launch_work<StreamActFwdBits<DT, 128, kActGelu, NBITS>>(p, ka, st);
+  } else {
+    if (p.unit_lanes == 64) return launch_work<StreamActBwdBits<DT, 64, kActGelu, NBITS>>(p, ka, st);
+    if (p.unit_lanes == 128) return launch_work<StreamActBwdBits<DT, 128, kActGelu, NBITS>>(p, ka, st);
+  }
+  return cudaErrorInvalidValue;
+}
+template <int KERNEL>
+cudaError_t launch_tile_bits_kernel(int dt, const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
+  if (p.bits == 2)
+    return dt == kF32 ? launch_bits_unit<KERNEL, kF32, 2>(p, ka, st) : launch_bits_unit<KERNEL, kBF16, 2>(p, ka, st);
+  if (p.bits == 8)
+    return dt == kF32 ? launch_bits_unit<KERNEL, kF32, 8>(p, ka, st) : launch_bits_unit<KERNEL, kBF16, 8>(p, ka, st);
+  return cudaErrorInvalidValue;
 }
 
 // One translation unit per entry point instantiates this.

@@ -273,12 +273,17 @@ def test_silu(rows, L, dt):
 @pytest.mark.parametrize("dt", [F32, BF16])
 @pytest.mark.parametrize("bits", [2, 4, 8])
 @pytest.mark.parametrize("kind,rows,L", [("gelu", 7, 3), ("gelu", 41, 197), ("gelu", 24, 3072), ("gelu", 5, 1),
+                                         ("gelu", 1237, 4096), ("gelu", 77, 1024), ("gelu", 311, 5120),
+                                         ("gelu", 13, 8192), ("gelu_narrow", 2001, 3072), ("gelu_narrow", 90, 2048),
                                          ("softmax", 9, 65), ("softmax", 300, 197), ("softmax", 12, 1024),
                                          ("softmax", 3, 2), ("softmax", 131, 257)])
 def test_other_bit_widths(kind, rows, L, bits, dt):
+    # "gelu_narrow": rows that do not reach the clip, so that every row has its own (min, s)
+    # and the backward's derivative table is rebuilt row after row
     n = rows * L
-    if kind == "gelu":
-        x, g = _gelu_inputs(rows, L, dt, seed=20 + bits)
+    if kind.startswith("gelu"):
+        x, g = _gelu_inputs(rows, L, dt, seed=20 + bits, scale=0.3 if kind == "gelu_narrow" else 1.3)
+        kind = "gelu"
     else:
         x, g = _softmax_inputs(rows, L, dt, seed=20 + bits)
     y_o, codes_o, meta_o = o.fwd_bits(kind, x, L, bits, dt)
