@@ -71,6 +71,15 @@ __global__ void __launch_bounds__(kThreads) cap_bwd_kernel(const void* gv, void*
   const T* g = (const T*)gv;
   T* out = (T*)ov;
   const uint64_t stride = (uint64_t)gridDim.x * kThreads;
+  if (R8 && DT == kF32) {
+    // one 16-byte store per thread, neighbours in a warp next to each other: thread q
+    // writes one half of group q / 2
+    for (uint64_t q = (uint64_t)blockIdx.x * kThreads + threadIdx.x; q < 2 * n_out; q += stride) {
+      const float v = Io<DT>::widen(g[q >> 1]) * 0.125f;
+      ((float4*)ov)[q] = make_float4(v, v, v, v);
+    }
+    return;
+  }
   for (uint64_t i = (uint64_t)blockIdx.x * kThreads + threadIdx.x; i < n_out; i += stride) {
     const float gi = Io<DT>::widen(g[i]);
     if (R8) {
@@ -89,16 +98,19 @@ __global__ void __launch_bounds__(kThreads) cap_bwd_kernel(const void* gv, void*
   }
 }
 
-// ---- LRP forward: y[b, t, c] = x[b, t, c] + sum_k A[t, k] B[k, c].  A thread owns 8
-// consecutive channels of one token: it forms its 8 prompt values once (binary32, k in
-// order) and then streams over its share of the batch.  VEC = false is the scalar form
-// for channel counts that are not a multiple of 8.
+// ---- LRP forward: y[b, t, c] = x[b, t, c] + sum_k A[t, k] B[k, c].  A thread owns the W
+// consecutive channels of one token that fill 16 bytes: it forms its W prompt values once
+// (binary32, k in order) and then streams over its share of the batch, four samples in
+// flight at a time (y may alias x, but only element for element, so a thread's loads may
+// run ahead of its own stores).  VEC = false is the scalar form for channel counts that are
+// not a multiple of W.
 template <int DT, bool VEC>
 __global__ void __launch_bounds__(kThreads) lrp_fwd_kernel(const void* xv, const float* A, const float* B, void* yv,
                                                            uint32_t batch, uint32_t tokens, uint32_t channels,
                                                            uint32_t rank) {
   using T = typename Io<DT>::T;
-  constexpr int W = VEC ? 8 : 1;
+  constexpr int W = VEC ? (DT == kBF16 ? 8 : 4) : 1;
+  constexpr int kAhead = 4;
   const uint32_t cgroups = channels / W;
   const uint64_t items = (uint64_t)tokens * cgroups;
   const uint64_t item = (uint64_t)blockIdx.x * kThreads + threadIdx.x;
@@ -109,29 +121,54 @@ __global__ void __launch_bounds__(kThreads) lrp_fwd_kernel(const void* xv, const
   for (int w = 0; w < W; ++w) p[w] = 0.0f;
   for (uint32_t k = 0; k < rank; ++k) {
     const float a = A[(uint64_t)t * rank + k];
+    if (VEC) {  // B is 16-byte aligned here and c0 a multiple of 4: whole float4 loads
+      const float4* brow = (const float4*)(B + (uint64_t)k * channels + c0);
 #pragma unroll
-    for (int w = 0; w < W; ++w) p[w] = fmaf(a, B[(uint64_t)k * channels + c0 + w], p[w]);
-  }
-  const uint64_t sample = (uint64_t)tokens * channels;
-  for (uint32_t b = blockIdx.y; b < batch; b += gridDim.y) {
-    const uint64_t e = (uint64_t)b * sample + (uint64_t)t * channels + c0;
-    if (VEC) {
-      float v[8];
-      if (DT == kBF16) {
-        widen8(*(const uint4*)((const T*)xv + e), v);
-      } else {
-        const float4 a = *(const float4*)((const T*)xv + e), b2 = *(const float4*)((const T*)xv + e + 4);
-        v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b2.x; v[5] = b2.y; v[6] = b2.z; v[7] = b2.w;
-      }
-#pragma unroll
-      for (int w = 0; w < 8; ++w) v[w] += p[w];
-      if (DT == kBF16) {
-        *(uint4*)((T*)yv + e) = narrow8(v);
-      } else {
-        *(float4*)((T*)yv + e) = make_float4(v[0], v[1], v[2], v[3]);
-        *(float4*)((T*)yv + e + 4) = make_float4(v[4], v[5], v[6], v[7]);
+      for (int h = 0; h < W / 4; ++h) {
+        const float4 bv = brow[h];
+        p[4 * h] = fmaf(a, bv.x, p[4 * h]);
+        p[(4 * h + 1) % W] = fmaf(a, bv.y, p[(4 * h + 1) % W]);
+        p[(4 * h + 2) % W] = fmaf(a, bv.z, p[(4 * h + 2) % W]);
+        p[(4 * h + 3) % W] = fmaf(a, bv.w, p[(4 * h + 3) % W]);
       }
     } else {
+#pragma unroll
+      for (int w = 0; w < W; ++w) p[w] = fmaf(a, B[(uint64_t)k * channels + c0 + w], p[w]);
+    }
+  }
+  const uint64_t sample = (uint64_t)tokens * channels;
+  const uint64_t e0 = (uint64_t)t * channels + c0;
+  if (VEC) {
+    const uint4* xin = (const uint4*)((const T*)xv + e0);
+    uint4* yout = (uint4*)((T*)yv + e0);
+    const uint64_t step = sample * sizeof(T) / 16;  // one sample, in 16-byte units
+    for (uint32_t b = blockIdx.y; b < batch; b += gridDim.y * kAhead) {
+      uint4 raw[kAhead];
+#pragma unroll
+      for (int j = 0; j < kAhead; ++j) {
+        const uint32_t bj = b + j * gridDim.y;
+        if (bj < batch) raw[j] = xin[bj * step];
+      }
+#pragma unroll
+      for (int j = 0; j < kAhead; ++j) {
+        const uint32_t bj = b + j * gridDim.y;
+        if (bj >= batch) continue;
+        if (DT == kBF16) {
+          float v[8];
+          widen8(raw[j], v);
+#pragma unroll
+          for (int w = 0; w < W; ++w) v[w] += p[w];
+          yout[bj * step] = narrow8(v);
+        } else {
+          float4 v = *(float4*)&raw[j];
+          v.x += p[0]; v.y += p[1 % W]; v.z += p[2 % W]; v.w += p[3 % W];
+          yout[bj * step] = *(uint4*)&v;
+        }
+      }
+    }
+  } else {
+    for (uint32_t b = blockIdx.y; b < batch; b += gridDim.y) {
+      const uint64_t e = (uint64_t)b * sample + e0;
       ((T*)yv)[e] = Io<DT>::narrow(Io<DT>::widen(((const T*)xv)[e]) + p[0]);
     }
   }
@@ -161,11 +198,13 @@ cudaError_t launch_cap(bool fwd, int dt, const void* in, void* out, uint64_t n_o
 cudaError_t launch_lrp_fwd(int dt, const void* x, const float* A, const float* B, void* y, uint32_t batch,
                            uint32_t tokens, uint32_t channels, uint32_t rank, cudaStream_t st) {
   if ((uint64_t)batch * tokens * channels == 0) return cudaSuccess;
-  const bool vec = channels % 8 == 0;
-  const uint64_t items = (uint64_t)tokens * (vec ? channels / 8 : channels);
-  // enough threads to fill the machine: the batch is split over gridDim.y (each split forms
-  // its prompt values again, 30 multiply-adds per element of one sample)
-  uint64_t splits = (148ull * 2048 + items - 1) / items;
+  const uint32_t w = dt == kF32 ? 4u : 8u;  // channels in 16 bytes
+  const bool vec = channels % w == 0 && ((uintptr_t)B & 15u) == 0;  // the vector form reads B 16 bytes at a time
+  const uint64_t items = (uint64_t)tokens * (vec ? channels / w : channels);
+  // The batch is split over gridDim.y.  Each split forms its prompt values again (rank
+  // multiply-adds per element of one sample), so only as many splits as give every SM a
+  // thousand threads: with four samples in flight per thread that covers the memory latency.
+  uint64_t splits = (148ull * 1024 + items - 1) / items;
   if (splits > batch) splits = batch;
   if (splits > 64) splits = 64;
   if (splits < 1) splits = 1;
