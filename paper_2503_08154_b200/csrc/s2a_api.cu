@@ -248,7 +248,7 @@ int s2a_describe_plan(int kernel, size_t n_elems, size_t row_len, int dt, char* 
     snprintf(out, cap,
              "tile variant=%s rows/tile=%u unit=%u vec=%u iters=%u warps=%u stages=%u smem=%u grid=%u "
              "tiles=%llu tail_rows=%llu",
-             p.variant == kVariantStream ? "stream" : (p.variant == kVariantPairFixed ? "pair-fixed" : "generic"),
+             p.variant == kVariantStream ? "stream" : (p.variant == kVariantPairFixed ? "pair-fixed" : (p.variant == kVariantAny ? "any-length" : "generic")),
              p.tile_rows, p.unit_lanes, p.vec_elems, p.iters, p.warps, p.stages, p.smem_bytes,
              p.grid, (unsigned long long)p.n_tiles,
              (unsigned long long)(n_rows - p.n_tiles * p.tile_rows));

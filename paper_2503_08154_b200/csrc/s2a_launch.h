@@ -56,11 +56,11 @@ cudaError_t launch_lrp_fwd(int dt, const void* x, const float* A, const float* B
 // A tile is `tile_rows` consecutive rows whose flat element span starts and ends on a
 // multiple of 32 elements (128 / bits in general), so that its data and its code bytes can
 // move with 16-byte bulk copies.  A plan with tile_rows == 0 means "no pipelined path for this shape".
-enum { kVariantGeneric = 0, kVariantStream = 1, kVariantPairFixed = 2 };
+enum { kVariantGeneric = 0, kVariantStream = 1, kVariantPairFixed = 2, kVariantAny = 3 };
 
 struct TilePlan {
   uint32_t tile_rows;   // rows per tile (0: not applicable)
-  uint32_t variant;     // kVariantGeneric / kVariantStream / kVariantPairFixed
+  uint32_t variant;     // kVariantGeneric / kVariantStream / kVariantPairFixed / kVariantAny
   uint32_t unit_lanes;  // lanes that cooperate on one row: 8, 16, 32 or 128
   uint32_t vec_elems;   // elements per shared-memory access: 2 (pair mode) or 16 bytes' worth
   uint32_t iters;       // accesses per lane per row kept in registers (0: streamed)

@@ -18,7 +18,8 @@ cudaError_t launch_tile_bits(int kernel, int dt, const TilePlan& p, const void* 
 
 namespace {
 
-constexpr uint32_t kMaxStageBytes = 56 * 1024;
+constexpr uint32_t kMaxStageBytes = 56 * 1024;   // tiles are not grown beyond this
+constexpr uint32_t kHardStageBytes = 96 * 1024;  // the smallest legal tile may be this large (one CTA per SM then)
 
 int env_int(const char* name, int dflt) {
   const char* v = getenv(name);
@@ -63,7 +64,7 @@ unsigned int* error_word_address() {
 
 // Launch-shape policy.  Environment overrides (for tuning sweeps): S2A_PATH=rowwise
 // disables this path; S2A_UNIT, S2A_TILE_ROWS, S2A_WARPS, S2A_STAGES, S2A_CTAS_PER_SM,
-// S2A_VARIANT=generic, S2A_FIXED=0, S2A_PDL=0.
+// S2A_VARIANT=generic|any, S2A_FIXED=0, S2A_PDL=0.
 TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
   TilePlan p{};
   p.bits = (uint32_t)bits;
@@ -84,7 +85,7 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
   const uint32_t epc = 128u / (uint32_t)bits;  // elements per 16 code bytes
   uint32_t r_min = epc / gcd_u32(L, epc);
   if (r_min < 2) r_min = 2;
-  if ((uint64_t)r_min * L * esize > kMaxStageBytes) return p;
+  if ((uint64_t)r_min * L * esize > kHardStageBytes) return p;
 
   uint32_t variant = kVariantGeneric, unit = 0, iters = 0;
   const int env_unit = env_int("S2A_UNIT", 0);
@@ -126,6 +127,23 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
     unit = 8;
     iters = (n_acc + 7) / 8;
   }
+  const bool force_any = var && var[0] == 'a';
+  if (!is_gelu && bits == 4 && !force_generic && L >= 16 &&
+      (force_any || variant == kVariantGeneric || (variant == kVariantStream && unit == 0))) {
+    // softmax rows of any other length (not whole vectors, or too long for registers):
+    // aligned vectors with masked ends, streamed from shared memory.  A lane should walk
+    // about 4 to 8 vectors per phase (measured: fewer and the row reductions dominate, more
+    // and too few rows are in flight), so short rows get units of 1, 2 or 4 lanes.
+    variant = kVariantAny;
+    const uint32_t nvr = (L + vec - 1) / vec + 1;  // vectors a row can touch
+    unit = 1;
+    while (unit < 16 && (nvr + unit - 1) / unit > 8) unit *= 2;
+    while (unit < 128 && (nvr + unit - 1) / unit > 16) unit *= 2;  // whole warps only for very long rows
+    if (env_unit == 1 || env_unit == 2 || env_unit == 4 || env_unit == 8 || env_unit == 16 || env_unit == 32 ||
+        env_unit == 64 || env_unit == 128)
+      unit = (uint32_t)env_unit;
+    iters = 0;
+  }
   if (variant == kVariantGeneric && is_silu) return p;  // SiLU has the streamed form only
   if (variant == kVariantGeneric) {
     // general register-resident form: pair accesses with 8 or 32 lanes per row, or 16-byte
@@ -145,6 +163,11 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
   }
 
   uint32_t warps = unit == 128 ? 8u : 4u;
+  if (variant == kVariantAny) {
+    // eight consumer warps, four when that many sub-warp units would need a tile beyond 40 KB
+    const uint32_t want = (256u / unit) * ((L & 1u) ? 2u : 1u);  // rows that keep eight warps busy
+    warps = (want > r_min && (uint64_t)want * L * esize > 40 * 1024) ? 4u : 8u;
+  }
   if (variant == kVariantStream && !is_gelu) {
     // A softmax row is a chain of dependent phases (reduce, evaluate, reduce, ...).  With few
     // elements per lane, or the cheaper bfloat16 arithmetic, four warps leave the SM waiting
@@ -174,7 +197,7 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
     while (rows % (n_units * G) != 0 && (uint64_t)(rows + r_min) * L * esize <= kMaxStageBytes) rows += r_min;
   }
   rows = (uint32_t)env_int("S2A_TILE_ROWS", (int)rows);
-  if (rows == 0 || rows % r_min != 0 || rows % G != 0 || (uint64_t)rows * L * esize > kMaxStageBytes) return p;
+  if (rows == 0 || rows % r_min != 0 || rows % G != 0 || (uint64_t)rows * L * esize > kHardStageBytes) return p;
 
   const uint32_t data_bytes = rows * L * esize;
   const uint32_t code_bytes = (uint32_t)((uint64_t)rows * L * (uint32_t)bits / 8);
@@ -195,6 +218,7 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
     uint32_t regs = 128;
     if (variant == kVariantStream) regs = is_gelu ? 64u : (uint32_t)softmax_stream_regs(dt, (int)(iters * epa));
     if (variant == kVariantPairFixed) regs = 96;
+    if (variant == kVariantAny) regs = 80;
     while (ctas_per_sm > 1 && (uint64_t)regs * (warps + 1) * 32 * (uint32_t)ctas_per_sm > 65536) ctas_per_sm /= 2;
   }
   const int env_stages = env_int("S2A_STAGES", 0);

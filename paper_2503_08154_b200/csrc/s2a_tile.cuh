@@ -1157,6 +1157,234 @@ struct StreamSoftmaxBwd {
   }
 };
 
+// ---------------------------------------------------------------- softmax rows of any length
+// Rows that are not a whole number of 16-byte vectors (attention widths such as 49, 145,
+// 198, 577, 1025) or too long to hold in registers.  The tile is still read in ALIGNED
+// 16-byte vectors: a row's first and last vector may hold elements of its neighbours, which
+// are masked out of the arithmetic and never written (interior vectors leave with one
+// 16-byte store, boundary vectors element by element, so two units never write the same
+// bytes).  Nothing is held in registers: the row is streamed from shared memory once per
+// phase, and the exponentials are evaluated twice (sum, then output) rather than kept in a
+// narrower type.  With an odd row length two consecutive rows share a code byte; one unit
+// takes both, in order, and the second merges its nibble into the byte the first one left.
+template <int DT>
+struct AnyRow {
+  using V = V16<DT>;
+  static constexpr int EPA = V::EPA;
+  static constexpr uint32_t kFull = (1u << EPA) - 1u;
+  uint32_t v0, v1;    // first and last vector (tile-relative) that hold elements of the row
+  uint32_t head;      // elements of v0 before the row
+  uint32_t tail;      // elements of v1 inside the row (1..EPA)
+  __device__ __forceinline__ void set(uint32_t r, uint32_t L) {
+    const uint32_t e0 = r * L;
+    v0 = e0 / EPA;
+    v1 = (e0 + L - 1) / EPA;
+    head = e0 - v0 * EPA;
+    tail = e0 + L - v1 * EPA;
+  }
+  __device__ __forceinline__ uint32_t mask(uint32_t j) const {
+    uint32_t m = kFull;
+    if (j == v0) m &= kFull << head;
+    if (j == v1) m &= (1u << tail) - 1u;
+    return m;
+  }
+  // Writes the elements of vector j named by msk (raw: the vector's 16 bytes).
+  static __device__ __forceinline__ void store(unsigned char* data, uint32_t j, const typename V::Raw& raw, uint32_t msk) {
+    if (msk == kFull) {
+      *(typename V::Raw*)(data + j * 16u) = raw;
+      return;
+    }
+    const uint32_t* w = (const uint32_t*)&raw;
+#pragma unroll
+    for (int k = 0; k < EPA; ++k) {
+      if (msk >> k & 1u) {
+        if (DT == kBF16) *(uint16_t*)(data + j * 16u + 2 * k) = (uint16_t)(w[k >> 1] >> (16 * (k & 1)));
+        else *(uint32_t*)(data + j * 16u + 4 * k) = w[k];
+      }
+    }
+  }
+};
+
+// Calls f(j, mask, is_interior) for the vectors of a row that this lane owns: the interior
+// vectors go round the unit's lanes with no mask at all; the first and the last vector of
+// the row (the only ones that can hold a neighbour's elements) are taken by lanes 0 and 1
+// in ONE divergent section, so that the masked code runs once per phase.
+template <int DT, int UNIT_, class F>
+__device__ __forceinline__ void any_row_vectors(const AnyRow<DT>& g, int ul, bool active, F&& f) {
+  if (!active) return;
+  for (uint32_t j = g.v0 + 1u + (uint32_t)ul; j < g.v1; j += UNIT_) f(j, AnyRow<DT>::kFull, std::true_type{});
+  if (UNIT_ == 1) {
+    f(g.v0, g.mask(g.v0), std::false_type{});
+    if (g.v1 != g.v0) f(g.v1, g.mask(g.v1), std::false_type{});
+  } else if (ul == 0 || (ul == 1 && g.v1 != g.v0)) {
+    const uint32_t j = ul == 0 ? g.v0 : g.v1;
+    f(j, g.mask(j), std::false_type{});
+  }
+}
+
+template <int DT, int UNIT_>
+struct AnySoftmaxFwd {
+  static constexpr int kMaxRegs = 80;  // 2 CTAs of 8 + 1 warps per SM
+  static constexpr int kKernel = kSoftmaxFwd;
+  static constexpr int UNIT = UNIT_;
+  using V = V16<DT>;
+  using R = AnyRow<DT>;
+  static constexpr int EPA = V::EPA;
+  struct State {};
+  static __device__ __forceinline__ void init(State&) {}
+  static __device__ __forceinline__ uint32_t rows_per_group(uint32_t L) { return (L & 1u) ? 2u : 1u; }
+
+  static __device__ __forceinline__ float ex(float x, float m, float nm) {
+    constexpr float kLog2e = 1.4426950408889634f;
+    return DT == kBF16 ? ex2_approx(fmaf(x, kLog2e, nm)) : exp_eval<DT>(x - m);
+  }
+
+  static __device__ __forceinline__ void row(Unit<UNIT_>& u, const StagePtrs& p, uint32_t r, bool active, uint32_t L) {
+    R g;
+    g.set(r, L);
+    const int ul = u.ul;
+    // ---- row maximum (interior vectors of bfloat16 rows: packed maxima on the raw words)
+    float m = -INFINITY;
+    typename V::MinMax pm;
+    pm.init();
+    any_row_vectors<DT, UNIT_>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
+      const typename V::Raw raw = *(const typename V::Raw*)(p.data + j * 16u);
+      if constexpr (decltype(interior)::value) {
+        pm.add(raw);
+      } else {
+        float v[EPA];
+        V::widen(raw, v);
+#pragma unroll
+        for (int k = 0; k < EPA; ++k) m = fmaxf(m, (msk >> k & 1u) ? v[k] : -INFINITY);
+      }
+    });
+    m = u.template reduce<kOpMax>(fmaxf(m, pm.hi()));
+    if (!active) m = 0.0f;
+    const float nm = -m * 1.4426950408889634f;
+    // ---- sum of exponentials
+    float z = 0.0f;
+    any_row_vectors<DT, UNIT_>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
+      float v[EPA];
+      V::widen(*(const typename V::Raw*)(p.data + j * 16u), v);
+#pragma unroll
+      for (int k = 0; k < EPA; ++k) {
+        const float e = ex(v[k], m, nm);
+        if constexpr (decltype(interior)::value) z += e;
+        else z += (msk >> k & 1u) ? e : 0.0f;
+      }
+    });
+    z = u.template reduce<kOpSum>(z);
+    const float rz = __fdiv_rn(1.0f, active ? z : 1.0f);
+    // ---- y, written in place, and the range of y as written
+    float mn = INFINITY, mx = -INFINITY;
+    typename V::MinMax py;
+    py.init();
+    any_row_vectors<DT, UNIT_>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
+      float v[EPA];
+      V::widen(*(const typename V::Raw*)(p.data + j * 16u), v);
+#pragma unroll
+      for (int k = 0; k < EPA; ++k) v[k] = ex(v[k], m, nm) * rz;
+      const typename V::Raw yw = V::narrow(v);  // v now holds y as written
+      if constexpr (decltype(interior)::value) {
+        *(typename V::Raw*)(p.data + j * 16u) = yw;
+        py.add(yw);
+      } else {
+        R::store(p.data, j, yw, msk);
+#pragma unroll
+        for (int k = 0; k < EPA; ++k) {
+          mn = fminf(mn, (msk >> k & 1u) ? v[k] : INFINITY);
+          mx = fmaxf(mx, (msk >> k & 1u) ? v[k] : -INFINITY);
+        }
+      }
+    });
+    mn = u.template reduce<kOpMin>(fminf(mn, py.lo()));
+    mx = u.template reduce<kOpMax>(fmaxf(mx, py.hi()));
+    const QRange q = make_qrange(mn, mx);
+    if (active && ul == 0) { p.meta[2 * r] = q.mn; p.meta[2 * r + 1] = q.s; }
+    // ---- codes of y as written (each lane reads back the vectors it wrote itself)
+    any_row_vectors<DT, UNIT_>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
+      float v[EPA];
+      V::widen(*(const typename V::Raw*)(p.data + j * 16u), v);
+      CodePacker<EPA> pk;
+      pk.init();
+      if constexpr (decltype(interior)::value) {
+#pragma unroll
+        for (int k = 0; k < EPA; ++k) pk.add(k, v[k], q);
+        V::store_codes(p.codes, j, pk.acc);
+      } else {
+#pragma unroll
+        for (int k = 0; k < EPA; ++k) pk.add(k, (msk >> k & 1u) ? v[k] : q.mn, q);  // a neighbour's element codes as 0
+        unsigned char* cb = p.codes + j * (EPA / 2);
+#pragma unroll
+        for (int b = 0; b < EPA / 2; ++b) {
+          const uint32_t pmk = (msk >> (2 * b)) & 3u;
+          const uint32_t byte = (pk.acc >> (8 * b)) & 0xFFu;
+          if (pmk == 3u) cb[b] = (unsigned char)byte;
+          else if (pmk == 1u) cb[b] = (unsigned char)(byte & 0x0Fu);                  // the high nibble is the next row's
+          else if (pmk == 2u) cb[b] = (unsigned char)((cb[b] & 0x0Fu) | (byte & 0xF0u));  // the low nibble is the previous row's
+        }
+      }
+    });
+  }
+
+  static __device__ __forceinline__ void group(Unit<UNIT_>& u, State&, const StagePtrs& p, float*, uint32_t grp,
+                                               bool active, uint32_t L) {
+    if (UNIT_ >= 32 && !active) return;  // whole warps (and whole multi-warp units) leave together
+    const uint32_t G = rows_per_group(L);
+    for (uint32_t h = 0; h < G; ++h) {
+      row(u, p, active ? grp * G + h : 0u, active, L);
+      u.sync();  // the next row of the pair reads the code byte this one left
+    }
+  }
+};
+
+template <int DT, int UNIT_>
+struct AnySoftmaxBwd {
+  static constexpr int kMaxRegs = 80;
+  static constexpr int kKernel = kSoftmaxBwd;
+  static constexpr int UNIT = UNIT_;
+  using V = V16<DT>;
+  using R = AnyRow<DT>;
+  static constexpr int EPA = V::EPA;
+  struct State {};
+  static __device__ __forceinline__ void init(State&) {}
+  static __device__ __forceinline__ uint32_t rows_per_group(uint32_t) { return 1u; }  // codes are only read
+
+  static __device__ __forceinline__ void group(Unit<UNIT_>& u, State&, const StagePtrs& p, float*, uint32_t r,
+                                               bool active, uint32_t L) {
+    if (UNIT_ >= 32 && !active) return;
+    R g;
+    g.set(active ? r : 0u, L);
+    const int ul = u.ul;
+    const float mn = active ? p.meta[2 * r] : 0.0f;
+    const float s = active ? p.meta[2 * r + 1] : 0.0f;
+    float dot = 0.0f;
+    any_row_vectors<DT, UNIT_>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
+      float v[EPA];
+      V::widen(*(const typename V::Raw*)(p.data + j * 16u), v);
+      const uint32_t bits = V::load_codes(p.codes, j);
+#pragma unroll
+      for (int k = 0; k < EPA; ++k) {
+        const float yh = dequant((bits >> (4 * k)) & 0xFu, mn, s);
+        if constexpr (decltype(interior)::value) dot = fmaf(v[k], yh, dot);
+        else dot = fmaf((msk >> k & 1u) ? v[k] : 0.0f, yh, dot);
+      }
+    });
+    dot = u.template reduce<kOpSum>(dot);
+    any_row_vectors<DT, UNIT_>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
+      float v[EPA];
+      V::widen(*(const typename V::Raw*)(p.data + j * 16u), v);
+      const uint32_t bits = V::load_codes(p.codes, j);
+#pragma unroll
+      for (int k = 0; k < EPA; ++k) v[k] = dequant((bits >> (4 * k)) & 0xFu, mn, s) * (v[k] - dot);
+      const typename V::Raw ow = V::narrow(v);
+      if constexpr (decltype(interior)::value) *(typename V::Raw*)(p.data + j * 16u) = ow;
+      else R::store(p.data, j, ow, msk);
+    });
+    if (UNIT_ < 32) u.sync();
+  }
+};
+
 // ---------------------------------------------------------------- odd rows, fixed length
 // Softmax rows of a compile-time odd length (the attention widths 197 and 257).  Rows
 // are read as 2-element words on the tile's even-element grid: a row that starts on an
@@ -1775,8 +2003,28 @@ cudaError_t launch_pair_fixed(const TilePlan& p, const TileKernelArgs& ka, cudaS
   return cudaErrorInvalidValue;
 }
 
+template <template <int, int> class WORK, int DT>
+cudaError_t launch_any(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
+  switch (p.unit_lanes) {
+    case 1: return launch_work<WORK<DT, 1>>(p, ka, st);
+    case 2: return launch_work<WORK<DT, 2>>(p, ka, st);
+    case 4: return launch_work<WORK<DT, 4>>(p, ka, st);
+    case 8: return launch_work<WORK<DT, 8>>(p, ka, st);
+    case 16: return launch_work<WORK<DT, 16>>(p, ka, st);
+    case 32: return launch_work<WORK<DT, 32>>(p, ka, st);
+    case 64: return launch_work<WORK<DT, 64>>(p, ka, st);
+    case 128: return launch_work<WORK<DT, 128>>(p, ka, st);
+  }
+  return cudaErrorInvalidValue;
+}
+
 template <int KERNEL, int DT>
 cudaError_t launch_variant(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
+  if (p.variant == kVariantAny) {
+    if constexpr (KERNEL == kSoftmaxFwd) return launch_any<AnySoftmaxFwd, DT>(p, ka, st);
+    if constexpr (KERNEL == kSoftmaxBwd) return launch_any<AnySoftmaxBwd, DT>(p, ka, st);
+    return cudaErrorInvalidValue;
+  }
   if (p.variant == kVariantStream) {
     if constexpr (KERNEL == kGeluFwd) return launch_gelu_stream<StreamGeluFwd, DT>(p, ka, st);
     if constexpr (KERNEL == kGeluBwd) return launch_gelu_stream<StreamGeluBwd, DT>(p, ka, st);

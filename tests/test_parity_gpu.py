@@ -85,7 +85,10 @@ GELU_SHAPES = [(5, 1), (3, 2), (7, 3), (9, 63), (701, 63), (64, 64), (1001, 64),
                (40, 3072), (13, 3072), (11, 4096), (9, 5120), (3, 8191), (5, 8192), (1, 16384), (2, 40000)]
 SOFTMAX_SHAPES = [(7, 1), (4, 2), (5, 3), (33, 63), (701, 63), (77, 64), (1001, 64), (531, 65), (300, 197),
                   (1, 197), (1283, 197), (130, 257), (257, 257), (323, 257), (137, 1024), (300, 66),
-                  (203, 1000), (9, 4096), (21, 3072), (7, 5120), (5, 8191), (5, 8192), (2, 40000)]
+                  (203, 1000), (9, 4096), (21, 3072), (7, 5120), (5, 8191), (5, 8192), (2, 40000),
+                  # widths that are not whole 16-byte vectors (masked vector ends), tiles + ragged tails
+                  (90, 17), (2049, 49), (1500, 50), (999, 145), (641, 198), (333, 577), (163, 1025),
+                  (1100, 196), (37, 16384)]
 
 
 @pytest.mark.parametrize("dt", [F32, BF16])
@@ -106,6 +109,7 @@ def test_in_place(dt):
     check_gelu(*_gelu_inputs(70, 197, dt, seed=3), 197, dt, inplace=True)
     check_softmax(*_softmax_inputs(700, 197, dt, seed=3), 197, dt, inplace=True)
     check_softmax(*_softmax_inputs(20, 4096, dt, seed=3), 4096, dt, inplace=True)
+    check_softmax(*_softmax_inputs(515, 145, dt, seed=3), 145, dt, inplace=True)
 
 
 def test_benchmark_shapes_take_the_pipelined_path():
@@ -119,9 +123,10 @@ def test_benchmark_shapes_take_the_pipelined_path():
 
 
 # ------------------------------------------------------------------ degenerate inputs
+@pytest.mark.parametrize("L", [197, 145, 200])
 @pytest.mark.parametrize("dt", [F32, BF16])
-def test_degenerate_rows(dt):
-    L, rows = 197, 66
+def test_degenerate_rows(dt, L):
+    rows = 66
     x = np.zeros((rows, L), dtype=np.float32)
     x[1] = 0.37          # constant rows: max == min
     x[2] = -5.0
