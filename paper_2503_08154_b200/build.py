@@ -11,7 +11,7 @@ CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 OUT = os.path.join(HERE, "libs2a.so")
 SOURCES = ["s2a_api.cu", "s2a_rowwise.cu", "s2a_relu.cu", "s2a_side.cu", "s2a_tensor_range.cu", "s2a_tile.cu", "s2a_tile_gelu_fwd.cu",
-           "s2a_tile_gelu_bwd.cu", "s2a_tile_softmax_fwd.cu", "s2a_tile_softmax_bwd.cu", "s2a_tile_silu.cu", "s2a_tile_bits.cu"]
+           "s2a_tile_gelu_bwd.cu", "s2a_tile_softmax_fwd.cu", "s2a_tile_softmax_bwd.cu", "s2a_tile_silu.cu", "s2a_tile_bits.cu", "s2a_tile_softmax_widths.cu"]
 HEADERS = ["s2a_common.cuh", "s2a_launch.h", "s2a_tile.cuh", os.path.join("..", "..", "include", "s2a.h")]
 
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]

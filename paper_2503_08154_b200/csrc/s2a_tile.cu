@@ -15,6 +15,7 @@ cudaError_t launch_tile_softmax_bwd(int dt, const TilePlan& p, const void* kerne
 cudaError_t launch_tile_silu_fwd(int dt, const TilePlan& p, const void* kernel_args, cudaStream_t st);
 cudaError_t launch_tile_silu_bwd(int dt, const TilePlan& p, const void* kernel_args, cudaStream_t st);
 cudaError_t launch_tile_bits(int kernel, int dt, const TilePlan& p, const void* kernel_args, cudaStream_t st);
+cudaError_t launch_tile_pair_widths(int kernel, int dt, const TilePlan& p, const void* kernel_args, cudaStream_t st);
 
 namespace {
 
@@ -77,7 +78,12 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
   const bool is_silu = act_of(kernel) == 1;
   const uint32_t esize = dt == kF32 ? 4u : 2u;
   const uint32_t vec = 16u / esize;  // elements per 16-byte access
-  const bool vec16 = (L % vec) == 0;
+  // attention widths with fixed-length kernels of their own (ViT 197 / 257, DeiT 198, no class
+  // token 196, patch-32 models 49 / 50, 145): read as 2-element words even where 16-byte
+  // vectors would fit (196 in binary32)
+  const bool pair_width = !is_gelu && bits == 4 && !force_generic && !(var && var[0] == 'a') &&
+                          (L == 197 || L == 257 || L == 49 || L == 50 || L == 145 || L == 196 || L == 198);
+  const bool vec16 = (L % vec) == 0 && !pair_width;
   const uint32_t epa = vec16 ? vec : 2u;
   const uint32_t n_acc = vec16 ? L / vec : (L + 1) / 2;  // accesses covering one row
   // rows per tile: the tile's code bytes must be a multiple of 16 (its element count a
@@ -122,7 +128,7 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
     } else {
       unit = 0;
     }
-  } else if (!vec16 && !force_generic && !is_gelu && (L == 197 || L == 257)) {
+  } else if (pair_width) {
     variant = kVariantPairFixed;
     unit = 8;
     iters = (n_acc + 7) / 8;
@@ -181,6 +187,7 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
   if (warps < 1 || warps > 16 || (warps * 32) % unit != 0) return p;
   const uint32_t n_units = warps * 32 / unit;
   uint32_t G = (!vec16 && (L & 1u)) ? 2u : 1u;  // rows a unit takes per round
+  if (variant == kVariantPairFixed) G = 2;       // always a pair, whatever the parity
   if (variant == kVariantStream && kernel == kSoftmaxFwd) {
     const uint32_t held = iters * epa;            // elements a lane keeps per row
     G = held <= 8 ? 4u : (held <= 16 ? 2u : 1u);  // as StreamSoftmaxFwd::RPU
@@ -279,6 +286,8 @@ cudaError_t launch_tile(int kernel, int dt, const TilePlan& p, const TileArgs& a
   ka.error_word = error_word_address();
   if (!ka.error_word) return cudaErrorInvalidDevice;
   if (p.bits != 4) return launch_tile_bits(kernel, dt, p, &ka, st);
+  if (p.variant == kVariantPairFixed && a.row_len != 197 && a.row_len != 257)
+    return launch_tile_pair_widths(kernel, dt, p, &ka, st);
   switch (kernel) {
     case kGeluFwd: return launch_tile_gelu_fwd(dt, p, &ka, st);
     case kGeluBwd: return launch_tile_gelu_bwd(dt, p, &ka, st);

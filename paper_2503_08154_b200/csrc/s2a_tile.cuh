@@ -1386,12 +1386,15 @@ struct AnySoftmaxBwd {
 };
 
 // ---------------------------------------------------------------- odd rows, fixed length
-// Softmax rows of a compile-time odd length (the attention widths 197 and 257).  Rows
-// are read as 2-element words on the tile's even-element grid: a row that starts on an
-// even element shares its LAST word (and code byte) with the next row, a row that starts
-// on an odd element shares its FIRST word with the previous one; a unit handles such a
-// pair back to back.  With the length fixed every mask is resolved at compile time
-// except on the one or two words that are actually shared or ragged.
+// Softmax rows of a compile-time length that is not a whole number of 16-byte vectors (the
+// attention widths 197 and 257, and 49, 50, 145, 196, 198).  Rows are read as 2-element
+// words on the tile's even-element grid.  With an odd length a row that starts on an even
+// element shares its LAST word (and code byte) with the next row, a row that starts on an
+// odd element shares its FIRST word with the previous one; a unit handles such a pair back
+// to back.  With the length fixed every mask is resolved at compile time except on the one
+// or two words that are actually shared or ragged.  HP names a row's kind: 0 starts even
+// and shares its last word, 1 starts odd and shares its first, 2 (even lengths) shares
+// nothing.
 template <int DT> struct P2;
 template <> struct P2<kBF16> {
   using Raw = uint32_t;
@@ -1421,7 +1424,7 @@ template <> struct P2<kF32> {
 
 template <int UNIT_, int LCT>
 struct PairGeom {
-  static_assert(LCT % 2 == 1, "odd row lengths only");
+  static constexpr bool kOdd = (LCT % 2) == 1;             // even lengths: rows own whole words
   static constexpr int NACC = (LCT + 1) / 2;               // words covering one row
   static constexpr int ITERS = (NACC + UNIT_ - 1) / UNIT_;
   static constexpr int NFULL = NACC / UNIT_;               // iterations in which every lane has a word
@@ -1515,9 +1518,14 @@ struct PairSoftmaxFwd {
   static __device__ __forceinline__ void group(Unit<UNIT_>& u, State&, const StagePtrs& p, float*, uint32_t grp,
                                                bool active, uint32_t) {
     const uint32_t r = active ? 2 * grp : 0;
-    row<0>(u, p, r, active);
-    u.sync();  // the odd row reads the shared word and code byte the even row left
-    row<1>(u, p, r + 1, active);
+    if (G::kOdd) {
+      row<0>(u, p, r, active);
+      u.sync();  // the odd row reads the shared word and code byte the even row left
+      row<1>(u, p, r + 1, active);
+    } else {
+      row<2>(u, p, r, active);
+      row<2>(u, p, r + 1, active);
+    }
     u.sync();
   }
 };
@@ -1630,10 +1638,11 @@ struct PairSoftmaxFwd<kBF16, UNIT_, LCT> {
                                                bool active, uint32_t) {
     const uint32_t r = active ? 2 * grp : 0;
     const int ul = u.ul;
-    const uint32_t a0 = (r * (uint32_t)LCT) >> 1, a1 = ((r + 1) * (uint32_t)LCT) >> 1;  // a1 = a0 + NACC - 1
+    const uint32_t a0 = (r * (uint32_t)LCT) >> 1, a1 = ((r + 1) * (uint32_t)LCT) >> 1;  // odd: a1 = a0 + NACC - 1
     Regs A, B;
-    float mA = load_max<0>(A, (const uint32_t*)p.data + a0 + ul, ul);
-    float mB = load_max<1>(B, (const uint32_t*)p.data + a1 + ul, ul);
+    constexpr int HA = G::kOdd ? 0 : 2, HB = G::kOdd ? 1 : 2;  // the kinds of the pair's two rows
+    float mA = load_max<HA>(A, (const uint32_t*)p.data + a0 + ul, ul);
+    float mB = load_max<HB>(B, (const uint32_t*)p.data + a1 + ul, ul);
     mA = u.template reduce<kOpMax>(mA);
     mB = u.template reduce<kOpMax>(mB);
     float zA = exp_sum(A, mA);
@@ -1641,8 +1650,8 @@ struct PairSoftmaxFwd<kBF16, UNIT_, LCT> {
     zA = u.template reduce<kOpSum>(zA);
     zB = u.template reduce<kOpSum>(zB);
     float mnA, mxA, mnB, mxB;
-    scale_store<0>(A, __fdiv_rn(1.0f, zA), (uint32_t*)p.data + a0 + ul, ul, active, mnA, mxA);
-    scale_store<1>(B, __fdiv_rn(1.0f, zB), (uint32_t*)p.data + a1 + ul, ul, active, mnB, mxB);
+    scale_store<HA>(A, __fdiv_rn(1.0f, zA), (uint32_t*)p.data + a0 + ul, ul, active, mnA, mxA);
+    scale_store<HB>(B, __fdiv_rn(1.0f, zB), (uint32_t*)p.data + a1 + ul, ul, active, mnB, mxB);
     reduce_minmax_bf16<UNIT_>(mnA, mxA);
     reduce_minmax_bf16<UNIT_>(mnB, mxB);
     const QRange qA = make_qrange(mnA, mxA), qB = make_qrange(mnB, mxB);
@@ -1652,16 +1661,16 @@ struct PairSoftmaxFwd<kBF16, UNIT_, LCT> {
     }
     // The byte the two rows share: row A's last element is its low nibble, row B's first
     // its high nibble.  A's nibble travels by shuffle to the lane that owns B's first word.
-    const uint32_t a_last = code_byte<0>(A, G::LAST_I, ul, qA);
+    const uint32_t a_last = code_byte<HA>(A, G::LAST_I, ul, qA);
     const uint32_t shared_lo = __shfl_sync(0xffffffffu, a_last, (threadIdx.x & 31 & ~(UNIT_ - 1)) | G::LAST_UL);
     unsigned char* cA = p.codes + a0 + ul;
     unsigned char* cB = p.codes + a1 + ul;
 #pragma unroll
     for (int i = 0; i < G::ITERS; ++i) {
       if (active && G::has(i, ul)) {
-        if (!(i == G::LAST_I && ul == G::LAST_UL)) cA[UNIT_ * i] = (unsigned char)code_byte<0>(A, i, ul, qA);
-        uint32_t b = code_byte<1>(B, i, ul, qB);
-        if (i == 0 && ul == 0) b |= shared_lo & 0x0Fu;
+        if (!G::kOdd || !(i == G::LAST_I && ul == G::LAST_UL)) cA[UNIT_ * i] = (unsigned char)code_byte<HA>(A, i, ul, qA);
+        uint32_t b = code_byte<HB>(B, i, ul, qB);
+        if (G::kOdd && i == 0 && ul == 0) b |= shared_lo & 0x0Fu;
         cB[UNIT_ * i] = (unsigned char)b;
       }
     }
@@ -1723,9 +1732,14 @@ struct PairSoftmaxBwd {
   static __device__ __forceinline__ void group(Unit<UNIT_>& u, State&, const StagePtrs& p, float*, uint32_t grp,
                                                bool active, uint32_t) {
     const uint32_t r = active ? 2 * grp : 0;
-    row<0>(u, p, r, active);
-    u.sync();  // the odd row's first word holds the even row's last result
-    row<1>(u, p, r + 1, active);
+    if (G::kOdd) {
+      row<0>(u, p, r, active);
+      u.sync();  // the odd row's first word holds the even row's last result
+      row<1>(u, p, r + 1, active);
+    } else {
+      row<2>(u, p, r, active);
+      row<2>(u, p, r + 1, active);
+    }
     u.sync();
   }
 };
@@ -2001,6 +2015,27 @@ cudaError_t launch_pair_fixed(const TilePlan& p, const TileKernelArgs& ka, cudaS
     case 257: return launch_work<WORK<DT, 8, 257>>(p, ka, st);
   }
   return cudaErrorInvalidValue;
+}
+
+// The other fixed widths (instantiated in a translation unit of their own).
+template <template <int, int, int> class WORK, int DT>
+cudaError_t launch_pair_widths(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
+  if (p.unit_lanes != 8) return cudaErrorInvalidValue;
+  switch (ka.row_len) {
+    case 49: return launch_work<WORK<DT, 8, 49>>(p, ka, st);
+    case 50: return launch_work<WORK<DT, 8, 50>>(p, ka, st);
+    case 145: return launch_work<WORK<DT, 8, 145>>(p, ka, st);
+    case 196: return launch_work<WORK<DT, 8, 196>>(p, ka, st);
+    case 198: return launch_work<WORK<DT, 8, 198>>(p, ka, st);
+  }
+  return cudaErrorInvalidValue;
+}
+template <int KERNEL>
+cudaError_t launch_tile_pair_widths_kernel(int dt, const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
+  if constexpr (KERNEL == kSoftmaxFwd)
+    return dt == kF32 ? launch_pair_widths<PairSoftmaxFwd, kF32>(p, ka, st) : launch_pair_widths<PairSoftmaxFwd, kBF16>(p, ka, st);
+  else
+    return dt == kF32 ? launch_pair_widths<PairSoftmaxBwd, kF32>(p, ka, st) : launch_pair_widths<PairSoftmaxBwd, kBF16>(p, ka, st);
 }
 
 template <template <int, int> class WORK, int DT>
