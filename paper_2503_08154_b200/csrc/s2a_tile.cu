@@ -120,10 +120,13 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
     for (int k = 0; k < 5 && unit == 0; ++k)
       if ((n_acc + units[k] - 1) / units[k] <= cap) unit = units[k];
     if (unit == 0 && (n_acc + 127) / 128 <= cap2) unit = 128;
-    if (env_unit == 8 || env_unit == 16 || env_unit == 32 || env_unit == 64 || env_unit == 128) unit = (uint32_t)env_unit;
+    if (dt == kBF16 && n_acc > 4 && n_acc <= 8) unit = 4;  // 40..64 elements: two vectors per lane, one shuffle step less
+    if (env_unit == 2 || env_unit == 4 || env_unit == 8 || env_unit == 16 || env_unit == 32 || env_unit == 64 ||
+        env_unit == 128)
+      unit = (uint32_t)env_unit;
     if (unit != 0 && (n_acc + unit - 1) / unit <= cap2) {
       variant = kVariantStream;
-      iters = unit >= 64 ? 4 : 1;
+      iters = unit >= 64 ? 4 : (unit < 8 ? 2 : 1);
       while (iters < (n_acc + unit - 1) / unit) iters *= 2;
     } else {
       unit = 0;

@@ -1967,9 +1967,21 @@ cudaError_t launch_softmax_wide(const TilePlan& p, const TileKernelArgs& ka, cud
   return cudaErrorInvalidValue;
 }
 
+// Units of 2 or 4 lanes take the very short rows: 2 or 4 vectors per lane.
+template <template <int, int, int> class WORK, int DT, int UNIT>
+cudaError_t launch_softmax_narrow(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
+  switch (p.iters) {
+    case 2: return launch_work<WORK<DT, UNIT, 2>>(p, ka, st);
+    case 4: return launch_work<WORK<DT, UNIT, 4>>(p, ka, st);
+  }
+  return cudaErrorInvalidValue;
+}
+
 template <template <int, int, int> class WORK, int DT>
 cudaError_t launch_softmax_stream(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
   switch (p.unit_lanes) {
+    case 2: return launch_softmax_narrow<WORK, DT, 2>(p, ka, st);
+    case 4: return launch_softmax_narrow<WORK, DT, 4>(p, ka, st);
     case 8: return launch_softmax_nv<WORK, DT, 8>(p, ka, st);
     case 16: return launch_softmax_nv<WORK, DT, 16>(p, ka, st);
     case 32: return launch_softmax_nv<WORK, DT, 32>(p, ka, st);
