@@ -197,6 +197,10 @@ def cases(quick: bool):
                 continue
             for dtype in (torch.bfloat16, torch.float32):
                 out.append(("softmax", rows, L, dtype))
+    # other attention widths (none a whole number of 16-byte vectors in bfloat16), about 1e8 elements
+    for L in (() if quick else (49, 50, 145, 196, 198, 577, 1025)):
+        for dtype in (torch.bfloat16, torch.float32):
+            out.append(("softmax", max(32, 10**8 // L // 32 * 32), L, dtype))
     return out
 
 

@@ -79,10 +79,11 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
   const uint32_t esize = dt == kF32 ? 4u : 2u;
   const uint32_t vec = 16u / esize;  // elements per 16-byte access
   // attention widths with fixed-length kernels of their own (ViT 197 / 257, DeiT 198, no class
-  // token 196, patch-32 models 49 / 50, 145): read as 2-element words even where 16-byte
+  // token 196, patch-32 models 49 / 50, 145, and 577 / 1025 of the 384 / 512 pixel models): read as 2-element words even where 16-byte
   // vectors would fit (196 in binary32)
   const bool pair_width = !is_gelu && bits == 4 && !force_generic && !(var && var[0] == 'a') &&
-                          (L == 197 || L == 257 || L == 49 || L == 50 || L == 145 || L == 196 || L == 198);
+                          (L == 197 || L == 257 || L == 49 || L == 50 || L == 145 || L == 196 || L == 198 || L == 577 ||
+                           L == 1025);
   const bool vec16 = (L % vec) == 0 && !pair_width;
   const uint32_t epa = vec16 ? vec : 2u;
   const uint32_t n_acc = vec16 ? L / vec : (L + 1) / 2;  // accesses covering one row
@@ -133,8 +134,8 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
     }
   } else if (pair_width) {
     variant = kVariantPairFixed;
-    unit = 8;
-    iters = (n_acc + 7) / 8;
+    unit = L > 257 ? 32u : 8u;
+    iters = (n_acc + unit - 1) / unit;
   }
   const bool force_any = var && var[0] == 'a';
   if (!is_gelu && bits == 4 && !force_generic && L >= 16 &&
@@ -172,6 +173,7 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
   }
 
   uint32_t warps = unit == 128 ? 8u : 4u;
+  if (variant == kVariantPairFixed && unit == 32) warps = 8;  // four row pairs in flight are too few (measured)
   if (variant == kVariantAny) {
     // eight consumer warps, four when that many sub-warp units would need a tile beyond 40 KB
     const uint32_t want = (256u / unit) * ((L & 1u) ? 2u : 1u);  // rows that keep eight warps busy

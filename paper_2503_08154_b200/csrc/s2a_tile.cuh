@@ -1387,7 +1387,7 @@ struct AnySoftmaxBwd {
 
 // ---------------------------------------------------------------- odd rows, fixed length
 // Softmax rows of a compile-time length that is not a whole number of 16-byte vectors (the
-// attention widths 197 and 257, and 49, 50, 145, 196, 198).  Rows are read as 2-element
+// attention widths 197 and 257, and 49, 50, 145, 196, 198, 577, 1025).  Rows are read as 2-element
 // words on the tile's even-element grid.  With an odd length a row that starts on an even
 // element shares its LAST word (and code byte) with the next row, a row that starts on an
 // odd element shares its FIRST word with the previous one; a unit handles such a pair back
@@ -2032,6 +2032,13 @@ cudaError_t launch_pair_fixed(const TilePlan& p, const TileKernelArgs& ka, cudaS
 // The other fixed widths (instantiated in a translation unit of their own).
 template <template <int, int, int> class WORK, int DT>
 cudaError_t launch_pair_widths(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
+  if (p.unit_lanes == 32) {  // the long widths: a warp per row pair
+    switch (ka.row_len) {
+      case 577: return launch_work<WORK<DT, 32, 577>>(p, ka, st);
+      case 1025: return launch_work<WORK<DT, 32, 1025>>(p, ka, st);
+    }
+    return cudaErrorInvalidValue;
+  }
   if (p.unit_lanes != 8) return cudaErrorInvalidValue;
   switch (ka.row_len) {
     case 49: return launch_work<WORK<DT, 8, 49>>(p, ka, st);

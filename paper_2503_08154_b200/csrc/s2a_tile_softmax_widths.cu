@@ -1,5 +1,5 @@
 // Instantiations of the fixed-width softmax kernels for the attention widths other than
-// 197 and 257 (49, 50, 145, 196, 198).
+// 197 and 257 (49, 50, 145, 196, 198, 577, 1025).
 #include "s2a_tile.cuh"
 
 namespace s2a {
