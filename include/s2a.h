@@ -196,10 +196,11 @@ int s2a_relu_bwd(const void* grad_out, const uint8_t* mask, void* grad_in, size_
  * bits = 4 is exactly s2a_gelu_fwd / _bwd / s2a_softmax_fwd / _bwd (same kernels, same
  * speed).  bits = 2 and bits = 8 use 3 and 255 quantisation levels, pack 4 codes or 1 code
  * per byte (element e owns bits [(e N) mod 8, (e N) mod 8 + N) of byte (e N) / 8, least
- * significant first).  The GELU pair has a pipelined form at these widths for rows of whole
- * 16-byte vectors with at least 128 of them (row_len >= 1024 bfloat16, 512 binary32); the
- * softmax pair and all other shapes run row at a time, well below the bandwidth of the 4-bit
- * kernels.  codes: s2a_codes_bytes_bits(n_elems, bits) bytes.  Any other
+ * significant first).  Pipelined forms at these widths: the GELU pair for rows of whole
+ * 16-byte vectors with at least 128 of them (row_len >= 1024 bfloat16, 512 binary32), the
+ * softmax pair for any row_len >= 16 whose rows fit a shared-memory tile (about half the
+ * bandwidth of the 4-bit kernels); other shapes run row at a time.
+ * codes: s2a_codes_bytes_bits(n_elems, bits) bytes.  Any other
  * `bits` returns S2A_ERR_SHAPE.  Everything else as for the 4-bit entry points.
  */
 size_t s2a_codes_bytes_bits(size_t n_elems, int bits);

@@ -153,7 +153,7 @@ def _time_side(seed: int):
 
 
 def _time_bits(seed: int):
-    """The 2-bit and 8-bit forms on one ViT-B/16 block, bfloat16 (GELU pipelined, softmax row at a time)."""
+    """The 2-bit and 8-bit forms on one ViT-B/16 block, bfloat16."""
     out = []
     g = torch.Generator(device="cuda").manual_seed(seed)
     for kind, rows, L in (("gelu", 12608, 3072), ("softmax", 151296, 197)):
@@ -178,8 +178,7 @@ def _time_bits(seed: int):
                 res[name] = (4 * n + n * bits // 8 + 8 * rows) / (e0.elapsed_time(e1) * 1e-3 / 12) / 1e9
             out.append({"kernel_pair": kind + "_bits", "bits": bits, "rows": rows, "row_len": L, "io_dtype": "bf16",
                         "fwd_GBps": round(res["fwd"], 1), "bwd_GBps": round(res["bwd"], 1),
-                        "note": ("pipelined path" if kind == "gelu" else "row-at-a-time path")
-                        + "; algorithmic bytes = 4*n + n*bits/8 + 8*rows"})
+                        "note": "pipelined path; algorithmic bytes = 4*n + n*bits/8 + 8*rows"})
     return out
 
 

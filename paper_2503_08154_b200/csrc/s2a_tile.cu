@@ -96,7 +96,15 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
 
   uint32_t variant = kVariantGeneric, unit = 0, iters = 0;
   const int env_unit = env_int("S2A_UNIT", 0);
-  if (bits != 4) {
+  if (bits != 4 && (kernel == kSoftmaxFwd || kernel == kSoftmaxBwd)) {
+    // other code widths, softmax: the any-length form (aligned vectors, masked row ends)
+    if (L < 16) return p;
+    variant = kVariantAny;
+    const uint32_t nvr = (L + vec - 1) / vec + 1;
+    unit = 2;
+    while (unit < 32 && (nvr + unit - 1) / unit > 4) unit *= 2;  // measured at 197: 8 lanes beat 4 and 16
+    if (env_unit == 2 || env_unit == 4 || env_unit == 8 || env_unit == 16 || env_unit == 32) unit = (uint32_t)env_unit;
+  } else if (bits != 4) {
     // other code widths: GELU rows of whole vectors, long enough for a two-warp unit
     if (!(kernel == kGeluFwd || kernel == kGeluBwd) || !vec16 || n_acc < 128) return p;
     variant = kVariantStream;
@@ -176,7 +184,7 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
   if (variant == kVariantPairFixed && unit == 32) warps = 8;  // four row pairs in flight are too few (measured)
   if (variant == kVariantAny) {
     // eight consumer warps, four when that many sub-warp units would need a tile beyond 40 KB
-    const uint32_t want = (256u / unit) * ((L & 1u) ? 2u : 1u);  // rows that keep eight warps busy
+    const uint32_t want = 256u / unit;  // rows that keep eight warps busy
     warps = (want > r_min && (uint64_t)want * L * esize > 40 * 1024) ? 4u : 8u;
   }
   if (variant == kVariantStream && !is_gelu) {
@@ -193,6 +201,7 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
   const uint32_t n_units = warps * 32 / unit;
   uint32_t G = (!vec16 && (L & 1u)) ? 2u : 1u;  // rows a unit takes per round
   if (variant == kVariantPairFixed) G = 2;       // always a pair, whatever the parity
+  if (variant == kVariantAny) G = 1;              // shared code bytes are merged atomically
   if (variant == kVariantStream && kernel == kSoftmaxFwd) {
     const uint32_t held = iters * epa;            // elements a lane keeps per row
     G = held <= 8 ? 4u : (held <= 16 ? 2u : 1u);  // as StreamSoftmaxFwd::RPU

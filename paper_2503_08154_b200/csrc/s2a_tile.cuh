@@ -1165,8 +1165,8 @@ struct StreamSoftmaxBwd {
 // 16-byte store, boundary vectors element by element, so two units never write the same
 // bytes).  Nothing is held in registers: the row is streamed from shared memory once per
 // phase, and the exponentials are evaluated twice (sum, then output) rather than kept in a
-// narrower type.  With an odd row length two consecutive rows share a code byte; one unit
-// takes both, in order, and the second merges its nibble into the byte the first one left.
+// narrower type.  With an odd row length two consecutive rows share a code byte: each merges
+// its own nibble into it atomically, so rows need no particular order.
 template <int DT>
 struct AnyRow {
   using V = V16<DT>;
@@ -1232,7 +1232,7 @@ struct AnySoftmaxFwd {
   static constexpr int EPA = V::EPA;
   struct State {};
   static __device__ __forceinline__ void init(State&) {}
-  static __device__ __forceinline__ uint32_t rows_per_group(uint32_t L) { return (L & 1u) ? 2u : 1u; }
+  static __device__ __forceinline__ uint32_t rows_per_group(uint32_t) { return 1u; }
 
   static __device__ __forceinline__ float ex(float x, float m, float nm) {
     constexpr float kLog2e = 1.4426950408889634f;
@@ -1319,9 +1319,18 @@ struct AnySoftmaxFwd {
         for (int b = 0; b < EPA / 2; ++b) {
           const uint32_t pmk = (msk >> (2 * b)) & 3u;
           const uint32_t byte = (pk.acc >> (8 * b)) & 0xFFu;
-          if (pmk == 3u) cb[b] = (unsigned char)byte;
-          else if (pmk == 1u) cb[b] = (unsigned char)(byte & 0x0Fu);                  // the high nibble is the next row's
-          else if (pmk == 2u) cb[b] = (unsigned char)((cb[b] & 0x0Fu) | (byte & 0xF0u));  // the low nibble is the previous row's
+          if (pmk == 3u) {
+            cb[b] = (unsigned char)byte;
+          } else if (pmk != 0u) {
+            // the byte's other nibble is a neighbouring row's (another unit may be writing it
+            // right now): clear and set this row's nibble atomically, on the enclosing word
+            const uint32_t mb = pmk == 1u ? 0x0Fu : 0xF0u;
+            const uint32_t off = j * (EPA / 2) + b;
+            unsigned int* word = (unsigned int*)(p.codes + (off & ~3u));
+            const uint32_t sh = 8u * (off & 3u);
+            atomicAnd(word, ~(mb << sh));
+            atomicOr(word, (byte & mb) << sh);
+          }
         }
       }
     });
@@ -1330,11 +1339,8 @@ struct AnySoftmaxFwd {
   static __device__ __forceinline__ void group(Unit<UNIT_>& u, State&, const StagePtrs& p, float*, uint32_t grp,
                                                bool active, uint32_t L) {
     if (UNIT_ >= 32 && !active) return;  // whole warps (and whole multi-warp units) leave together
-    const uint32_t G = rows_per_group(L);
-    for (uint32_t h = 0; h < G; ++h) {
-      row(u, p, active ? grp * G + h : 0u, active, L);
-      u.sync();  // the next row of the pair reads the code byte this one left
-    }
+    row(u, p, active ? grp : 0u, active, L);
+    if (UNIT_ < 32) u.sync();
   }
 };
 
@@ -1377,6 +1383,192 @@ struct AnySoftmaxBwd {
       const uint32_t bits = V::load_codes(p.codes, j);
 #pragma unroll
       for (int k = 0; k < EPA; ++k) v[k] = dequant((bits >> (4 * k)) & 0xFu, mn, s) * (v[k] - dot);
+      const typename V::Raw ow = V::narrow(v);
+      if constexpr (decltype(interior)::value) *(typename V::Raw*)(p.data + j * 16u) = ow;
+      else R::store(p.data, j, ow, msk);
+    });
+    if (UNIT_ < 32) u.sync();
+  }
+};
+
+// The any-length softmax at 2 and 8 bits per code.  A 16-byte vector still owns whole code
+// bytes (8 or 4 elements times NBITS is a multiple of 8), so interior vectors store their
+// codes in one access; on a row's first and last vector the row's bits are merged into
+// their bytes, atomically where a byte is shared with a neighbouring row (2 bits: up to
+// four rows meet in one byte when the length is odd), so rows need no particular order.
+template <int DT, int UNIT_, int NBITS>
+struct AnySoftmaxFwdBits {
+  static_assert(NBITS == 2 || NBITS == 8, "4 bits have kernels of their own");
+  static constexpr int kMaxRegs = 80;
+  static constexpr int kKernel = kSoftmaxFwd;
+  static constexpr int UNIT = UNIT_;
+  using V = V16<DT>;
+  using R = AnyRow<DT>;
+  using C = CodeIo<DT, NBITS>;
+  static constexpr int EPA = V::EPA;
+  struct State {};
+  static __device__ __forceinline__ void init(State&) {}
+  static __device__ __forceinline__ uint32_t rows_per_group(uint32_t) { return 1u; }
+  static __device__ __forceinline__ float ex(float x, float m, float nm) {
+    constexpr float kLog2e = 1.4426950408889634f;
+    return DT == kBF16 ? ex2_approx(fmaf(x, kLog2e, nm)) : exp_eval<DT>(x - m);
+  }
+
+  static __device__ __forceinline__ void row(Unit<UNIT_>& u, const StagePtrs& p, uint32_t r, bool active, uint32_t L) {
+    R g;
+    g.set(r, L);
+    const int ul = u.ul;
+    float m = -INFINITY;
+    typename V::MinMax pm;
+    pm.init();
+    any_row_vectors<DT, UNIT_>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
+      const typename V::Raw raw = *(const typename V::Raw*)(p.data + j * 16u);
+      if constexpr (decltype(interior)::value) {
+        pm.add(raw);
+      } else {
+        float v[EPA];
+        V::widen(raw, v);
+#pragma unroll
+        for (int k = 0; k < EPA; ++k) m = fmaxf(m, (msk >> k & 1u) ? v[k] : -INFINITY);
+      }
+    });
+    m = u.template reduce<kOpMax>(fmaxf(m, pm.hi()));
+    if (!active) m = 0.0f;
+    const float nm = -m * 1.4426950408889634f;
+    float z = 0.0f;
+    any_row_vectors<DT, UNIT_>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
+      float v[EPA];
+      V::widen(*(const typename V::Raw*)(p.data + j * 16u), v);
+#pragma unroll
+      for (int k = 0; k < EPA; ++k) {
+        const float e = ex(v[k], m, nm);
+        if constexpr (decltype(interior)::value) z += e;
+        else z += (msk >> k & 1u) ? e : 0.0f;
+      }
+    });
+    z = u.template reduce<kOpSum>(z);
+    const float rz = __fdiv_rn(1.0f, active ? z : 1.0f);
+    float mn = INFINITY, mx = -INFINITY;
+    typename V::MinMax py;
+    py.init();
+    any_row_vectors<DT, UNIT_>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
+      float v[EPA];
+      V::widen(*(const typename V::Raw*)(p.data + j * 16u), v);
+#pragma unroll
+      for (int k = 0; k < EPA; ++k) v[k] = ex(v[k], m, nm) * rz;
+      const typename V::Raw yw = V::narrow(v);  // v now holds y as written
+      if constexpr (decltype(interior)::value) {
+        *(typename V::Raw*)(p.data + j * 16u) = yw;
+        py.add(yw);
+      } else {
+        R::store(p.data, j, yw, msk);
+#pragma unroll
+        for (int k = 0; k < EPA; ++k) {
+          mn = fminf(mn, (msk >> k & 1u) ? v[k] : INFINITY);
+          mx = fmaxf(mx, (msk >> k & 1u) ? v[k] : -INFINITY);
+        }
+      }
+    });
+    mn = u.template reduce<kOpMin>(fminf(mn, py.lo()));
+    mx = u.template reduce<kOpMax>(fmaxf(mx, py.hi()));
+    const QRange q = make_qrange(mn, mx, (float)((1 << NBITS) - 1));
+    if (active && ul == 0) { p.meta[2 * r] = q.mn; p.meta[2 * r + 1] = q.s; }
+    any_row_vectors<DT, UNIT_>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
+      float v[EPA];
+      V::widen(*(const typename V::Raw*)(p.data + j * 16u), v);
+      CodePackerBits<EPA, NBITS> pk;
+      pk.init();
+      if constexpr (decltype(interior)::value) {
+#pragma unroll
+        for (int k = 0; k < EPA; ++k) pk.add(k, v[k], q);
+        C::store(p.codes, j, pk.acc);
+      } else {
+#pragma unroll
+        for (int k = 0; k < EPA; ++k) pk.add(k, (msk >> k & 1u) ? v[k] : q.mn, q);
+        // the row's bits of each code byte, merged with one access per byte
+        unsigned char* cb = p.codes + j * C::BYTES;
+        constexpr int PER = 32 / NBITS;
+        constexpr uint32_t kCodeMask = (1u << NBITS) - 1u;
+        uint32_t own[C::W] = {};
+#pragma unroll
+        for (int k = 0; k < EPA; ++k)
+          if (msk >> k & 1u) own[k / PER] |= kCodeMask << (NBITS * (k % PER));
+#pragma unroll
+        for (int b = 0; b < C::BYTES; ++b) {
+          const uint32_t mb = (own[b / 4] >> (8 * (b % 4))) & 0xFFu;
+          const uint32_t vb = (pk.acc[b / 4] >> (8 * (b % 4))) & mb;
+          if (mb == 0xFFu) {
+            cb[b] = (unsigned char)vb;
+          } else if (mb != 0u) {
+            // a byte shared with a neighbouring row (another unit may be merging its own bits
+            // into it right now): clear and set this row's bits atomically, on the enclosing word
+            const uint32_t off = (uint32_t)(cb + b - p.codes);
+            unsigned int* word = (unsigned int*)(p.codes + (off & ~3u));
+            const uint32_t sh = 8u * (off & 3u);
+            atomicAnd(word, ~(mb << sh));
+            atomicOr(word, vb << sh);
+          }
+        }
+      }
+    });
+  }
+
+  static __device__ __forceinline__ void group(Unit<UNIT_>& u, State&, const StagePtrs& p, float*, uint32_t grp,
+                                               bool active, uint32_t L) {
+    if (UNIT_ >= 32 && !active) return;
+    row(u, p, active ? grp : 0u, active, L);
+    if (UNIT_ < 32) u.sync();
+  }
+};
+
+template <int DT, int UNIT_, int NBITS>
+struct AnySoftmaxBwdBits {
+  static_assert(NBITS == 2 || NBITS == 8, "4 bits have kernels of their own");
+  static constexpr int kMaxRegs = 80;
+  static constexpr int kKernel = kSoftmaxBwd;
+  static constexpr int UNIT = UNIT_;
+  using V = V16<DT>;
+  using R = AnyRow<DT>;
+  using C = CodeIo<DT, NBITS>;
+  static constexpr int EPA = V::EPA;
+  struct State {};
+  static __device__ __forceinline__ void init(State&) {}
+  static __device__ __forceinline__ uint32_t rows_per_group(uint32_t) { return 1u; }  // codes are only read
+
+  static __device__ __forceinline__ float yhat(const uint32_t* w, int k, float mn, float s) {
+    constexpr int PER = 32 / NBITS;
+    return dequant((w[k / PER] >> (NBITS * (k % PER))) & ((1u << NBITS) - 1u), mn, s);
+  }
+
+  static __device__ __forceinline__ void group(Unit<UNIT_>& u, State&, const StagePtrs& p, float*, uint32_t r,
+                                               bool active, uint32_t L) {
+    if (UNIT_ >= 32 && !active) return;
+    R g;
+    g.set(active ? r : 0u, L);
+    const int ul = u.ul;
+    const float mn = active ? p.meta[2 * r] : 0.0f;
+    const float s = active ? p.meta[2 * r + 1] : 0.0f;
+    float dot = 0.0f;
+    any_row_vectors<DT, UNIT_>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
+      float v[EPA];
+      V::widen(*(const typename V::Raw*)(p.data + j * 16u), v);
+      uint32_t w[C::W];
+      C::load(p.codes, j, w);
+#pragma unroll
+      for (int k = 0; k < EPA; ++k) {
+        const float yh = yhat(w, k, mn, s);
+        if constexpr (decltype(interior)::value) dot = fmaf(v[k], yh, dot);
+        else dot = fmaf((msk >> k & 1u) ? v[k] : 0.0f, yh, dot);
+      }
+    });
+    dot = u.template reduce<kOpSum>(dot);
+    any_row_vectors<DT, UNIT_>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
+      float v[EPA];
+      V::widen(*(const typename V::Raw*)(p.data + j * 16u), v);
+      uint32_t w[C::W];
+      C::load(p.codes, j, w);
+#pragma unroll
+      for (int k = 0; k < EPA; ++k) v[k] = yhat(w, k, mn, s) * (v[k] - dot);
       const typename V::Raw ow = V::narrow(v);
       if constexpr (decltype(interior)::value) *(typename V::Raw*)(p.data + j * 16u) = ow;
       else R::store(p.data, j, ow, msk);
@@ -2097,9 +2289,25 @@ cudaError_t launch_variant(const TilePlan& p, const TileKernelArgs& ka, cudaStre
 }
 
 // The 2- and 8-bit GELU kernels (their own translation unit instantiates this).
+template <template <int, int, int> class WORK, int DT, int NBITS>
+cudaError_t launch_any_bits(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
+  switch (p.unit_lanes) {
+    case 2: return launch_work<WORK<DT, 2, NBITS>>(p, ka, st);
+    case 4: return launch_work<WORK<DT, 4, NBITS>>(p, ka, st);
+    case 8: return launch_work<WORK<DT, 8, NBITS>>(p, ka, st);
+    case 16: return launch_work<WORK<DT, 16, NBITS>>(p, ka, st);
+    case 32: return launch_work<WORK<DT, 32, NBITS>>(p, ka, st);
+  }
+  return cudaErrorInvalidValue;
+}
+
 template <int KERNEL, int DT, int NBITS>
 cudaError_t launch_bits_unit(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
-  if constexpr (KERNEL == kGeluFwd) {
+  if constexpr (KERNEL == kSoftmaxFwd) {
+    return launch_any_bits<AnySoftmaxFwdBits, DT, NBITS>(p, ka, st);
+  } else if constexpr (KERNEL == kSoftmaxBwd) {
+    return launch_any_bits<AnySoftmaxBwdBits, DT, NBITS>(p, ka, st);
+  } else if constexpr (KERNEL == kGeluFwd) {
     if (p.unit_lanes == 64) return launch_work<StreamActFwdBits<DT, 64, kActGelu, NBITS>>(p, ka, st);
     if (p.unit_lanes == 128) return launch_work<StreamActFwdBits<DT, 128, kActGelu, NBITS>>(p, ka, st);
   } else {

@@ -281,7 +281,9 @@ def test_silu(rows, L, dt):
                                          ("gelu", 1237, 4096), ("gelu", 77, 1024), ("gelu", 311, 5120),
                                          ("gelu", 13, 8192), ("gelu_narrow", 2001, 3072), ("gelu_narrow", 90, 2048),
                                          ("softmax", 9, 65), ("softmax", 300, 197), ("softmax", 12, 1024),
-                                         ("softmax", 3, 2), ("softmax", 131, 257)])
+                                         ("softmax", 3, 2), ("softmax", 131, 257), ("softmax", 1283, 198),
+                                         ("softmax", 700, 49), ("softmax", 401, 50), ("softmax", 150, 577),
+                                         ("softmax", 90, 4096), ("softmax", 517, 64), ("softmax", 1000, 197)])
 def test_other_bit_widths(kind, rows, L, bits, dt):
     # "gelu_narrow": rows that do not reach the clip, so that every row has its own (min, s)
     # and the backward's derivative table is rebuilt row after row
