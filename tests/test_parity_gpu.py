@@ -88,7 +88,8 @@ SOFTMAX_SHAPES = [(7, 1), (4, 2), (5, 3), (33, 63), (701, 63), (77, 64), (1001, 
                   (203, 1000), (9, 4096), (21, 3072), (7, 5120), (5, 8191), (5, 8192), (2, 40000),
                   # widths that are not whole 16-byte vectors (masked vector ends), tiles + ragged tails
                   (90, 17), (2049, 49), (1500, 50), (999, 145), (641, 198), (333, 577), (163, 1025),
-                  (1100, 196), (37, 16384), (300, 40), (513, 56), (2000, 48)]
+                  (1100, 196), (37, 16384), (300, 40), (513, 56), (2000, 48),
+                  (700, 401), (300, 785), (200, 1370), (1500, 100), (901, 33), (350, 255)]
 
 
 @pytest.mark.parametrize("dt", [F32, BF16])
