@@ -1205,20 +1205,54 @@ struct AnyRow {
   }
 };
 
-// Calls f(j, mask, is_interior) for the vectors of a row that this lane owns: the interior
-// vectors go round the unit's lanes with no mask at all; the first and the last vector of
-// the row (the only ones that can hold a neighbour's elements) are taken by lanes 0 and 1
-// in ONE divergent section, so that the masked code runs once per phase.
-template <int DT, int UNIT_, class F>
+// Calls f(j, mask, is_interior) for the vectors of a row that this lane owns.  The "edge"
+// vectors are those that share a 32-bit word of CODES with the row's first or last vector
+// (VPW vectors share a word; 1 if a vector's codes fill whole words): only there can
+// another row's unit write the same word, so the forward kernels write codes atomically
+// there and with plain stores everywhere else -- no word ever sees both kinds of access.
+// The interior vectors go round the unit's lanes with no mask at all; the edge vectors are
+// dealt out to the lanes in ONE divergent section, so that the masked code runs once per
+// phase.  Every phase of a kernel must use the same VPW (a lane reads back what it wrote).
+template <int DT, int UNIT_, int VPW = 1, class F>
 __device__ __forceinline__ void any_row_vectors(const AnyRow<DT>& g, int ul, bool active, F&& f) {
   if (!active) return;
-  for (uint32_t j = g.v0 + 1u + (uint32_t)ul; j < g.v1; j += UNIT_) f(j, AnyRow<DT>::kFull, std::true_type{});
-  if (UNIT_ == 1) {
-    f(g.v0, g.mask(g.v0), std::false_type{});
-    if (g.v1 != g.v0) f(g.v1, g.mask(g.v1), std::false_type{});
-  } else if (ul == 0 || (ul == 1 && g.v1 != g.v0)) {
-    const uint32_t j = ul == 0 ? g.v0 : g.v1;
+  const uint32_t lo_last = min(g.v1, (g.v0 / VPW + 1u) * VPW - 1u);   // last vector of the low edge group
+  const uint32_t hi_first = max(lo_last + 1u, (g.v1 / VPW) * VPW);     // first vector of the high edge group
+  for (uint32_t j = lo_last + 1u + (uint32_t)ul; j < hi_first; j += UNIT_) f(j, AnyRow<DT>::kFull, std::true_type{});
+  const uint32_t n_lo = lo_last - g.v0 + 1u, n_hi = g.v1 >= hi_first ? g.v1 - hi_first + 1u : 0u;
+  for (uint32_t t = (uint32_t)ul; t < n_lo + n_hi; t += UNIT_) {
+    const uint32_t j = t < n_lo ? g.v0 + t : hi_first + (t - n_lo);
     f(j, g.mask(j), std::false_type{});
+  }
+}
+
+// Merges the codes of the elements of vector j named by msk into the code bytes, with
+// atomics on the enclosing 32-bit words (acc: the vector's packed codes, NBITS each).
+template <int NBITS, int EPA>
+__device__ __forceinline__ void any_merge_codes(unsigned char* codes, uint32_t j, const uint32_t* acc, uint32_t msk) {
+  constexpr int PER = 32 / NBITS;                 // codes per word of acc
+  constexpr int BYTES = EPA * NBITS / 8;          // code bytes of one vector
+  constexpr int W = (BYTES + 3) / 4;
+  constexpr uint32_t kCodeMask = (1u << NBITS) - 1u;
+  uint32_t own[W] = {};
+#pragma unroll
+  for (int k = 0; k < EPA; ++k)
+    if (msk >> k & 1u) own[k / PER] |= kCodeMask << (NBITS * (k % PER));
+  if (BYTES >= 4) {
+#pragma unroll
+    for (int w = 0; w < W; ++w) {
+      unsigned int* word = (unsigned int*)codes + j * W + w;
+      if (own[w] != 0u) {
+        atomicAnd(word, ~own[w]);
+        atomicOr(word, acc[w] & own[w]);
+      }
+    }
+  } else {
+    const uint32_t off = j * BYTES;
+    unsigned int* word = (unsigned int*)(codes + (off & ~3u));
+    const uint32_t sh = 8u * (off & 3u);
+    atomicAnd(word, ~(own[0] << sh));
+    atomicOr(word, (acc[0] & own[0]) << sh);
   }
 }
 
@@ -1230,6 +1264,7 @@ struct AnySoftmaxFwd {
   using V = V16<DT>;
   using R = AnyRow<DT>;
   static constexpr int EPA = V::EPA;
+  static constexpr int kVPW = EPA == 8 ? 1 : 2;  // vectors per 32-bit word of codes
   struct State {};
   static __device__ __forceinline__ void init(State&) {}
   static __device__ __forceinline__ uint32_t rows_per_group(uint32_t) { return 1u; }
@@ -1247,7 +1282,7 @@ struct AnySoftmaxFwd {
     float m = -INFINITY;
     typename V::MinMax pm;
     pm.init();
-    any_row_vectors<DT, UNIT_>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
+    any_row_vectors<DT, UNIT_, kVPW>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
       const typename V::Raw raw = *(const typename V::Raw*)(p.data + j * 16u);
       if constexpr (decltype(interior)::value) {
         pm.add(raw);
@@ -1263,7 +1298,7 @@ struct AnySoftmaxFwd {
     const float nm = -m * 1.4426950408889634f;
     // ---- sum of exponentials
     float z = 0.0f;
-    any_row_vectors<DT, UNIT_>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
+    any_row_vectors<DT, UNIT_, kVPW>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
       float v[EPA];
       V::widen(*(const typename V::Raw*)(p.data + j * 16u), v);
 #pragma unroll
@@ -1279,7 +1314,7 @@ struct AnySoftmaxFwd {
     float mn = INFINITY, mx = -INFINITY;
     typename V::MinMax py;
     py.init();
-    any_row_vectors<DT, UNIT_>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
+    any_row_vectors<DT, UNIT_, kVPW>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
       float v[EPA];
       V::widen(*(const typename V::Raw*)(p.data + j * 16u), v);
 #pragma unroll
@@ -1302,7 +1337,7 @@ struct AnySoftmaxFwd {
     const QRange q = make_qrange(mn, mx);
     if (active && ul == 0) { p.meta[2 * r] = q.mn; p.meta[2 * r + 1] = q.s; }
     // ---- codes of y as written (each lane reads back the vectors it wrote itself)
-    any_row_vectors<DT, UNIT_>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
+    any_row_vectors<DT, UNIT_, kVPW>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
       float v[EPA];
       V::widen(*(const typename V::Raw*)(p.data + j * 16u), v);
       CodePacker<EPA> pk;
@@ -1314,24 +1349,7 @@ struct AnySoftmaxFwd {
       } else {
 #pragma unroll
         for (int k = 0; k < EPA; ++k) pk.add(k, (msk >> k & 1u) ? v[k] : q.mn, q);  // a neighbour's element codes as 0
-        unsigned char* cb = p.codes + j * (EPA / 2);
-#pragma unroll
-        for (int b = 0; b < EPA / 2; ++b) {
-          const uint32_t pmk = (msk >> (2 * b)) & 3u;
-          const uint32_t byte = (pk.acc >> (8 * b)) & 0xFFu;
-          if (pmk == 3u) {
-            cb[b] = (unsigned char)byte;
-          } else if (pmk != 0u) {
-            // the byte's other nibble is a neighbouring row's (another unit may be writing it
-            // right now): clear and set this row's nibble atomically, on the enclosing word
-            const uint32_t mb = pmk == 1u ? 0x0Fu : 0xF0u;
-            const uint32_t off = j * (EPA / 2) + b;
-            unsigned int* word = (unsigned int*)(p.codes + (off & ~3u));
-            const uint32_t sh = 8u * (off & 3u);
-            atomicAnd(word, ~(mb << sh));
-            atomicOr(word, (byte & mb) << sh);
-          }
-        }
+        any_merge_codes<4, EPA>(p.codes, j, &pk.acc, msk);
       }
     });
   }
@@ -1406,6 +1424,7 @@ struct AnySoftmaxFwdBits {
   using R = AnyRow<DT>;
   using C = CodeIo<DT, NBITS>;
   static constexpr int EPA = V::EPA;
+  static constexpr int kVPW = C::BYTES >= 4 ? 1 : 4 / C::BYTES;  // vectors per 32-bit word of codes
   struct State {};
   static __device__ __forceinline__ void init(State&) {}
   static __device__ __forceinline__ uint32_t rows_per_group(uint32_t) { return 1u; }
@@ -1421,7 +1440,7 @@ struct AnySoftmaxFwdBits {
     float m = -INFINITY;
     typename V::MinMax pm;
     pm.init();
-    any_row_vectors<DT, UNIT_>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
+    any_row_vectors<DT, UNIT_, kVPW>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
       const typename V::Raw raw = *(const typename V::Raw*)(p.data + j * 16u);
       if constexpr (decltype(interior)::value) {
         pm.add(raw);
@@ -1436,7 +1455,7 @@ struct AnySoftmaxFwdBits {
     if (!active) m = 0.0f;
     const float nm = -m * 1.4426950408889634f;
     float z = 0.0f;
-    any_row_vectors<DT, UNIT_>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
+    any_row_vectors<DT, UNIT_, kVPW>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
       float v[EPA];
       V::widen(*(const typename V::Raw*)(p.data + j * 16u), v);
 #pragma unroll
@@ -1451,7 +1470,7 @@ struct AnySoftmaxFwdBits {
     float mn = INFINITY, mx = -INFINITY;
     typename V::MinMax py;
     py.init();
-    any_row_vectors<DT, UNIT_>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
+    any_row_vectors<DT, UNIT_, kVPW>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
       float v[EPA];
       V::widen(*(const typename V::Raw*)(p.data + j * 16u), v);
 #pragma unroll
@@ -1473,7 +1492,7 @@ struct AnySoftmaxFwdBits {
     mx = u.template reduce<kOpMax>(fmaxf(mx, py.hi()));
     const QRange q = make_qrange(mn, mx, (float)((1 << NBITS) - 1));
     if (active && ul == 0) { p.meta[2 * r] = q.mn; p.meta[2 * r + 1] = q.s; }
-    any_row_vectors<DT, UNIT_>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
+    any_row_vectors<DT, UNIT_, kVPW>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
       float v[EPA];
       V::widen(*(const typename V::Raw*)(p.data + j * 16u), v);
       CodePackerBits<EPA, NBITS> pk;
@@ -1485,30 +1504,7 @@ struct AnySoftmaxFwdBits {
       } else {
 #pragma unroll
         for (int k = 0; k < EPA; ++k) pk.add(k, (msk >> k & 1u) ? v[k] : q.mn, q);
-        // the row's bits of each code byte, merged with one access per byte
-        unsigned char* cb = p.codes + j * C::BYTES;
-        constexpr int PER = 32 / NBITS;
-        constexpr uint32_t kCodeMask = (1u << NBITS) - 1u;
-        uint32_t own[C::W] = {};
-#pragma unroll
-        for (int k = 0; k < EPA; ++k)
-          if (msk >> k & 1u) own[k / PER] |= kCodeMask << (NBITS * (k % PER));
-#pragma unroll
-        for (int b = 0; b < C::BYTES; ++b) {
-          const uint32_t mb = (own[b / 4] >> (8 * (b % 4))) & 0xFFu;
-          const uint32_t vb = (pk.acc[b / 4] >> (8 * (b % 4))) & mb;
-          if (mb == 0xFFu) {
-            cb[b] = (unsigned char)vb;
-          } else if (mb != 0u) {
-            // a byte shared with a neighbouring row (another unit may be merging its own bits
-            // into it right now): clear and set this row's bits atomically, on the enclosing word
-            const uint32_t off = (uint32_t)(cb + b - p.codes);
-            unsigned int* word = (unsigned int*)(p.codes + (off & ~3u));
-            const uint32_t sh = 8u * (off & 3u);
-            atomicAnd(word, ~(mb << sh));
-            atomicOr(word, vb << sh);
-          }
-        }
+        any_merge_codes<NBITS, EPA>(p.codes, j, pk.acc, msk);
       }
     });
   }
