@@ -148,6 +148,21 @@ def test_degenerate_rows(dt, L):
     check_softmax(synth.to_io(xs.reshape(-1), dt), synth.to_io(g, dt), L, dt)
 
 
+@pytest.mark.parametrize("L", [197, 64, 145, 1024])
+@pytest.mark.parametrize("dt", [F32, BF16])
+def test_softmax_large_common_offset(dt, L):
+    # softmax is invariant to a per-row shift: rows riding on offsets of thousands (where the
+    # spacing of the I/O type is far coarser than near zero) must still match the oracle.  The
+    # offsets are exactly representable, so the shifted logits are too where they fit the type.
+    rows = 320
+    z = synth.normal(5, ("off", L, dt), rows * L).reshape(rows, L)
+    step = np.float32(32.0 if dt == BF16 else 0.25)       # a multiple of the spacing at the offsets used
+    offs = np.array([0, 1024, -2048, 4096, -4096, 3072, 512, -1536], dtype=np.float32)
+    x = np.round(z * np.float32(2.0)) * step + offs[np.arange(rows) % offs.size, None]
+    g = synth.normal(5, ("offg", L, dt), rows * L)
+    check_softmax(synth.to_io(x.reshape(-1).astype(np.float32), dt), synth.to_io(g, dt), L, dt, max_flip_frac=5e-3)
+
+
 def test_gelu_saturated_row_hand_codes():
     # bin edges of a [-2, 2] row; 0 is the exact tie 7.5 and must round to 8
     row = np.array([-3, -2, -1, -0.1333333, 0, 0.1333334, 0.5, 1, 2, 2.5], dtype=np.float32)
