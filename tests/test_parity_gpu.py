@@ -354,6 +354,41 @@ def test_other_bit_widths(kind, rows, L, bits, dt):
         assert np.array_equal(c4, codes_g) and np.array_equal(m4, meta_g) and np.array_equal(y4, y_g)
 
 
+@pytest.mark.parametrize("dt", [F32, BF16])
+@pytest.mark.parametrize("bits", [2, 8])
+@pytest.mark.parametrize("kind,L", [("gelu", 3072), ("softmax", 197), ("softmax", 1024)])
+def test_other_bit_widths_degenerate_rows(kind, L, bits, dt):
+    # constant rows (max == min: codes 0, s = 0), rows beyond the clip, one-hot rows
+    rows = 130
+    x = synth.normal(9, ("bdeg", kind, L), rows * L).reshape(rows, L).astype(np.float32)
+    x[1] = 0.37
+    x[2] = -5.0
+    x[3] = 7.0
+    x[4] = 0.0
+    x[4, 5] = 30.0
+    x[5, ::2] = 80.0
+    x[5, 1::2] = -80.0
+    n = rows * L
+    xi = synth.to_io(x.reshape(-1), dt)
+    y_o, codes_o, meta_o = o.fwd_bits(kind, xi, L, bits, dt)
+    tdt = pu.torch_dtype(dt)
+    yg, cg, mg = pu.Guarded(n * synth.io_itemsize(dt)), pu.Guarded(binding.codes_bytes_bits(n, bits)), pu.Guarded(binding.meta_bytes(n, L))
+    binding.s2a_fwd_bits(kind, pu.to_device(xi, dt), yg.view(tdt), cg.view(torch.uint8), mg.view(torch.float32), L, bits)
+    torch.cuda.synchronize()
+    for buf, what in ((yg, "y"), (cg, "codes"), (mg, "meta")):
+        buf.check("%s bits=%d %s" % (kind, bits, what))
+    meta_g = mg.view(torch.float32).cpu().numpy()
+    q_g = o.unpack_bits(cg.view(torch.uint8).cpu().numpy(), n, bits).reshape(rows, L)
+    q_o = o.unpack_bits(codes_o, n, bits).reshape(rows, L)
+    for r in (1, 2, 3):  # constant rows
+        assert meta_g[2 * r + 1] == 0.0 and not q_g[r].any()
+    if kind == "gelu":
+        assert np.array_equal(q_g, q_o) and np.array_equal(meta_g.view(np.uint32), meta_o.view(np.uint32))
+    else:
+        assert q_g[4].max() == 2 ** bits - 1 and int((q_g[4] != 0).sum()) == 1   # one-hot row
+        assert np.abs(q_g.astype(int) - q_o.astype(int)).max() <= 1
+
+
 def test_other_bit_widths_reject_unsupported_values():
     L = binding.lib()
     x = torch.zeros(64, device="cuda")
