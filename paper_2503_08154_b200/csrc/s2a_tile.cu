@@ -20,7 +20,8 @@ cudaError_t launch_tile_pair_widths(int kernel, int dt, const TilePlan& p, const
 namespace {
 
 constexpr uint32_t kMaxStageBytes = 56 * 1024;   // tiles are not grown beyond this
-constexpr uint32_t kHardStageBytes = 96 * 1024;  // the smallest legal tile may be this large (one CTA per SM then)
+constexpr uint32_t kHardStageBytes = 176 * 1024;  // the smallest legal tile may be this large (one CTA per SM,
+                                                  // and a single stage beyond ~96 KB)
 
 int env_int(const char* name, int dflt) {
   const char* v = getenv(name);
@@ -251,6 +252,14 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
     if (fit > 4) fit = 4;
     if (env_stages > 0 && (uint32_t)env_stages <= fit) fit = (uint32_t)env_stages;
     if (fit >= 2) { stages = fit; ctas_per_sm = c; smem = budget; }
+  }
+  if (stages == 0 && env_int("S2A_SINGLE_STAGE", 1) != 0) {
+    // A tile too large to double-buffer: one CTA per SM with a single stage.  Load, row work
+    // and store of a CTA then run one after the other, but the SMs drift out of step and
+    // keep the memory system busy between them -- still well ahead of the row-at-a-time path.
+    const uint32_t budget = kMaxSmem - 1024;
+    const uint32_t fixed = kHeaderBytes + (bits == 8 ? n_units * 1024u : 0u);
+    if (budget > fixed && stage_bytes <= budget - fixed) { stages = 1; ctas_per_sm = 1; smem = budget; }
   }
   if (stages == 0) return p;
 

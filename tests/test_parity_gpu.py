@@ -89,7 +89,8 @@ SOFTMAX_SHAPES = [(7, 1), (4, 2), (5, 3), (33, 63), (701, 63), (77, 64), (1001, 
                   # widths that are not whole 16-byte vectors (masked vector ends), tiles + ragged tails
                   (90, 17), (2049, 49), (1500, 50), (999, 145), (641, 198), (333, 577), (163, 1025),
                   (1100, 196), (37, 16384), (300, 40), (513, 56), (2000, 48),
-                  (700, 401), (300, 785), (200, 1370), (1500, 100), (901, 33), (350, 255)]
+                  (700, 401), (300, 785), (200, 1370), (1500, 100), (901, 33), (350, 255),
+                  (170, 2049), (9000, 1025)]   # tiles too large to double-buffer: a single stage
 
 
 @pytest.mark.parametrize("dt", [F32, BF16])
@@ -287,7 +288,9 @@ def test_silu(rows, L, dt):
         gin_g = pu.gpu_bwd("silu", g, codes_o, meta_o, L, dt, inplace=inplace)
         pu.assert_close(pu.widen(gin_g, dt), pu.widen(gin_o, dt), dt, "silu grad_in")
     plan = binding.s2a_describe_plan(binding.SILU_FWD, n, L, dt)
-    assert plan.startswith("tile") == (L % (4 if dt == F32 else 8) == 0 and rows >= 2 and L <= 8192), plan
+    # pipelined whenever rows are whole 16-byte vectors and two of them fit a shared-memory stage
+    fits = 2 * L * synth.io_itemsize(dt) <= 176 * 1024
+    assert plan.startswith("tile") == (L % (4 if dt == F32 else 8) == 0 and rows >= 2 and fits), plan
 
 
 # ------------------------------------------------------------------ other bit widths (Eq. 8, general N)
