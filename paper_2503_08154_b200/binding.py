@@ -120,8 +120,17 @@ def check(status: int) -> None:
         raise S2AError(status_string(status))
 
 
-def _stream_ptr() -> int:
-    return torch.cuda.current_stream().cuda_stream
+_raw_stream = getattr(torch._C, "_cuda_getCurrentRawStream", None)
+
+
+def _stream_ptr(t: torch.Tensor = None) -> int:
+    """The current CUDA stream of the tensor's device (of the current device without one) as
+    a raw handle.  torch's raw-stream query is several times cheaper than building a Stream
+    object on every call; the slower public route is the fallback."""
+    if _raw_stream is not None:
+        idx = t.device.index if t is not None and t.device.index is not None else torch.cuda.current_device()
+        return _raw_stream(idx)
+    return torch.cuda.current_stream(t.device if t is not None else None).cuda_stream
 
 
 def _dev(t: torch.Tensor, what: str) -> torch.Tensor:
@@ -149,7 +158,7 @@ def _fwd(fn, x, y, codes, meta, row_len):
     if row_len > 0 and (codes.numel() < codes_bytes(n) or meta.numel() * 4 < meta_bytes(n, row_len)):
         raise S2AError("codes/meta buffers are too small")
     check(fn(x.data_ptr(), y.data_ptr(), codes.data_ptr(), meta.data_ptr(), n, row_len,
-             dtype_code(x), _stream_ptr()))
+             dtype_code(x), _stream_ptr(x)))
 
 
 def _bwd(fn, grad_out, codes, meta, grad_in, row_len):
@@ -162,7 +171,7 @@ def _bwd(fn, grad_out, codes, meta, grad_in, row_len):
     if row_len > 0 and (codes.numel() < codes_bytes(n) or meta.numel() * 4 < meta_bytes(n, row_len)):
         raise S2AError("codes/meta buffers are too small")
     check(fn(grad_out.data_ptr(), codes.data_ptr(), meta.data_ptr(), grad_in.data_ptr(), n,
-             row_len, dtype_code(grad_out), _stream_ptr()))
+             row_len, dtype_code(grad_out), _stream_ptr(grad_out)))
 
 
 def s2a_gelu_fwd(x, y, codes, meta, row_len: int) -> None:
@@ -207,7 +216,7 @@ def s2a_gelu_fwd_tensor_range(x, y, codes, meta, scratch, row_len: int) -> None:
     if scratch.numel() * scratch.element_size() < tensor_range_scratch_bytes(n):
         raise S2AError("scratch is too small")
     check(lib().s2a_gelu_fwd_tensor_range(x.data_ptr(), y.data_ptr(), codes.data_ptr(), meta.data_ptr(),
-                                          scratch.data_ptr(), n, row_len, dtype_code(x), _stream_ptr()))
+                                          scratch.data_ptr(), n, row_len, dtype_code(x), _stream_ptr(x)))
 
 
 def tensor_range_static_max_elems() -> int:
@@ -228,14 +237,14 @@ def s2a_gelu_fwd_tensor_range_static(x, y, codes, meta, row_len: int) -> None:
     if row_len > 0 and (codes.numel() < codes_bytes(n) or meta.numel() * 4 < meta_bytes(n, row_len)):
         raise S2AError("codes/meta buffers are too small")
     check(lib().s2a_gelu_fwd_tensor_range_static(x.data_ptr(), y.data_ptr(), codes.data_ptr(), meta.data_ptr(),
-                                                 n, row_len, dtype_code(x), _stream_ptr()))
+                                                 n, row_len, dtype_code(x), _stream_ptr(x)))
 
 
 def s2a_cap_fwd(x, y, n_rows: int, channels: int, r: int) -> None:
     _dev(x, "x"), _dev(y, "y")
     if x.numel() != n_rows * channels or r <= 0 or y.numel() * r != x.numel() or y.dtype != x.dtype:
         raise S2AError("x must be [n_rows, channels] and y [n_rows, channels / r] of the same dtype")
-    check(lib().s2a_cap_fwd(x.data_ptr(), y.data_ptr(), n_rows, channels, r, dtype_code(x), _stream_ptr()))
+    check(lib().s2a_cap_fwd(x.data_ptr(), y.data_ptr(), n_rows, channels, r, dtype_code(x), _stream_ptr(x)))
 
 
 def s2a_cap_bwd(grad_out, grad_in, n_rows: int, channels: int, r: int) -> None:
@@ -254,7 +263,7 @@ def s2a_lrp_fwd(x, A, B, y, batch: int, tokens: int, channels: int, rank: int) -
     if A.dtype != torch.float32 or B.dtype != torch.float32 or A.numel() != tokens * rank or B.numel() != rank * channels:
         raise S2AError("A must be float32 [tokens, rank] and B float32 [rank, channels]")
     check(lib().s2a_lrp_fwd(x.data_ptr(), A.data_ptr(), B.data_ptr(), y.data_ptr(), batch, tokens, channels, rank,
-                            dtype_code(x), _stream_ptr()))
+                            dtype_code(x), _stream_ptr(x)))
 
 
 def codes_bytes_bits(n_elems: int, bits: int) -> int:
@@ -296,7 +305,7 @@ def s2a_relu_fwd(x, y, mask) -> None:
         raise S2AError("y must match x in size and dtype")
     if mask.dtype != torch.uint8 or mask.numel() < mask_bytes(n):
         raise S2AError("mask must be uint8 with at least mask_bytes(n) elements")
-    check(lib().s2a_relu_fwd(x.data_ptr(), y.data_ptr(), mask.data_ptr(), n, dtype_code(x), _stream_ptr()))
+    check(lib().s2a_relu_fwd(x.data_ptr(), y.data_ptr(), mask.data_ptr(), n, dtype_code(x), _stream_ptr(x)))
 
 
 def s2a_relu_bwd(grad_out, mask, grad_in) -> None:

@@ -86,6 +86,10 @@ __global__ void __launch_bounds__(kThreads) rowwise_kernel(RowwiseArgs a) {
   while ((P * (uint64_t)L) % EPB != 0) P *= 2;
   const uint64_t n_groups = (a.n_rows + P - 1) / P;
   const int tid = threadIdx.x % TEAM;
+  // Launched with programmatic stream serialization: let the next kernel of the stream set
+  // up while this one runs, and touch no global memory before the previous one has finished.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 
   for (uint64_t g = (uint64_t)blockIdx.x * kTeams + team; g < n_groups; g += (uint64_t)gridDim.x * kTeams) {
     const uint64_t r0 = a.row0 + g * P;
@@ -195,9 +199,17 @@ cudaError_t launch_one(const RowwiseArgs& a, cudaStream_t st) {
   const bool warp_teams = (uint64_t)P * a.row_len <= 2048;
   const uint64_t ctas = warp_teams ? (groups + kWarps - 1) / kWarps : groups;
   const unsigned grid = (unsigned)(ctas < (1ull << 20) ? ctas : (1ull << 20));
-  if (warp_teams) rowwise_kernel<KERNEL, DT, NBITS, 32><<<grid, kThreads, 0, st>>>(a);
-  else rowwise_kernel<KERNEL, DT, NBITS, kThreads><<<grid, kThreads, 0, st>>>(a);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kThreads);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (warp_teams) return cudaLaunchKernelEx(&cfg, rowwise_kernel<KERNEL, DT, NBITS, 32>, a);
+  return cudaLaunchKernelEx(&cfg, rowwise_kernel<KERNEL, DT, NBITS, kThreads>, a);
 }
 
 template <int KERNEL, int DT>
