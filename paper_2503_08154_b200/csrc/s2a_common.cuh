@@ -97,7 +97,13 @@ __device__ __forceinline__ float act_value(float x) {
   float z = __fmul_rn(a, x);
   float zlo = __fmaf_rn(a, x, -z);
   float t = expf(-fabsf(z)) * (1.0f - (z >= 0.0f ? zlo : -zlo));
-  return __fdiv_rn(z >= 0.0f ? x : x * t, 1.0f + t);
+  // a / b with b = 1 + t in [1, 2]: the hardware reciprocal (1 ulp) and one correction step
+  // on the remainder, which leaves about an ulp -- no special cases can arise for such b
+  const float a_num = z >= 0.0f ? x : x * t, b_den = 1.0f + t;
+  float r;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(b_den));
+  const float q = a_num * r;
+  return __fmaf_rn(__fmaf_rn(-b_den, q, a_num), r, q);
 }
 __device__ __forceinline__ float gelu_value(float x) { return act_value<kActGelu>(x); }
 
