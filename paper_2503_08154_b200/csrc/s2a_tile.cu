@@ -191,8 +191,9 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
   if (variant == kVariantStream && !is_gelu) {
     // A softmax row is a chain of dependent phases (reduce, evaluate, reduce, ...).  With few
     // elements per lane, or the cheaper bfloat16 arithmetic, four warps leave the SM waiting
-    // on shuffles; binary32 rows with 32 elements per lane run best with four (measured).
-    warps = (dt == kBF16 || iters * epa <= 16) ? 8u : 4u;
+    // on shuffles; binary32 rows with 32 elements per lane run best with four, except the
+    // one-warp units of 1024-element rows (measured at 512, 1024, 2048 and 4096).
+    warps = (dt == kBF16 || iters * epa <= 16 || unit == 32) ? 8u : 4u;
   }
   int ctas_per_sm = 2;
   if (variant == kVariantStream && is_gelu) ctas_per_sm = 4;

@@ -356,9 +356,11 @@ __device__ __forceinline__ RowGeom row_geom(uint32_t r, uint32_t L) {
   return g;
 }
 
+// e^d for d = x - max <= 0.  One multiply and the hardware 2^x (2 ulp): the rounding of the
+// product moves the result by at most 2^-24 |d| relative, which is the allowance the softmax
+// output carries for the rounding of its exponent's argument.
 template <int DT>
-__device__ __forceinline__ float exp_eval(float d) {  // d <= 0
-  if (DT == kF32) return expf(d);
+__device__ __forceinline__ float exp_eval(float d) {
   return ex2_approx(1.4426950408889634f * d);
 }
 
