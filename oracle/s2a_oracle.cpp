@@ -491,16 +491,14 @@ void s2a_oracle_unpack_bits(const uint8_t* bytes, size_t n, int bits, uint8_t* q
 // ---- Quantise an already materialised tensor row by row (Eq. 8 + packing); lets a
 // test check that stored codes are exactly Q(values as written).
 int s2a_oracle_quantize_tensor(const void* v, uint8_t* codes, float* meta, size_t n, size_t L,
-                               int dt, int clip_to_2, int threads) {
+                               int dt, int threads) {
   if (n == 0) return 0;
   if (bad_shape(n, L)) return 2;
   std::vector<uint8_t> q(n);
   for_rows(n / L, threads, [&](size_t r) {
     std::vector<float> c(L);
     for (size_t i = 0; i < L; ++i) {
-      double vi = load_elem(v, r * L + i, dt);
-      if (clip_to_2) vi = std::min(std::max(vi, -2.0), 2.0);
-      c[i] = (float)vi;
+      c[i] = (float)load_elem(v, r * L + i, dt);
     }
     quantize_row(c.data(), L, &q[r * L], &meta[2 * r], &meta[2 * r + 1]);
   });

@@ -86,7 +86,7 @@ def lib() -> ctypes.CDLL:
         L.s2a_oracle_pack_bits.restype = None
         L.s2a_oracle_unpack_bits.argtypes = [vp, sz, i32, vp]
         L.s2a_oracle_unpack_bits.restype = None
-        L.s2a_oracle_quantize_tensor.argtypes = [vp, vp, vp, sz, sz, i32, i32, i32]
+        L.s2a_oracle_quantize_tensor.argtypes = [vp, vp, vp, sz, sz, i32, i32]
         L.s2a_oracle_quantize_tensor.restype = i32
         L.s2a_oracle_relu_fwd.argtypes = [vp, vp, vp, sz, i32]
         L.s2a_oracle_relu_fwd.restype = i32
@@ -371,14 +371,13 @@ def bwd_bits(kind: str, g, codes, meta, row_len: int, bits: int, dt: int):
     return gin
 
 
-def quantize_tensor(v, row_len: int, dt: int, clip_to_2: bool = False, threads: int = 1):
+def quantize_tensor(v, row_len: int, dt: int, threads: int = 1):
     """Eq. 8 + packing over an existing tensor.  Returns (packed codes, meta)."""
     v = _check_io(v, dt).reshape(-1)
     n = v.size
     codes = np.zeros(codes_bytes(n), dtype=np.uint8)
     meta = np.zeros(2 * (n // row_len), dtype=np.float32)
-    rc = lib().s2a_oracle_quantize_tensor(_ptr(v), _ptr(codes), _ptr(meta), n, row_len, dt,
-                                          int(clip_to_2), threads)
+    rc = lib().s2a_oracle_quantize_tensor(_ptr(v), _ptr(codes), _ptr(meta), n, row_len, dt, threads)
     if rc != 0:
         raise ValueError("oracle rejected the shape")
     return codes, meta

@@ -120,13 +120,28 @@ __device__ __forceinline__ float rcp_approx(float x) {
   return y;
 }
 
+// y = x / (1 + 2^k), k = -a log2(e) x.  Both forms below are for bfloat16 outputs.
+//
+// The short form is exact enough while 2^k is finite and 1 / 2^k is a normal number, i.e.
+// for k <= 126 (x >= kFastFloor): beyond that ex2.approx returns +inf (or rcp.approx.ftz
+// flushes a subnormal reciprocal) and y would come out as -0 although its true magnitude,
+// |x| 2^-k, is still a normal bfloat16 number down to k = 126 + log2|x|.  Callers use it
+// only on rows whose minimum is at or above kFastFloor.
+template <int ACT>
+struct ActFast {
+  static constexpr float kC = -Act<ACT>::kSlopeOf * 1.4426950408889634f;
+  static constexpr float kFastFloor = -125.0f / (Act<ACT>::kSlopeOf * 1.4426950408889634f);
+  static __device__ __forceinline__ float eval(float x) { return x * rcp_approx(1.0f + ex2_approx(kC * x)); }
+};
+
+// The general form carries the denominator scaled by 2^-8: 2^-8 + 2^(k-8) stays finite, and
+// its reciprocal normal, up to k = 134; from there on |y| = |x| 2^-k is below 2^-126 (k = 134
+// is reached at |x| = 92.9 / a), so only results below the normal range flush to zero.
 template <int DT, int ACT = kActGelu>
 __device__ __forceinline__ float gelu_eval(float x) {
   if (DT == kF32) return act_value<ACT>(x);
-  // y = x / (1 + 2^(-1.702 log2(e) x)).  For x < -52 the power overflows and y becomes
-  // -0 instead of a value below 2^-120: the bfloat16 path flushes such results.
-  constexpr float c = -Act<ACT>::kSlopeOf * 1.4426950408889634f;
-  return x * rcp_approx(1.0f + ex2_approx(c * x));
+  const float w = 0.00390625f + ex2_approx(__fmaf_rn(ActFast<ACT>::kC, x, -8.0f));
+  return (x * rcp_approx(w)) * 0.00390625f;
 }
 
 // The derivative used by the backward pass at a dequantised x_hat = code * s + min, in

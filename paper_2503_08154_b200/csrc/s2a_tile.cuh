@@ -708,6 +708,9 @@ struct StreamActFwd {
   static __device__ __forceinline__ void init(State&) {}
   static __device__ __forceinline__ uint32_t rows_per_group(uint32_t) { return 1u; }
 
+  // FAST: the short bfloat16 form of the activation, valid on rows with no element below
+  // ActFast::kFastFloor (the caller knows the row minimum before the second pass).
+  template <bool FAST>
   static __device__ __forceinline__ void vec(unsigned char* row, unsigned char* crow, uint32_t j, const QRange& q) {
     float v[V::EPA];
     V::widen(*(const typename V::Raw*)(row + j * 16u), v);
@@ -716,10 +719,25 @@ struct StreamActFwd {
 #pragma unroll
     for (int k = 0; k < V::EPA; ++k) {
       pk.add(k, fminf(fmaxf(v[k], -kActClip), kActClip), q);
-      v[k] = gelu_eval<DT, ACT>(v[k]);
+      v[k] = FAST ? ActFast<ACT>::eval(v[k]) : gelu_eval<DT, ACT>(v[k]);
     }
     *(typename V::Raw*)(row + j * 16u) = V::narrow(v);
     V::store_codes(crow, j, pk.acc);
+  }
+  template <bool FAST>
+  static __device__ __forceinline__ void second_pass(unsigned char* row, unsigned char* crow, int ul, uint32_t nv,
+                                                     const QRange& q) {
+    if (DT == kBF16 && !FAST) {
+      // the rare rows with an element below the short form's range: kept rolled and small
+#pragma unroll 1
+      for (uint32_t j = ul; j < nv; j += UNIT_) vec<false>(row, crow, j, q);
+    } else if (NVL > 0) {
+#pragma unroll
+      for (int i = 0; i < NVL; ++i) vec<FAST>(row, crow, ul + UNIT_ * i, q);
+    } else {
+#pragma unroll 2
+      for (uint32_t j = ul; j < nv; j += UNIT_) vec<FAST>(row, crow, j, q);
+    }
   }
 
   static __device__ __forceinline__ void group(Unit<UNIT_>& u, State&, const StagePtrs& p, float*, uint32_t r,
@@ -742,13 +760,9 @@ struct StreamActFwd {
     // min / max of the clipped row = clipped min / max of the row (the clip is monotone)
     const QRange q = make_qrange(fminf(fmaxf(mn, -kActClip), kActClip), fminf(fmaxf(mx, -kActClip), kActClip));
     if (active && u.ul == 0) { p.meta[2 * r] = q.mn; p.meta[2 * r + 1] = q.s; }
-    if (NVL > 0) {
-#pragma unroll
-      for (int i = 0; i < NVL; ++i) vec(row, crow, u.ul + UNIT_ * i, q);
-    } else {
-#pragma unroll 2
-      for (uint32_t j = u.ul; j < nv; j += UNIT_) vec(row, crow, j, q);
-    }
+    // mn is the same in every lane of the unit, so the branch does not diverge
+    if (DT == kBF16 && mn >= ActFast<ACT>::kFastFloor) second_pass<true>(row, crow, u.ul, nv, q);
+    else second_pass<false>(row, crow, u.ul, nv, q);
   }
 };
 

@@ -9,12 +9,18 @@ Tolerances (all written out here, used by every parity test):
   tolerance, and may differ from the oracle's codes only where the GPU's y (or the
   row's min/max) differs from the oracle's by its allowed rounding -- such elements sit
   within one ulp of a bin edge; they are counted and the count is bounded.
-* binary32 outputs: |a - b| <= rtol * (|b| + M) + 2^-120 with rtol = 1e-6 (results below
-  2^-120 in magnitude may be flushed to zero).  M is 0
+* binary32 outputs: |a - b| <= rtol * (|b| + M) + 2^-126 with rtol = 1e-6 (results below
+  the normal range, 2^-126, may be flushed to zero).  M is 0
   except for the softmax VJP, where it is y_hat_i * sum_j |g_j| y_hat_j (the size of the
   terms that cancel in g_i - dot), and for softmax y, where rtol is widened by
   2^-24 * |x_i - max_j x_j| (the rounding of the exponent's argument).
-* bfloat16 outputs: within 1 bfloat16 ulp of max(|b|, M), plus the same 2^-120 floor.
+* bfloat16 outputs: within 1 bfloat16 ulp of max(|b|, M), plus the same 2^-126 floor.
+* softmax codes against the ORACLE's codes: an element's code may differ only if the oracle's
+  scaled value t = (y - min) * 15 / (max - min), evaluated in binary64 from the oracle's own
+  y, lies within B of a bin edge k + 1/2, where B is what the tolerances above allow y, min
+  and max to move t by: B = inv * (tol(y_i) + (1 - t/15) tol(min) + (t/15) tol(max)) plus
+  1e-5 for the binary32 evaluation of t.  Every such element is counted; the count, the worst
+  distance as a fraction of B, and the worst distance in units of ulp(y_i) * inv are reported.
 """
 from __future__ import annotations
 
@@ -24,6 +30,7 @@ import torch
 from paper_2503_08154_b200 import binding, synth
 
 F32, BF16 = 0, 1
+FLOOR = 2.0 ** -126  # the smallest normal binary32 / bfloat16 magnitude: results below it may flush
 GUARD = 512  # bytes of canary on each side of every output buffer
 CANARY = 0xA5
 
@@ -147,19 +154,26 @@ def bf16_ulp(mag: np.ndarray) -> np.ndarray:
     return np.exp2(np.floor(np.log2(mag)) - 7)
 
 
-def assert_close(got, want, dt, what, extra_mag=None, extra_rtol=None):
-    """got/want: float64 arrays of widened outputs.  See the module docstring."""
-    got = np.asarray(got, dtype=np.float64).reshape(-1)
+def tolerance(want, dt, extra_mag=None, extra_rtol=None):
+    """The allowed |got - want| per element (see the module docstring); want is float64."""
     want = np.asarray(want, dtype=np.float64).reshape(-1)
     mag = np.abs(want) if extra_mag is None else np.abs(want) + np.asarray(extra_mag).reshape(-1)
     if dt == F32:
         rtol = 1e-6 if extra_rtol is None else 1e-6 + np.asarray(extra_rtol).reshape(-1)
-        tol = rtol * mag + 2.0 ** -120
+        tol = rtol * mag + FLOOR
     else:
         ref = np.abs(want) if extra_mag is None else np.maximum(np.abs(want), np.asarray(extra_mag).reshape(-1))
-        tol = bf16_ulp(ref) + 2.0 ** -120
+        tol = bf16_ulp(ref) + FLOOR
         if extra_rtol is not None:
             tol = tol + np.asarray(extra_rtol).reshape(-1) * mag
+    return tol, mag
+
+
+def assert_close(got, want, dt, what, extra_mag=None, extra_rtol=None):
+    """got/want: float64 arrays of widened outputs.  See the module docstring."""
+    got = np.asarray(got, dtype=np.float64).reshape(-1)
+    want = np.asarray(want, dtype=np.float64).reshape(-1)
+    tol, mag = tolerance(want, dt, extra_mag, extra_rtol)
     err = np.abs(got - want)
     bad = err > tol
     if bad.any():
@@ -167,3 +181,48 @@ def assert_close(got, want, dt, what, extra_mag=None, extra_rtol=None):
         raise AssertionError("%s: %d of %d outside tolerance; worst at %d: got %r want %r tol %r"
                              % (what, int(bad.sum()), got.size, i, got[i], want[i], tol[i]))
     return float(np.max(err / np.maximum(mag, 1e-300)))
+
+
+def ulp_of(v, dt):
+    """Spacing of the I/O type at |v| (float64 in, float64 out)."""
+    if dt == BF16:
+        return bf16_ulp(v)
+    a = np.maximum(np.abs(np.asarray(v, dtype=np.float64)), 2.0 ** -126)
+    return np.exp2(np.floor(np.log2(a)) - 23)
+
+
+def check_edge_flips(q_got, q_want, y_want, meta_want, tol_y, dt, levels=15, what="softmax"):
+    """Code differences against the oracle (see the module docstring).  q_*: unpacked codes
+    [rows, L]; y_want: the oracle's y widened to float64 [rows, L]; meta_want: the oracle's
+    (min, s) float32 [2 * rows]; tol_y: allowed |y_got - y_want| per element [rows, L].
+    Returns {"flips", "elements", "worst_frac_of_bound", "worst_ulps"}."""
+    rows, L = q_want.shape
+    diff = q_got != q_want
+    out = {"flips": int(diff.sum()), "elements": int(q_want.size), "worst_frac_of_bound": 0.0, "worst_ulps": 0.0}
+    if not diff.any():
+        return out
+    assert np.abs(q_got.astype(int) - q_want.astype(int)).max() <= 1, "%s: a code differs by more than one level" % what
+    r, c = np.nonzero(diff)
+    yw = np.asarray(y_want, dtype=np.float64).reshape(rows, L)
+    tol_y = np.asarray(tol_y, dtype=np.float64).reshape(rows, L)
+    mn = meta_want[0::2].astype(np.float64)
+    # the row maximum as the oracle saw it (s is rounded, so take max from y itself)
+    amin, amax = yw.argmin(axis=1), yw.argmax(axis=1)
+    mx = yw[np.arange(rows), amax]
+    assert np.array_equal(yw[np.arange(rows), amin], mn), "oracle metadata is not the row minimum"
+    d = (mx - mn)[r]
+    assert (d > 0).all(), "%s: a constant row has differing codes" % what
+    inv = levels / d
+    t = (yw[r, c] - mn[r]) * inv
+    dist = np.abs((t - np.floor(t)) - 0.5)
+    w = t / levels
+    bound = inv * (tol_y[r, c] + (1.0 - w) * tol_y[r, amin[r]] + w * tol_y[r, amax[r]]) + 1e-5
+    frac = dist / bound
+    if (frac > 1.0).any():
+        i = int(np.argmax(frac))
+        raise AssertionError("%s: code differs at row %d col %d although the oracle's t = %.9g is %.3g from a bin "
+                             "edge (allowed %.3g): codes %d vs %d" % (what, r[i], c[i], t[i], dist[i], bound[i],
+                                                                      q_got[r[i], c[i]], q_want[r[i], c[i]]))
+    out["worst_frac_of_bound"] = float(frac.max())
+    out["worst_ulps"] = float((dist / (inv * ulp_of(yw[r, c], dt))).max())
+    return out
