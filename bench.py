@@ -49,6 +49,8 @@ def parse_args():
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--repeats", type=int, default=0,
+                    help="how many times the K-step timed region is repeated (0: at least 5, and enough for about a second)")
     return ap.parse_args()
 
 
@@ -189,39 +191,87 @@ def stored_traffic(kernel, workload):
 # ------------------------------------------------------------------ the CPU oracle legs
 def oracle_time_block(shape, arrays, threads):
     """Forward+backward of both nonlinearities through the oracle on one block's arrays.
-    Returns (algorithmic bytes, elements, seconds)."""
+    Returns (algorithmic bytes, elements, seconds, forward results)."""
     from oracle import s2a_oracle as o
     gx, gg, sx, sg = arrays
     item = synth.io_itemsize(shape.dtype)
     t0 = time.perf_counter()
-    y, c, m = o.gelu_fwd(gx, shape.hidden, shape.dtype, threads)
-    o.gelu_bwd(gg, c, m, shape.hidden, shape.dtype, threads)
+    gy, gc, gm = o.gelu_fwd(gx, shape.hidden, shape.dtype, threads)
+    o.gelu_bwd(gg, gc, gm, shape.hidden, shape.dtype, threads)
     nbytes = 2 * algorithmic_bytes(gx.size, shape.hidden, item)
     nelem = gx.size
+    fwd = {"gelu": (gy, gc, gm)}
     if sx is not None:
-        y, c, m = o.softmax_fwd(sx, shape.tokens, shape.dtype, threads)
-        o.softmax_bwd(sg, c, m, shape.tokens, shape.dtype, threads)
+        sy, sc, sm = o.softmax_fwd(sx, shape.tokens, shape.dtype, threads)
+        o.softmax_bwd(sg, sc, sm, shape.tokens, shape.dtype, threads)
         nbytes += 2 * algorithmic_bytes(sx.size, shape.tokens, item)
         nelem += sx.size
-    return nbytes, nelem, time.perf_counter() - t0
+        fwd["softmax"] = (sy, sc, sm)
+    return nbytes, nelem, time.perf_counter() - t0, fwd
 
 
-def oracle_sample_rate(shape, blocks_arrays, threads, core_seconds=12.0):
+def oracle_sample_rate(shape, blocks_arrays, threads, core_seconds=12.0, on_block=None):
     """Times the oracle, as it stands, on whole blocks of the workload until about
-    `core_seconds` of CPU work (threads x wall time) have been spent."""
+    `core_seconds` of CPU work (threads x wall time) have been spent.  on_block(index, forward
+    results) is called outside the timed part (the parity counts of the benchmark line)."""
     from oracle import s2a_oracle as o
     o.lib()
     nbytes = nelem = 0
     secs = 0.0
     used = 0
-    for arrays in blocks_arrays:
-        b, e, t = oracle_time_block(shape, arrays, threads)
+    for i, arrays in enumerate(blocks_arrays):
+        b, e, t, fwd = oracle_time_block(shape, arrays, threads)
         nbytes, nelem, secs, used = nbytes + b, nelem + e, secs + t, used + 1
+        if on_block is not None:
+            on_block(i, arrays, fwd)
+        del fwd
         if secs * threads >= core_seconds:
             break
     sample = "fwd+bwd of GELU%s on %d of the workload's blocks, full size (%.1f core-seconds)" % (
         " and softmax" if blocks_arrays[0][2] is not None else "", used, secs * threads)
     return nbytes / secs / 1e9, nelem / secs / 1e9, secs, sample
+
+
+# ------------------------------------------------------------------ parity counts for the line
+def _unpack4(codes, n):
+    q = np.empty(2 * codes.size, dtype=np.uint8)
+    q[0::2], q[1::2] = codes & 0xF, codes >> 4
+    return q[:n]
+
+
+def softmax_code_flips(codes_gpu, y_oracle, codes_oracle, x, L, dt):
+    """Elements whose 4-bit code differs from the oracle's, and how many of them are NOT within
+    reach of a bin edge.  Reach: what the output tolerance (1 bfloat16 ulp; 1e-6 relative plus
+    2^-24 |x_i - max x| in binary32) allows the oracle's scaled value t = (y - min) 15 / (max - min)
+    to move by, through y_i, the row minimum and the row maximum, plus 1e-5."""
+    n = y_oracle.size
+    rows = n // L
+    qg, qo = _unpack4(codes_gpu, n), _unpack4(codes_oracle, n)
+    flip = np.nonzero(qg != qo)[0]
+    if flip.size == 0:
+        return 0, 0
+    yo = synth.io_to_f32(y_oracle, dt).astype(np.float64).reshape(rows, L)
+    xw = synth.io_to_f32(x, dt).astype(np.float64).reshape(rows, L)
+    r, c = flip // L, flip % L
+    rows_hit = np.unique(r)
+    amin = dict(zip(rows_hit, yo[rows_hit].argmin(axis=1)))
+    amax = dict(zip(rows_hit, yo[rows_hit].argmax(axis=1)))
+    cmin = np.array([amin[k] for k in r])
+    cmax = np.array([amax[k] for k in r])
+
+    def tol(rr, cc):
+        v = yo[rr, cc]
+        if dt == synth.BF16:
+            return np.exp2(np.floor(np.log2(np.maximum(np.abs(v), 2.0 ** -126))) - 7)
+        return (1e-6 + 2.0 ** -24 * (xw[rr].max(axis=1) - xw[rr, cc])) * np.abs(v)
+
+    mn, mx = yo[r, cmin], yo[r, cmax]
+    inv = 15.0 / (mx - mn)
+    t = (yo[r, c] - mn) * inv
+    w = t / 15.0
+    reach = inv * (tol(r, c) + (1 - w) * tol(r, cmin) + w * tol(r, cmax)) + 1e-5
+    outside = (np.abs(t - np.floor(t) - 0.5) > reach) | (np.abs(qg[flip].astype(int) - qo[flip].astype(int)) > 1)
+    return int(flip.size), int(outside.sum())
 
 
 def run_reference(args, shape, blocks):
@@ -296,14 +346,19 @@ def run_ours(args, shape, blocks, rank, world):
     def dview(t):
         return t.view(tdt) if tdt == torch.bfloat16 else t
 
+    # Distinct buffer sets, rotated step by step, so that what is touched between two uses of
+    # the same buffer is several times the L2 (a workload of one small block would otherwise
+    # run out of the cache).  The large workloads need one set.
+    touched = blocks * (4 * item + 1) * (shape.gelu_elems + (shape.softmax_elems if has_softmax else 0))
+    sets = max(1, -(-3 * L2_BYTES // touched))
     host = [tuple(pin(a) if a is not None else None for a in blk) for blk in host_inputs(
-        shape, blocks, args.seed + 1000 * rank, with_softmax=has_softmax)]
+        shape, blocks * sets, args.seed + 1000 * rank, with_softmax=has_softmax)]
 
     class Block:
         pass
 
     blks = []
-    for b in range(blocks):
+    for b in range(blocks * sets):
         B = Block()
         gx, gg, sx, sg = host[b]
         B.gx, B.gg = dview(gx.to(dev)), dview(gg.to(dev))
@@ -321,22 +376,29 @@ def run_ours(args, shape, blocks, rank, world):
     ng, Lg = shape.gelu_elems, shape.hidden
     ns, Ls = shape.softmax_elems, shape.tokens
 
-    # the sequence of C-ABI calls of one step, with pre-marshalled arguments
-    calls = []
-    for B in blks:
-        if has_softmax:
-            calls.append(("softmax_fwd", lib.s2a_softmax_fwd, (B.sx.data_ptr(), B.sy.data_ptr(), B.scodes.data_ptr(), B.smeta.data_ptr(), ns, Ls, dtc, sp)))
-        calls.append(("gelu_fwd", lib.s2a_gelu_fwd, (B.gx.data_ptr(), B.gy.data_ptr(), B.gcodes.data_ptr(), B.gmeta.data_ptr(), ng, Lg, dtc, sp)))
-    for B in reversed(blks):
-        calls.append(("gelu_bwd", lib.s2a_gelu_bwd, (B.gg.data_ptr(), B.gcodes.data_ptr(), B.gmeta.data_ptr(), B.gin.data_ptr(), ng, Lg, dtc, sp)))
-        if has_softmax:
-            calls.append(("softmax_bwd", lib.s2a_softmax_bwd, (B.sg.data_ptr(), B.scodes.data_ptr(), B.smeta.data_ptr(), B.sin.data_ptr(), ns, Ls, dtc, sp)))
+    # the sequence of C-ABI calls of one step on one buffer set, with pre-marshalled arguments
+    def calls_of(set_blks):
+        out = []
+        for B in set_blks:
+            if has_softmax:
+                out.append(("softmax_fwd", lib.s2a_softmax_fwd, (B.sx.data_ptr(), B.sy.data_ptr(), B.scodes.data_ptr(), B.smeta.data_ptr(), ns, Ls, dtc, sp)))
+            out.append(("gelu_fwd", lib.s2a_gelu_fwd, (B.gx.data_ptr(), B.gy.data_ptr(), B.gcodes.data_ptr(), B.gmeta.data_ptr(), ng, Lg, dtc, sp)))
+        for B in reversed(set_blks):
+            out.append(("gelu_bwd", lib.s2a_gelu_bwd, (B.gg.data_ptr(), B.gcodes.data_ptr(), B.gmeta.data_ptr(), B.gin.data_ptr(), ng, Lg, dtc, sp)))
+            if has_softmax:
+                out.append(("softmax_bwd", lib.s2a_softmax_bwd, (B.sg.data_ptr(), B.scodes.data_ptr(), B.smeta.data_ptr(), B.sin.data_ptr(), ns, Ls, dtc, sp)))
+        return out
+
+    set_calls = [calls_of(blks[i * blocks:(i + 1) * blocks]) for i in range(sets)]
+    calls = set_calls[0]
+    step_no = [0]
 
     def step():
-        for _, fn, a in calls:
+        for _, fn, a in set_calls[step_no[0] % sets]:
             rc = fn(*a)
             if rc:
                 raise RuntimeError(binding.status_string(rc))
+        step_no[0] += 1
 
     def barrier():
         if world > 1:
@@ -351,39 +413,56 @@ def run_ours(args, shape, blocks, rank, world):
 
     # ---- timed region: K steps back to back, one event on the stream at each end.  (An
     # event between two launches would defeat programmatic dependent launch, so the
-    # per-kernel figures are taken in separate loops below.)
+    # per-kernel figures are taken in separate loops below.)  The region is repeated R times
+    # (each bracketed by a barrier and a device synchronisation on both sides); the reported
+    # time is the median region, `spread` is (max - min) / median, and the clock sampler runs
+    # across all repeats.
     n_calls = len(calls)
     sampler = ClockSampler(getattr(torch.cuda.get_device_properties(local), "uuid", ""), local)
+
+    def timed_region():
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        ev0.record(stream)
+        for k in range(args.steps):
+            step()
+        ev1.record(stream)
+        barrier()
+        return max_over_ranks(ev0.elapsed_time(ev1), world, dev)
+
+    probe_ms = timed_region()          # decides the number of repeats; not reported
+    repeats = args.repeats if args.repeats > 0 else max(5, min(100, int(1000.0 / max(probe_ms, 1e-3)) + 1))
+    if world > 1:                      # every rank must run the same number of regions
+        t = torch.tensor([repeats], device=dev)
+        dist.broadcast(t, 0)
+        repeats = int(t.item())
     sampler.start()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
     t0 = time.perf_counter()
-    ev0.record(stream)
-    for k in range(args.steps):
-        step()
-    ev1.record(stream)
-    barrier()
+    region_ms = [timed_region() for _ in range(repeats)]
     t1 = time.perf_counter()
     clocks = sampler.finish(t0, t1)
-    total_ms = ev0.elapsed_time(ev1)
+    total_ms = statistics.median(region_ms)
+    spread = (max(region_ms) - min(region_ms)) / total_ms
     if binding.s2a_device_error() != 0:
         raise RuntimeError("a kernel gave up on a bounded wait during the timed region")
 
-    # ---- per kernel: the same launches grouped by kernel, K * blocks back to back
+    # ---- per kernel: the same launches grouped by kernel, K * blocks back to back (rotating
+    # over the buffer sets like the steps do)
     per_kernel_ms = {}
     for name in per_launch:
-        mine = [(fn, a) for n_, fn, a in calls if n_ == name]
-        for fn, a in mine:
-            fn(*a)
+        mine = [[(fn, a) for n_, fn, a in sc if n_ == name] for sc in set_calls]
+        for grp in mine:
+            for fn, a in grp:
+                fn(*a)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier()
         e0.record(stream)
         for k in range(args.steps):
-            for fn, a in mine:
+            for fn, a in mine[k % sets]:
                 fn(*a)
         e1.record(stream)
         barrier()
-        per_kernel_ms[name] = e0.elapsed_time(e1) / (args.steps * len(mine))
+        per_kernel_ms[name] = e0.elapsed_time(e1) / (args.steps * len(mine[0]))
 
     # ---- per kernel with an event before every launch of a step (for comparison: this
     # serialises the launches and adds the event's own cost to each)
@@ -401,8 +480,6 @@ def run_ours(args, shape, blocks, rank, world):
     for ev in events:
         for i, (name, _, _) in enumerate(calls):
             bracketed_ms[name].append(ev[i].elapsed_time(ev[i + 1]))
-
-    total_ms = max_over_ranks(total_ms, world, dev)
 
     # ---- end to end: pinned host inputs in, results out, every step
     e2e = None
@@ -432,12 +509,12 @@ def run_ours(args, shape, blocks, rank, world):
 
         def e2e_step():
             s_in.wait_stream(stream)  # last step's kernels have finished with the input buffers
-            for B, (gx, gg, sx, sg) in zip(blks, host):
+            for B, (gx, gg, sx, sg) in zip(blks[:blocks], host[:blocks]):
                 if has_softmax:
                     staged([(B.sx, sx)], lambda: binding.s2a_softmax_fwd(B.sx, B.sy, B.scodes, B.smeta, Ls),
                            [(hy_s, B.sy)])
                 staged([(B.gx, gx)], lambda: binding.s2a_gelu_fwd(B.gx, B.gy, B.gcodes, B.gmeta, Lg), [(hy_g, B.gy)])
-            for B, (gx, gg, sx, sg) in zip(reversed(blks), reversed(host)):
+            for B, (gx, gg, sx, sg) in zip(reversed(blks[:blocks]), reversed(host[:blocks])):
                 staged([(B.gg, gg)], lambda: binding.s2a_gelu_bwd(B.gg, B.gcodes, B.gmeta, B.gin, Lg), [(hy_g, B.gin)])
                 if has_softmax:
                     staged([(B.sg, sg)], lambda: binding.s2a_softmax_bwd(B.sg, B.scodes, B.smeta, B.sin, Ls),
@@ -479,6 +556,7 @@ def run_ours(args, shape, blocks, rank, world):
 
     value = aggregate_throughput(step_bytes, args.steps, total_ms, world)
     cpu_baseline = None
+    parity = None
     if not args.skip_cpu_baseline:
         from oracle import s2a_oracle as o
         threads = o.hardware_threads()
@@ -486,7 +564,29 @@ def run_ours(args, shape, blocks, rank, world):
         for blk in host:
             np_blocks.append(tuple(None if t is None else (t.numpy().view(np.uint16) if t.dtype == torch.int16 else t.numpy())
                                    for t in blk))
-        gbs, gel, dtc_s, sample = oracle_sample_rate(shape, np_blocks, threads)
+        # While the oracle's forward results of a block are at hand, the stash the kernels left
+        # for that block (same inputs) is compared with them: the counts go into the line.
+        parity = {"blocks_checked": 0, "gelu_elements": 0, "gelu_code_mismatches": 0, "gelu_meta_mismatches": 0,
+                  "softmax_elements": 0, "softmax_code_flips": 0, "softmax_flips_not_at_a_bin_edge": 0,
+                  "softmax_meta_mismatches": 0}
+
+        def count_parity(i, arrays, fwd):
+            B = blks[i]
+            gy, gc, gm = fwd["gelu"]
+            parity["blocks_checked"] += 1
+            parity["gelu_elements"] += int(gy.size)
+            parity["gelu_code_mismatches"] += int(np.count_nonzero(_unpack4(B.gcodes.cpu().numpy(), gy.size) != _unpack4(gc, gy.size)))
+            parity["gelu_meta_mismatches"] += int(np.count_nonzero(B.gmeta.cpu().numpy().view(np.uint32) != gm.view(np.uint32)))
+            if "softmax" in fwd:
+                sy, sc, sm = fwd["softmax"]
+                flips, outside = softmax_code_flips(B.scodes.cpu().numpy(), sy, sc, arrays[2], shape.tokens, shape.dtype)
+                parity["softmax_elements"] += int(sy.size)
+                parity["softmax_code_flips"] += flips
+                parity["softmax_flips_not_at_a_bin_edge"] += outside
+                parity["softmax_meta_mismatches"] += int(np.count_nonzero(
+                    (B.smeta.cpu().numpy().view(np.uint32) != sm.view(np.uint32)).reshape(-1, 2).any(axis=1)))
+
+        gbs, gel, dtc_s, sample = oracle_sample_rate(shape, np_blocks, threads, on_block=count_parity)
         cpu_baseline = {"value": gbs, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": sample,
                         "gelem_per_s": gel, "seconds": dtc_s}
 
@@ -494,18 +594,21 @@ def run_ours(args, shape, blocks, rank, world):
     line = {
         "metric": "s2a_fwd_bwd_algorithmic_bandwidth", "value": value, "unit": "GB/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
+        "repeats": repeats, "spread": spread, "timing": "median of %d regions of %d steps each" % (repeats, args.steps),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": shape.name, "blocks": blocks, "io_dtype": "bf16" if shape.dtype else "f32",
                    "gelu": [shape.gelu_rows, shape.hidden], "softmax": [shape.softmax_rows, shape.tokens] if has_softmax else None,
-                   "l2": "inputs larger than L2: %.2f GB touched per step, distinct buffers per block" % (step_bytes / 1e9),
+                   "l2": ("inputs larger than L2: %.2f GB touched per step, distinct buffers per block" % (touched / 1e9)) if sets == 1
+                   else ("inputs larger than L2: steps rotate over %d distinct buffer sets, %.2f GB touched between two "
+                         "uses of a buffer" % (sets, sets * touched / 1e9)),
                    "multi_gpu": "independent replicas, no collective"},
         "gelem_per_s": world * step_elems * args.steps / (total_ms * 1e-3) / 1e9,
         "frac_of_8TBps": value / world / NOMINAL_HBM_GBS,
         "frac_of_%s_peak" % peak_kind: value / world / peak,
         "saved_activation_bytes": {"stash": stash, "bf16_stash": bf16_stash, "fp32_stash": 2 * bf16_stash,
                                    "reduction_vs_bf16": bf16_stash / stash},
-        "per_kernel": per_kernel, "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e,
+        "per_kernel": per_kernel, "roofline": roofline, "cpu_baseline": cpu_baseline, "parity": parity, "e2e": e2e,
         "gpu_launches": n_calls * args.steps, "clocks": clocks,
     }
     print(json.dumps(line))
@@ -521,8 +624,16 @@ def main():
         if rank == 0:
             run_reference(args, shape, blocks)
         return
-    if world != args.gpus and world == 1 and args.gpus > 1:
-        sys.exit("--gpus %d needs a torchrun launch with one rank per GPU" % args.gpus)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started as a plain `python bench.py --gpus N`: start again under torch.distributed.run,
+        # one rank per GPU on this node
+        import socket
+        with socket.socket() as sock:
+            sock.bind(("127.0.0.1", 0))
+            port = sock.getsockname()[1]
+        os.execv(sys.executable, [sys.executable, "-m", "torch.distributed.run", "--nnodes=1",
+                                  "--nproc-per-node", str(args.gpus), "--master-addr", "127.0.0.1",
+                                  "--master-port", str(port), os.path.abspath(__file__), *sys.argv[1:]])
     run_ours(args, shape, blocks, rank, world)
 
 

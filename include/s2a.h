@@ -28,11 +28,19 @@
  *   a constant row (d == 0) gets codes 0 and s = 0.  Dequantiser (Eq. 9):
  *   v_hat = code * s + min.
  * - Alignment: x, y, grad_out, grad_in and codes must be 16-byte aligned, meta 8-byte
- *   aligned.  In-place use (y == x, grad_in == grad_out) is allowed; codes and meta
- *   must not overlap any other argument.
- * - Errors: arguments are checked on the host before anything is enqueued; on an
- *   error nothing is launched and nothing is written.  n_elems == 0 returns S2A_OK
- *   without a launch.  Inputs must be finite.
+ *   aligned.  In-place use (y == x, grad_in == grad_out) is allowed; an output that
+ *   overlaps its input without being the same tensor returns S2A_ERR_OVERLAP; codes and
+ *   meta must not overlap any other argument (not checked).
+ * - Errors: arguments are checked on the host before anything is enqueued; an argument
+ *   error (every status but S2A_ERR_CUDA) launches nothing and writes nothing.
+ *   S2A_ERR_CUDA means the runtime refused a launch; a call that needs two launches (full
+ *   tiles, then the rows left over) may by then have enqueued the first.  n_elems == 0
+ *   returns S2A_OK without a launch.  Inputs must be finite.
+ * - State: the library reads no environment variable and keeps no tensor state.  What it
+ *   keeps per GPU is a 4-byte error word (s2a_device_error) and, on the host, the results
+ *   of one-time look-ups per device (kernel attributes, the SM count, device addresses of
+ *   its own symbols).  Any thread may make the first call on a GPU; the look-ups do not
+ *   survive a cudaDeviceReset of that GPU in the same process.
  * - Supported row_len: 1 .. 2^31-1 (row lengths whose rows fit a shared-memory tile
  *   take the pipelined path; others a slower row-at-a-time path).
  */
@@ -56,7 +64,8 @@ typedef enum {
   S2A_ERR_DTYPE = 4,  /* dt is neither S2A_F32 nor S2A_BF16                      */
   S2A_ERR_CUDA = 5,   /* the CUDA runtime refused the launch                     */
   S2A_ERR_DEVICE = 6, /* a kernel gave up on a bounded wait (see s2a_device_error) */
-  S2A_ERR_TOO_LARGE = 7 /* beyond the built-in scratch of s2a_gelu_fwd_tensor_range_static */
+  S2A_ERR_TOO_LARGE = 7, /* beyond the built-in scratch of s2a_gelu_fwd_tensor_range_static */
+  S2A_ERR_OVERLAP = 8 /* the output overlaps the input without being the same tensor   */
 } s2a_status;
 
 /* Bytes of packed codes for n_elems elements: (n_elems + 1) / 2. */
@@ -103,10 +112,9 @@ int s2a_softmax_fwd(const void* x, void* y, uint8_t* codes, float* meta, size_t 
 int s2a_softmax_bwd(const void* grad_out, const uint8_t* codes, const float* meta, void* grad_in,
                     size_t n_elems, size_t row_len, int dt, void* cuda_stream);
 
-/* SiLU / Swish forward and backward with the same 4-bit input stash.  The paper names
- * these functions (Section 3.2, end of "GeLU layer": the design "is also effective for
- * similar non-parametric functions, such as SiLU and Swish") without giving constants, so
- * the reading is this library's: y = x * sigmoid(x); the input is clipped into [-C, C] with
+/* SiLU / Swish forward and backward with the same 4-bit input stash.  Section 3.2 (end of
+ * the "GeLU layer" paragraph) says the design carries over to SiLU and Swish but prints no
+ * constants for them, so the reading is this library's: y = x * sigmoid(x); the input is clipped into [-C, C] with
  * C = 2 * 1.702 = 3.404 (binary32), which spans the same range of the sigmoid's argument as
  * GELU's [-2, 2]; Eq. 8 / Eq. 9 per row as for GELU; the backward pass multiplies grad_out by
  * the EXACT derivative sigmoid(x_hat) * (1 + x_hat * (1 - sigmoid(x_hat))), evaluated in
@@ -123,17 +131,20 @@ int s2a_silu_bwd(const void* grad_out, const uint8_t* codes, const float* meta, 
 size_t s2a_tensor_range_scratch_bytes(size_t n_elems);
 
 /* GELU forward whose stash uses ONE quantiser range for the whole tensor -- the other
- * reading of Section 3.2, "GeLU layer" ("quantized between the maximal and minimal value"):
- * Eq. 8's min and max are taken over the whole clipped tensor.  y is as for s2a_gelu_fwd;
+ * reading of Section 3.2, "GeLU layer", which says that the clipped input is quantised over
+ * its min-to-max range without saying over which elements: here Eq. 8's min and max are
+ * taken over the whole clipped tensor.  y is as for s2a_gelu_fwd;
  * every row's metadata carries the same (min, s), so s2a_gelu_bwd consumes the stash
  * unchanged.  The range must be known before the first code, so x is read twice
  * (6.5 bytes per bfloat16 element instead of 4.5).  Three kernels are enqueued.
- *   x, y, codes, meta  as for s2a_gelu_fwd, except that y must NOT alias x
+ *   x, y, codes, meta  as for s2a_gelu_fwd (y may be x itself: the range pass has finished
+ *                      with x before the pass that writes y starts, and that pass reads
+ *                      each element before it writes it)
  *   scratch            device memory, s2a_tensor_range_scratch_bytes(n_elems) bytes, 8-byte
  *                      aligned, owned by the caller; contents on entry are ignored, and it
  *                      must not be used by other work on the GPU until the call's kernels
  *                      have finished
- * Errors as for s2a_gelu_fwd; x == y returns S2A_ERR_ALIGN.
+ * Errors as for s2a_gelu_fwd.
  */
 int s2a_gelu_fwd_tensor_range(const void* x, void* y, uint8_t* codes, float* meta, void* scratch,
                               size_t n_elems, size_t row_len, int dt, void* cuda_stream);
@@ -165,8 +176,8 @@ size_t s2a_tensor_range_static_max_elems(void);
  *   on one stream or order them yourself.
  * - The first call on each GPU looks up the array's device address (with that GPU current);
  *   make that first call outside any stream capture.
- * Arguments, aliasing rule (y must not alias x) and the other errors are those of
- * s2a_gelu_fwd_tensor_range without `scratch`.
+ * - The look-up is safe from any thread; it does not survive a cudaDeviceReset of the GPU.
+ * Arguments and the other errors are those of s2a_gelu_fwd_tensor_range without `scratch`.
  */
 int s2a_gelu_fwd_tensor_range_static(const void* x, void* y, uint8_t* codes, float* meta, size_t n_elems,
                                      size_t row_len, int dt, void* cuda_stream);

@@ -345,9 +345,9 @@ int s2a_oracle_silu_bwd(const void* g, const uint8_t* codes, const float* meta, 
   return 0;
 }
 
-// ---- GELU forward, per-TENSOR range: the other reading of "quantized between the maximal
-// and minimal value" (Section 3.2, "GeLU layer"): Eq. 8's min and max are taken over the
-// whole clipped tensor instead of over each row.  Every row's metadata carries the same
+// ---- GELU forward, per-TENSOR range: the other reading of Section 3.2, "GeLU layer", which
+// quantises the clipped input over its min-to-max range without saying over which elements:
+// here Eq. 8's min and max are taken over the whole clipped tensor instead of over each row.  Every row's metadata carries the same
 // (min, s), so the backward pass is unchanged.
 int s2a_oracle_gelu_fwd_tensor_range(const void* x, void* y, uint8_t* codes, float* meta, size_t n,
                                      size_t L, int dt) {

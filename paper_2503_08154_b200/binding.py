@@ -36,6 +36,15 @@ class S2AError(RuntimeError):
     pass
 
 
+def use_library(path: str) -> None:
+    """Loads another build of the library (e.g. libs2a_tuning.so) instead of libs2a.so.
+    Must be called before the first call into the library."""
+    global LIB_PATH
+    if _lib is not None:
+        raise S2AError("the library is already loaded")
+    LIB_PATH = os.path.abspath(path)
+
+
 def lib() -> ctypes.CDLL:
     """Loads libs2a.so (built in-tree by ``build.py``); raises if it is absent."""
     global _lib

@@ -1,4 +1,11 @@
-"""Builds libs2a.so in-tree with nvcc for sm_100a (no GPU needed to compile)."""
+"""Builds libs2a.so in-tree with nvcc for sm_100a (no GPU needed to compile).
+
+    python -m paper_2503_08154_b200.build [--force] [-v] [--tuning]
+
+--tuning builds a SECOND library, libs2a_tuning.so, with -DS2A_TUNING: the only build in
+which the launch-shape planner honours its S2A_* environment overrides (for sweeps; load
+it with binding.use_library).  libs2a.so itself reads no environment variable.
+"""
 from __future__ import annotations
 
 import os
@@ -25,16 +32,19 @@ def _newer(deps, target) -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, tuning: bool = False) -> str:
     nvcc = os.environ.get("NVCC", "nvcc")
     hdrs = [os.path.join(CSRC, h) for h in HEADERS] + [os.path.abspath(__file__)]
-    os.makedirs(OBJ, exist_ok=True)
+    obj_dir = OBJ + "_tuning" if tuning else OBJ
+    out = os.path.join(HERE, "libs2a_tuning.so") if tuning else OUT
+    os.makedirs(obj_dir, exist_ok=True)
     jobs = []
     for src in SOURCES:
         path = os.path.join(CSRC, src)
-        obj = os.path.join(OBJ, src[:-3] + ".o")
+        obj = os.path.join(obj_dir, src[:-3] + ".o")
         if force or _newer([path, *hdrs], obj):
-            jobs.append([nvcc, *NVCC_FLAGS, *(["-Xptxas", "-v"] if verbose else []), "-c", path, "-o", obj])
+            jobs.append([nvcc, *NVCC_FLAGS, *(["-DS2A_TUNING"] if tuning else []),
+                         *(["-Xptxas", "-v"] if verbose else []), "-c", path, "-o", obj])
 
     def run(cmd):
         r = subprocess.run(cmd, capture_output=True, text=True)
@@ -47,12 +57,12 @@ def build(force: bool = False, verbose: bool = False) -> str:
                     sys.stderr.write(r.stdout + r.stderr)
                 if r.returncode != 0:
                     raise RuntimeError("nvcc failed: " + " ".join(cmd))
-    objs = [os.path.join(OBJ, s[:-3] + ".o") for s in SOURCES]
-    if jobs or _newer(objs, OUT):
-        subprocess.run([nvcc, *ARCH, "-shared", *objs, "-o", OUT + ".tmp"], check=True)
-        os.replace(OUT + ".tmp", OUT)
-    return OUT
+    objs = [os.path.join(obj_dir, s[:-3] + ".o") for s in SOURCES]
+    if jobs or _newer(objs, out):
+        subprocess.run([nvcc, *ARCH, "-shared", *objs, "-o", out + ".tmp"], check=True)
+        os.replace(out + ".tmp", out)
+    return out
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, tuning="--tuning" in sys.argv))

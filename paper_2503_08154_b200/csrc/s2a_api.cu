@@ -20,6 +20,13 @@ int check_args(const void* a, const void* b, const void* codes, const void* meta
   if (!a || !b || !codes || !meta) return S2A_ERR_NULL;
   if (misaligned(a, 16) || misaligned(b, 16) || misaligned(codes, 16) || misaligned(meta, 8))
     return S2A_ERR_ALIGN;
+  // in-place (a == b) is fine: every element, and every row, is read before it is written;
+  // an output that merely overlaps its input would be overwritten while still unread
+  if (a != b) {
+    const uintptr_t bytes = (uintptr_t)n * (dt == S2A_F32 ? 4u : 2u);
+    const uintptr_t pa = (uintptr_t)a, pb = (uintptr_t)b;
+    if (pa < pb + bytes && pb < pa + bytes) return S2A_ERR_OVERLAP;
+  }
   return S2A_OK;
 }
 
@@ -67,6 +74,7 @@ const char* s2a_status_string(int status) {
     case S2A_ERR_TOO_LARGE:
       return "S2A_ERR_TOO_LARGE: n_elems exceeds the built-in scratch of the allocation-free entry point "
              "(536,870,912 elements); use s2a_gelu_fwd_tensor_range with your own scratch";
+    case S2A_ERR_OVERLAP: return "S2A_ERR_OVERLAP: the output overlaps the input without being the same tensor";
     default: return "unknown s2a status";
   }
 }
@@ -144,8 +152,6 @@ int s2a_gelu_fwd_tensor_range(const void* x, void* y, uint8_t* codes, float* met
   if (rc != S2A_OK || n_elems == 0) return rc;
   if (!scratch) return S2A_ERR_NULL;
   if (misaligned(scratch, 8)) return S2A_ERR_ALIGN;
-  // x is read again after y has been written: the two may not alias in this variant
-  if (x == (const void*)y) return S2A_ERR_ALIGN;
   return launch_gelu_fwd_tensor_range(dt, x, y, codes, meta, (float*)scratch, n_elems, n_elems / row_len,
                                       (cudaStream_t)cuda_stream) == cudaSuccess ? S2A_OK : S2A_ERR_CUDA;
 }
@@ -157,7 +163,6 @@ int s2a_gelu_fwd_tensor_range_static(const void* x, void* y, uint8_t* codes, flo
   int rc = check_args(x, y, codes, meta, n_elems, row_len, dt);
   if (rc != S2A_OK || n_elems == 0) return rc;
   if (n_elems > tensor_range_static_max_elems()) return S2A_ERR_TOO_LARGE;
-  if (x == (const void*)y) return S2A_ERR_ALIGN;
   return launch_gelu_fwd_tensor_range_static(dt, x, y, codes, meta, n_elems, n_elems / row_len,
                                              (cudaStream_t)cuda_stream) == cudaSuccess ? S2A_OK : S2A_ERR_CUDA;
 }
@@ -247,10 +252,10 @@ int s2a_describe_plan(int kernel, size_t n_elems, size_t row_len, int dt, char* 
   } else {
     snprintf(out, cap,
              "tile variant=%s rows/tile=%u unit=%u vec=%u iters=%u warps=%u stages=%u smem=%u grid=%u "
-             "tiles=%llu tail_rows=%llu",
+             "group=%u spread=%u tiles=%llu tail_rows=%llu",
              p.variant == kVariantStream ? "stream" : (p.variant == kVariantPairFixed ? "pair-fixed" : (p.variant == kVariantAny ? "any-length" : "generic")),
              p.tile_rows, p.unit_lanes, p.vec_elems, p.iters, p.warps, p.stages, p.smem_bytes,
-             p.grid, (unsigned long long)p.n_tiles,
+             p.grid, p.rows_per_group, p.spread_units, (unsigned long long)p.n_tiles,
              (unsigned long long)(n_rows - p.n_tiles * p.tile_rows));
   }
   return S2A_OK;

@@ -6,6 +6,10 @@
 
 namespace s2a {
 
+// Per-device host-side caches (attribute set-up, symbol addresses, SM counts) are tables of
+// this many entries indexed by the CUDA device ordinal.
+constexpr int kMaxDevices = 64;
+
 enum { kGeluFwd = 0, kGeluBwd = 1, kSoftmaxFwd = 2, kSoftmaxBwd = 3, kSiluFwd = 4, kSiluBwd = 5 };
 
 // Kernel-id predicates (GELU and SiLU share their code: "act" kernels).
@@ -71,6 +75,8 @@ struct TilePlan {
   uint64_t n_tiles;     // full tiles covered; remaining rows go to the row-at-a-time path
   uint32_t overlap_launch;  // 1: launched with programmatic stream serialization
   uint32_t bits;        // code width of Eq. 8: 4, or 2 / 8 (GELU rows of whole 16-byte vectors)
+  uint32_t rows_per_group;  // rows a unit takes together (the kernel's WORK::rows_per_group); divides tile_rows
+  uint32_t spread_units;    // 1: the sub-warp units of a warp take groups tile_groups / (units per warp) apart
 };
 
 struct TileArgs {

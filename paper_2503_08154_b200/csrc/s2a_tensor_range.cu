@@ -1,5 +1,6 @@
 // GELU forward whose 4-bit stash uses ONE quantiser range for the whole tensor (the other
-// reading of Section 3.2, "GeLU layer": "quantized between the maximal and minimal value").
+// reading of Section 3.2, "GeLU layer": the paragraph quantises the clipped input over its
+// min-to-max range and leaves open over which elements that range is taken).
 // The range must be known before the first code can be formed, so the tensor is read twice:
 //   1. range_partials: one CTA per chunk of 65,536 elements writes the chunk's (min, max)
 //      of x into scratch memory;
@@ -10,6 +11,8 @@
 // binary32 element) against 4.5 / 8.5 for the per-row stash.
 #include "s2a_common.cuh"
 #include "s2a_launch.h"
+
+#include <atomic>
 
 namespace s2a {
 namespace {
@@ -155,20 +158,24 @@ uint64_t tensor_range_static_max_elems() { return (uint64_t)kStaticChunks * kChu
 // current) and that pointer is what the kernels receive.
 cudaError_t launch_gelu_fwd_tensor_range_static(int dt, const void* x, void* y, uint8_t* codes, float* meta,
                                                 uint64_t n, uint64_t n_rows, cudaStream_t st) {
-  static float* device_address[64] = {};
+  static std::atomic<float*> device_address[kMaxDevices] = {};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
-  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-  if (device_address[dev] == nullptr) {
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  float* scratch = device_address[dev].load(std::memory_order_acquire);
+  if (scratch == nullptr) {
+    // two threads making the first call on a device both look the address up and store the
+    // same value; the address stays valid until the device is reset
     void* p = nullptr;
     e = cudaGetSymbolAddress(&p, g_static_range_scratch);
     if (e != cudaSuccess) return e;
-    device_address[dev] = (float*)p;
+    scratch = (float*)p;
+    device_address[dev].store(scratch, std::memory_order_release);
   }
   // Nothing in the scratch has to start at zero: the first kernel overwrites the partial of
   // every chunk this call uses, the second overwrites the folded range, the third only reads.
-  return launch_gelu_fwd_tensor_range(dt, x, y, codes, meta, device_address[dev], n, n_rows, st);
+  return launch_gelu_fwd_tensor_range(dt, x, y, codes, meta, scratch, n, n_rows, st);
 }
 
 uint64_t tensor_range_scratch_bytes(uint64_t n) {

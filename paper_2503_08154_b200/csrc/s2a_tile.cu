@@ -4,6 +4,8 @@
 
 #include <stdlib.h>
 
+#include <atomic>
+
 namespace s2a {
 
 __device__ unsigned int g_error_word = 0;
@@ -23,10 +25,19 @@ constexpr uint32_t kMaxStageBytes = 56 * 1024;   // tiles are not grown beyond t
 constexpr uint32_t kHardStageBytes = 176 * 1024;  // the smallest legal tile may be this large (one CTA per SM,
                                                   // and a single stage beyond ~96 KB)
 
+// Launch-shape overrides for tuning sweeps exist only in a library built with -DS2A_TUNING
+// (build.py --tuning writes it to a file of its own).  The library proper reads no
+// environment variable: a plan is a pure function of its arguments and the device.
+#ifdef S2A_TUNING
 int env_int(const char* name, int dflt) {
   const char* v = getenv(name);
   return (v && *v) ? atoi(v) : dflt;
 }
+const char* env_str(const char* name) { return getenv(name); }
+#else
+constexpr int env_int(const char*, int dflt) { return dflt; }
+constexpr const char* env_str(const char*) { return nullptr; }
+#endif
 
 uint32_t gcd_u32(uint32_t a, uint32_t b) {
   while (b) { uint32_t t = a % b; a = b; b = t; }
@@ -35,45 +46,50 @@ uint32_t gcd_u32(uint32_t a, uint32_t b) {
 
 uint32_t align_up(uint32_t v, uint32_t a) { return (v + a - 1) / a * a; }
 
+// SMs of the current device, looked up once per device.  Concurrent first calls may both
+// query and store the same value.
 int sm_count() {
-  static int cached = 0;
-  if (cached == 0) {
-    int dev = 0, n = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess &&
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
-      cached = n;
-    else
-      return 148;  // no device visible (planning on a build host): assume a B200
+  static std::atomic<int> cached[kMaxDevices] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices)
+    return 148;  // no device visible (planning on a build host): assume a B200
+  int n = cached[dev].load(std::memory_order_relaxed);
+  if (n == 0) {
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
+    cached[dev].store(n, std::memory_order_relaxed);
   }
-  return cached;
+  return n;
 }
 
-
 unsigned int* error_word_address() {
-  // one address per device; looked up on first use with that device current
-  static unsigned int* addr[64] = {};
+  // one address per device; looked up on first use with that device current (two threads
+  // making the first call both store the same address)
+  static std::atomic<unsigned int*> addr[kMaxDevices] = {};
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-  if (!addr[dev]) {
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  unsigned int* a = addr[dev].load(std::memory_order_acquire);
+  if (!a) {
     void* p = nullptr;
     if (cudaGetSymbolAddress(&p, g_error_word) != cudaSuccess) return nullptr;
-    addr[dev] = (unsigned int*)p;
+    a = (unsigned int*)p;
+    addr[dev].store(a, std::memory_order_release);
   }
-  return addr[dev];
+  return a;
 }
 
 }  // namespace
 
-// Launch-shape policy.  Environment overrides (for tuning sweeps): S2A_PATH=rowwise
-// disables this path; S2A_UNIT, S2A_TILE_ROWS, S2A_WARPS, S2A_STAGES, S2A_CTAS_PER_SM,
-// S2A_VARIANT=generic|any, S2A_FIXED=0, S2A_PDL=0.
+// Launch-shape policy.  In a -DS2A_TUNING build (and only there) the environment overrides
+// it: S2A_PATH=rowwise disables this path; S2A_UNIT, S2A_TILE_ROWS, S2A_WARPS, S2A_STAGES,
+// S2A_CTAS_PER_SM, S2A_VARIANT=generic|any, S2A_FIXED=0, S2A_PDL=0, S2A_SPREAD=0,
+// S2A_SINGLE_STAGE=0.
 TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
   TilePlan p{};
   p.bits = (uint32_t)bits;
   if (bits != 4 && bits != 2 && bits != 8) return p;
-  const char* path = getenv("S2A_PATH");
+  const char* path = env_str("S2A_PATH");
   if (path && path[0] == 'r') return p;
-  const char* var = getenv("S2A_VARIANT");
+  const char* var = env_str("S2A_VARIANT");
   const bool force_generic = var && var[0] == 'g';
   const bool is_gelu = is_act_fwd(kernel) || is_act_bwd(kernel);  // GELU and SiLU share their kernels
   const bool is_silu = act_of(kernel) == 1;
@@ -278,6 +294,15 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
   if (grid > p.n_tiles) grid = p.n_tiles;
   p.grid = (uint32_t)grid;
   p.overlap_launch = env_int("S2A_PDL", 1) != 0 ? 1u : 0u;
+  p.rows_per_group = G;
+  {
+    // The sub-warp units of one warp may take row groups a fixed stride apart (different
+    // shared-memory banks for the odd attention widths); that needs every unit of a warp to
+    // find a group in every round, i.e. the tile's groups to divide evenly among them.
+    const uint32_t upw = unit < 32 ? 32 / unit : 1;
+    const uint32_t n_groups = rows / G;
+    p.spread_units = (upw > 1 && n_groups % upw == 0 && env_int("S2A_SPREAD", 1) != 0) ? 1u : 0u;
+  }
   return p;
 }
 
@@ -300,13 +325,7 @@ cudaError_t launch_tile(int kernel, int dt, const TilePlan& p, const TileArgs& a
   ka.stage_bytes = ka.meta_off + align_up(ka.meta_bytes, 128);
   ka.stages = p.stages;
   ka.tab_off = p.bits == 8 ? kHeaderBytes + p.stages * ka.stage_bytes : 0u;
-  {
-    // spreading needs every warp's units to find a group in every round
-    const uint32_t upw = p.unit_lanes < 32 ? 32 / p.unit_lanes : 1;
-    const uint32_t G = (p.vec_elems == 2 && (a.row_len & 1u)) ? 2u : 1u;
-    const uint32_t n_groups = p.tile_rows / G;
-    ka.spread_units = (upw > 1 && n_groups % upw == 0 && env_int("S2A_SPREAD", 1) != 0) ? 1u : 0u;
-  }
+  ka.spread_units = p.spread_units;
   ka.error_word = error_word_address();
   if (!ka.error_word) return cudaErrorInvalidDevice;
   if (p.bits != 4) return launch_tile_bits(kernel, dt, p, &ka, st);

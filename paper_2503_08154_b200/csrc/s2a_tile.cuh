@@ -23,6 +23,7 @@
 #include "s2a_common.cuh"
 #include "s2a_launch.h"
 
+#include <atomic>
 #include <type_traits>
 
 namespace s2a {
@@ -2093,17 +2094,19 @@ constexpr uint32_t kMaxSmem = 227 * 1024;
 template <class WORK>
 cudaError_t launch_work(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
   auto kfn = tile_kernel<WORK>;
-  static int configured_dev = -1;  // per instantiation; the attribute belongs to a device's context
+  // The attributes belong to a device's context: one bit per device and instantiation.  Two
+  // threads making the first launch on a device may both set them (the same values).
+  static std::atomic<uint64_t> configured{0};
   int dev = 0;
-  cudaGetDevice(&dev);
-  if (configured_dev != dev) {
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  if (!(configured.load(std::memory_order_acquire) >> dev & 1ull)) {
     cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem);
     if (e != cudaSuccess) return e;
     // Always the largest shared-memory carve-out: kernels of different kinds then leave the
     // SMs in the same configuration, and consecutive launches need no reconfiguration.
     e = cudaFuncSetAttribute(kfn, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
     if (e != cudaSuccess) return e;
-    configured_dev = dev;
+    configured.fetch_or(1ull << dev, std::memory_order_release);
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(p.grid);

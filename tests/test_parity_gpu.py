@@ -509,7 +509,7 @@ def test_gelu_tensor_range(rows, L, scale, dt):
     pu.assert_close(pu.widen(gin_g, dt), pu.widen(gin_o, dt), dt, "gelu grad_in (tensor range)")
 
 
-def test_gelu_tensor_range_rejects_aliasing_and_missing_scratch():
+def test_gelu_tensor_range_in_place_and_argument_errors():
     L = binding.lib()
     x = torch.zeros(64, device="cuda")
     y = torch.zeros(64, device="cuda")
@@ -517,10 +517,34 @@ def test_gelu_tensor_range_rejects_aliasing_and_missing_scratch():
     scratch = torch.zeros(64, dtype=torch.uint8, device="cuda")
     s = torch.cuda.current_stream().cuda_stream
     f = L.s2a_gelu_fwd_tensor_range
-    assert f(x.data_ptr(), x.data_ptr(), codes.data_ptr(), meta.data_ptr(), scratch.data_ptr(), 64, 8, 0, s) == 3
+    assert f(x.data_ptr(), x.data_ptr() + 64, codes.data_ptr(), meta.data_ptr(), scratch.data_ptr(), 32, 8, 0, s) == 8
     assert f(x.data_ptr(), y.data_ptr(), codes.data_ptr(), meta.data_ptr(), None, 64, 8, 0, s) == 1
     assert f(x.data_ptr(), y.data_ptr(), codes.data_ptr(), meta.data_ptr(), scratch.data_ptr(), 63, 8, 0, s) == 2
     assert binding.tensor_range_scratch_bytes(1) == 16 and binding.tensor_range_scratch_bytes(65537) == 24
+    # in place (y is x itself): the same results as out of place
+    for dt in (F32, BF16):
+        rows, Lr = 300, 3072
+        xh = synth.to_io(synth.gelu_preact(17, ("gtr_inplace", dt), rows * Lr) * np.float32(0.4), dt)
+        y_o, codes_o, meta_o = o.gelu_fwd_tensor_range(xh, Lr, dt)
+        xd = pu.to_device(xh, dt)
+        cg, mg = binding.alloc_stash(rows * Lr, Lr, "cuda")
+        sc = torch.empty(binding.tensor_range_scratch_bytes(rows * Lr), dtype=torch.uint8, device="cuda")
+        binding.s2a_gelu_fwd_tensor_range(xd, xd, cg, mg, sc, Lr)
+        torch.cuda.synchronize()
+        assert np.array_equal(cg.cpu().numpy(), codes_o) and np.array_equal(mg.cpu().numpy(), meta_o)
+        pu.assert_close(pu.widen(pu.to_host(xd, dt), dt), pu.widen(y_o, dt), dt, "gelu y (tensor range, in place)")
+
+
+def test_device_error_word_reads_zero_and_clears():
+    # no kernel of this suite gives up on a wait: the word stays 0, and reading it with
+    # clear = 1 leaves it 0 (the expiry path itself is not provoked on a shared GPU)
+    lib = binding.lib()
+    import ctypes
+    flags = ctypes.c_uint(0xFFFFFFFF)
+    assert lib.s2a_device_error(ctypes.byref(flags), 1) == 0 and flags.value == 0
+    flags = ctypes.c_uint(0xFFFFFFFF)
+    assert lib.s2a_device_error(ctypes.byref(flags), 0) == 0 and flags.value == 0
+    assert lib.s2a_device_error(None, 0) == 1
 
 
 # ------------------------------------------------------------------ ReLU with a 1-bit stash

@@ -74,5 +74,5 @@ def test_static_scratch_variant_refuses_tensors_beyond_its_array():
     limit = binding.tensor_range_static_max_elems()
     assert limit == 8192 * 65536
     a = 0x10000                               # never dereferenced: the size check comes first
-    rc = lib.s2a_gelu_fwd_tensor_range_static(a, a + 0x100, a, a, limit + 4096, 4096, binding.BF16, None)
+    rc = lib.s2a_gelu_fwd_tensor_range_static(a, a + (1 << 40), a, a, limit + 4096, 4096, binding.BF16, None)
     assert rc == 7 and "TOO_LARGE" in binding.status_string(rc)
