@@ -160,6 +160,75 @@ __device__ __forceinline__ double gelu_sine_derivative(uint32_t code, float mn, 
   return act_derivative<kActGelu>(code, mn, s);
 }
 
+// ---------------------------------------------------------------- packed binary32 pairs
+// sm_100 executes add / sub / mul / fma on TWO binary32 values held in a 64-bit register
+// pair with one instruction, each half correctly rounded exactly like the scalar operation
+// (so the pinned operation sequence of Eq. 8 keeps its results bit for bit).  The kernels
+// are bound by instruction issue as much as by memory, and this halves the issue slots of
+// their floating-point arithmetic.
+struct F2 {
+  uint64_t v;
+};
+__device__ __forceinline__ F2 f2_pack(float lo, float hi) {
+  F2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r.v) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ F2 f2_both(float x) { return f2_pack(x, x); }
+__device__ __forceinline__ void f2_unpack(F2 a, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(a.v));
+}
+__device__ __forceinline__ F2 f2_fma(F2 a, F2 b, F2 c) {
+  F2 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d.v) : "l"(a.v), "l"(b.v), "l"(c.v));
+  return d;
+}
+__device__ __forceinline__ F2 f2_add(F2 a, F2 b) {
+  F2 d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d.v) : "l"(a.v), "l"(b.v));
+  return d;
+}
+__device__ __forceinline__ F2 f2_sub(F2 a, F2 b) {
+  F2 d;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d.v) : "l"(a.v), "l"(b.v));
+  return d;
+}
+__device__ __forceinline__ F2 f2_mul(F2 a, F2 b) {
+  F2 d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d.v) : "l"(a.v), "l"(b.v));
+  return d;
+}
+// The two halves of a packed bfloat16 pair, widened (exact).
+__device__ __forceinline__ F2 f2_from_bf16x2(uint32_t w) {
+  return f2_pack(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+}
+// Rounds both halves to bfloat16 (nearest even): low half in the low 16 bits.
+__device__ __forceinline__ uint32_t f2_to_bf16x2(F2 a) {
+  float lo, hi;
+  f2_unpack(a, lo, hi);
+  __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);
+  return *(uint32_t*)&b;
+}
+// Eq. 8 on a pair: (code of lo) + 16 * (code of hi) + a constant the caller removes or
+// ignores above bit 7 -- the rounded scaled values sit in the low mantissa bits of
+// t + 1.5 * 2^23 (see quant_code).  min2 / inv2 hold the row's min and 15 / (max - min) twice.
+//
+// The product is formed by an fma with +0 (the same value as the multiply: the scaled values
+// are never -0).  A packed multiply followed directly by a packed add is contracted by the
+// assembler into ONE fused operation, explicit rounding modifiers notwithstanding (measured:
+// 7e-4 of random pairs then differ), and a single rounding breaks the ties that Eq. 8's
+// pinned sequence resolves with two: a product that rounds to exactly k + 1/2 must go to the
+// even code.  An fma result is not contracted further.
+__device__ __forceinline__ F2 f2_scaled(F2 v, F2 min2, F2 inv2) {
+  return f2_fma(f2_sub(v, min2), inv2, f2_both(0.0f));
+}
+__device__ __forceinline__ uint32_t f2_code_byte(F2 v, F2 min2, F2 inv2) {
+  const F2 t = f2_add(f2_scaled(v, min2, inv2), f2_both(12582912.0f));
+  float lo, hi;
+  f2_unpack(t, lo, hi);
+  return __float_as_uint(lo) + (__float_as_uint(hi) << 4);  // bits 0..7: the two codes (0x4B400000 has none there)
+}
+
 // ---------------------------------------------------------------- warp reductions
 __device__ __forceinline__ float warp_max(float v) {
 #pragma unroll

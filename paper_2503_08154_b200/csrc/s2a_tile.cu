@@ -326,6 +326,11 @@ cudaError_t launch_tile(int kernel, int dt, const TilePlan& p, const TileArgs& a
   ka.stages = p.stages;
   ka.tab_off = p.bits == 8 ? kHeaderBytes + p.stages * ka.stage_bytes : 0u;
   ka.spread_units = p.spread_units;
+  // two tiles per CTA ahead of the dependency wait (measured on the ViT-B/16 step: 0 tiles
+  // 5286 GB/s, 1: 5640, 2: 5810, 3: 5700, 4: 5666, 6: 5407 -- more than the first two compete
+  // with the predecessor's last stores)
+  ka.prefetch_tiles = p.overlap_launch ? (uint32_t)env_int("S2A_PREFETCH", p.stages < 2 ? (int)p.stages : 2) : 0u;
+  ka.prefetch_ahead = (uint32_t)env_int("S2A_X1", 0);
   ka.error_word = error_word_address();
   if (!ka.error_word) return cudaErrorInvalidDevice;
   if (p.bits != 4) return launch_tile_bits(kernel, dt, p, &ka, st);

@@ -58,6 +58,8 @@ struct TileKernelArgs {
   uint32_t stages;
   uint32_t spread_units;     // 1: sub-warp units of a warp take groups a fixed stride apart
   uint32_t tab_off;          // byte offset of the wide derivative tables (8-bit codes), else 0
+  uint32_t prefetch_tiles;   // tiles whose inputs the copy lane asks into the L2 before the dependency wait
+  uint32_t prefetch_ahead;   // steady state: with the load of tile i, tile i + this many is asked into the L2 (0: off)
   unsigned int* error_word;  // device address of the per-device error word
 };
 
@@ -133,6 +135,12 @@ __device__ __forceinline__ void bulk_load(void* dst_smem, const void* src, uint3
           "r"(smem_u32(dst_smem)),
       "l"(src), "r"(bytes), "r"(smem_u32(bar))
       : "memory");
+}
+// Asks for a span of this GPU's global memory to be brought into the L2.  A prefetch changes
+// no architectural state (the L2 is the point of coherence: a line written later by an
+// earlier kernel is simply updated there), so it may run ahead of the dependency wait.
+__device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
 }
 // shared -> global bulk copy, tracked by the thread's bulk-group.
 __device__ __forceinline__ void bulk_store(void* dst, const void* src_smem, uint32_t bytes) {
@@ -1766,7 +1774,7 @@ struct PairSoftmaxFwd<kBF16, UNIT_, LCT> {
   // and stores nothing, so that every lane takes part in the shuffles.
   struct Regs {
     uint32_t w[G::ITERS];      // input words, later y as written
-    float e[G::ITERS][2];
+    F2 e[G::ITERS];            // the two exponentials of each word, as a packed binary32 pair
   };
   template <int HP>
   static __device__ __forceinline__ bool drop_lo(int i, int ul) { return HP == 1 && i == 0 && ul == 0; }
@@ -1789,28 +1797,31 @@ struct PairSoftmaxFwd<kBF16, UNIT_, LCT> {
     return fmaxf(lo(mx2), hi(mx2));
   }
 
+  // All binary32 arithmetic below runs on packed pairs (one instruction per word).
   static __device__ __forceinline__ float exp_sum(Regs& R, float m) {
     constexpr float kLog2e = 1.4426950408889634f;
-    const float nm = -m * kLog2e;
-    float z = 0.0f;
+    const F2 k2 = f2_both(kLog2e), nm2 = f2_both(-m * kLog2e);
+    F2 z2 = f2_both(0.0f);
 #pragma unroll
     for (int i = 0; i < G::ITERS; ++i) {
-      R.e[i][0] = ex2_approx(fmaf(lo(R.w[i]), kLog2e, nm));  // foreign / absent: 2^-inf = 0
-      R.e[i][1] = ex2_approx(fmaf(hi(R.w[i]), kLog2e, nm));
-      z += R.e[i][0];
-      z += R.e[i][1];
+      float a0, a1;
+      f2_unpack(f2_fma(f2_from_bf16x2(R.w[i]), k2, nm2), a0, a1);
+      R.e[i] = f2_pack(ex2_approx(a0), ex2_approx(a1));  // foreign / absent: 2^-inf = 0
+      z2 = f2_add(z2, R.e[i]);
     }
-    return z;
+    float z0, z1;
+    f2_unpack(z2, z0, z1);
+    return z0 + z1;
   }
 
   template <int HP>
   static __device__ __forceinline__ void scale_store(Regs& R, float rz, uint32_t* out, int ul, bool active,
                                                      float& mn, float& mx) {
     uint32_t mn2 = 0x7F807F80u, mx2 = 0xFF80FF80u;
+    const F2 rz2 = f2_both(rz);
 #pragma unroll
     for (int i = 0; i < G::ITERS; ++i) {
-      __nv_bfloat162 b = __floats2bfloat162_rn(R.e[i][0] * rz, R.e[i][1] * rz);
-      const uint32_t w = *(uint32_t*)&b;  // y as written
+      const uint32_t w = f2_to_bf16x2(f2_mul(R.e[i], rz2));  // y as written
       R.w[i] = w;
       if (G::has(i, ul)) {
         uint32_t wm = w;  // for min/max a foreign half is replaced by its neighbour
@@ -1829,14 +1840,13 @@ struct PairSoftmaxFwd<kBF16, UNIT_, LCT> {
     mx = fmaxf(lo(mx2), hi(mx2));
   }
 
-  // Code byte of word i of a row (a foreign half codes as 0).
+  // Code byte of word i of a row (a foreign half codes as 0: it is replaced by the minimum).
   template <int HP>
-  static __device__ __forceinline__ uint32_t code_byte(const Regs& R, int i, int ul, const QRange& q) {
-    CodePacker<2> pk;
-    pk.init();
-    pk.add(0, drop_lo<HP>(i, ul) ? q.mn : lo(R.w[i]), q);
-    pk.add(1, drop_hi<HP>(i, ul) ? q.mn : hi(R.w[i]), q);
-    return pk.acc & 0xFFu;
+  static __device__ __forceinline__ uint32_t code_byte(const Regs& R, int i, int ul, const QRange& q, F2 min2, F2 inv2) {
+    float v0 = lo(R.w[i]), v1 = hi(R.w[i]);
+    if (drop_lo<HP>(i, ul)) v0 = q.mn;
+    if (drop_hi<HP>(i, ul)) v1 = q.mn;
+    return f2_code_byte(f2_pack(v0, v1), min2, inv2) & 0xFFu;
   }
 
   static __device__ __forceinline__ void group(Unit<UNIT_>& u, State&, const StagePtrs& p, float*, uint32_t grp,
@@ -1866,15 +1876,17 @@ struct PairSoftmaxFwd<kBF16, UNIT_, LCT> {
     }
     // The byte the two rows share: row A's last element is its low nibble, row B's first
     // its high nibble.  A's nibble travels by shuffle to the lane that owns B's first word.
-    const uint32_t a_last = code_byte<HA>(A, G::LAST_I, ul, qA);
+    const F2 minA = f2_both(qA.mn), invA = f2_both(qA.inv), minB = f2_both(qB.mn), invB = f2_both(qB.inv);
+    const uint32_t a_last = code_byte<HA>(A, G::LAST_I, ul, qA, minA, invA);
     const uint32_t shared_lo = __shfl_sync(0xffffffffu, a_last, (threadIdx.x & 31 & ~(UNIT_ - 1)) | G::LAST_UL);
     unsigned char* cA = p.codes + a0 + ul;
     unsigned char* cB = p.codes + a1 + ul;
 #pragma unroll
     for (int i = 0; i < G::ITERS; ++i) {
       if (active && G::has(i, ul)) {
-        if (!G::kOdd || !(i == G::LAST_I && ul == G::LAST_UL)) cA[UNIT_ * i] = (unsigned char)code_byte<HA>(A, i, ul, qA);
-        uint32_t b = code_byte<HB>(B, i, ul, qB);
+        if (!G::kOdd || !(i == G::LAST_I && ul == G::LAST_UL))
+          cA[UNIT_ * i] = (unsigned char)code_byte<HA>(A, i, ul, qA, minA, invA);
+        uint32_t b = code_byte<HB>(B, i, ul, qB, minB, invB);
         if (G::kOdd && i == 0 && ul == 0) b |= shared_lo & 0x0Fu;
         cB[UNIT_ * i] = (unsigned char)b;
       }
@@ -1978,10 +1990,25 @@ __global__ void __maxnreg__(WORK::kMaxRegs) tile_kernel(TileKernelArgs a) {
     fence_barrier_init();
     grid_launch_dependents();
   }
+  if (threadIdx.x == (uint32_t)n_cwarps * 32u && a.prefetch_tiles != 0) {
+    // A CTA that was scheduled while the previous kernel of the stream is still draining
+    // uses the time: the inputs of its first tiles are on their way into the L2 when the
+    // dependency wait below releases it, which takes the HBM latency out of the pipeline's
+    // fill and keeps the read side of the memory busy during the predecessor's last stores.
+    const uint32_t pf = my_tiles < a.prefetch_tiles ? (uint32_t)my_tiles : a.prefetch_tiles;
+    for (uint32_t i = 0; i < pf; ++i) {
+      const uint64_t t = blockIdx.x + (uint64_t)i * gridDim.x;
+      bulk_prefetch_l2(a.in + t * a.data_bytes, a.data_bytes);
+      if (!kFwd) {
+        bulk_prefetch_l2(a.codes + t * a.code_bytes, a.code_bytes);
+        bulk_prefetch_l2(a.meta + t * a.meta_bytes, a.meta_bytes);
+      }
+    }
+  }
   __syncthreads();
-  // Everything above touched shared memory only.  All threads park here (not only the
-  // copy lane) so that an early-launched CTA does not spin on its barriers, taking issue
-  // slots from the previous kernel's last CTAs.
+  // Everything above touched shared memory only or asked for prefetches.  All threads park
+  // here (not only the copy lane) so that an early-launched CTA does not spin on its
+  // barriers, taking issue slots from the previous kernel's last CTAs.
   grid_dependency_wait();
 
   if (warp == n_cwarps) {
@@ -1997,6 +2024,14 @@ __global__ void __maxnreg__(WORK::kMaxRegs) tile_kernel(TileKernelArgs a) {
       if (!kFwd) {
         bulk_load(st + a.code_off, a.codes + t * a.code_bytes, a.code_bytes, bar);
         bulk_load(st + a.meta_off, a.meta + t * a.meta_bytes, a.meta_bytes, bar);
+      }
+    };
+    auto prefetch_tile = [&](uint64_t it) {
+      const uint64_t t = blockIdx.x + it * gridDim.x;
+      bulk_prefetch_l2(a.in + t * a.data_bytes, a.data_bytes);
+      if (!kFwd) {
+        bulk_prefetch_l2(a.codes + t * a.code_bytes, a.code_bytes);
+        bulk_prefetch_l2(a.meta + t * a.meta_bytes, a.meta_bytes);
       }
     };
     const uint32_t pre = my_tiles < S ? (uint32_t)my_tiles : S;
@@ -2020,6 +2055,7 @@ __global__ void __maxnreg__(WORK::kMaxRegs) tile_kernel(TileKernelArgs a) {
       if (issued < my_tiles) {
         bulk_wait_read<0>();    // the stores of this tile have left shared memory
         issue_load(issued, s);  // tile it + S refills the stage just drained
+        if (a.prefetch_ahead != 0 && issued + a.prefetch_ahead < my_tiles) prefetch_tile(issued + a.prefetch_ahead);
         ++issued;
       }
       if (++s == S) { s = 0; phase ^= 1u; }
