@@ -229,6 +229,27 @@ __device__ __forceinline__ uint32_t f2_code_byte(F2 v, F2 min2, F2 inv2) {
   return __float_as_uint(lo) + (__float_as_uint(hi) << 4);  // bits 0..7: the two codes (0x4B400000 has none there)
 }
 
+// Packed pair forms of the bfloat16 activation (see ActFast / gelu_eval for the two ranges).
+template <int ACT>
+__device__ __forceinline__ F2 f2_act_fast(F2 x) {
+  float k0, k1, d0, d1;
+  f2_unpack(f2_mul(x, f2_both(ActFast<ACT>::kC)), k0, k1);
+  f2_unpack(f2_add(f2_pack(ex2_approx(k0), ex2_approx(k1)), f2_both(1.0f)), d0, d1);
+  return f2_mul(x, f2_pack(rcp_approx(d0), rcp_approx(d1)));
+}
+template <int ACT>
+__device__ __forceinline__ F2 f2_act_general(F2 x) {
+  float k0, k1, d0, d1;
+  f2_unpack(f2_fma(x, f2_both(ActFast<ACT>::kC), f2_both(-8.0f)), k0, k1);
+  f2_unpack(f2_add(f2_pack(ex2_approx(k0), ex2_approx(k1)), f2_both(0.00390625f)), d0, d1);
+  return f2_mul(f2_mul(x, f2_pack(rcp_approx(d0), rcp_approx(d1))), f2_both(0.00390625f));
+}
+__device__ __forceinline__ F2 f2_clip(F2 x, float c) {
+  float a, b;
+  f2_unpack(x, a, b);
+  return f2_pack(fminf(fmaxf(a, -c), c), fminf(fmaxf(b, -c), c));
+}
+
 // ---------------------------------------------------------------- warp reductions
 __device__ __forceinline__ float warp_max(float v) {
 #pragma unroll

@@ -721,17 +721,39 @@ struct StreamActFwd {
   // ActFast::kFastFloor (the caller knows the row minimum before the second pass).
   template <bool FAST>
   static __device__ __forceinline__ void vec(unsigned char* row, unsigned char* crow, uint32_t j, const QRange& q) {
-    float v[V::EPA];
-    V::widen(*(const typename V::Raw*)(row + j * 16u), v);
-    CodePacker<V::EPA> pk;
-    pk.init();
+    // packed binary32 pairs throughout: one instruction per two elements
+    const F2 min2 = f2_both(q.mn), inv2 = f2_both(q.inv), magic2 = f2_both(12582912.0f);
+    uint32_t acc = 0u - kMagicBits * CodePacker<V::EPA>::kOnes;   // see CodePacker
+    if constexpr (DT == kBF16) {
+      const uint4 raw = *(const uint4*)(row + j * 16u);
+      const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+      uint32_t o[4];
 #pragma unroll
-    for (int k = 0; k < V::EPA; ++k) {
-      pk.add(k, fminf(fmaxf(v[k], -kActClip), kActClip), q);
-      v[k] = FAST ? ActFast<ACT>::eval(v[k]) : gelu_eval<DT, ACT>(v[k]);
+      for (int k = 0; k < 4; ++k) {
+        const F2 x = f2_from_bf16x2(w[k]);
+        float t0, t1;
+        f2_unpack(f2_add(f2_scaled(f2_clip(x, kActClip), min2, inv2), magic2), t0, t1);
+        acc += __float_as_uint(t0) << (8 * k);
+        acc += __float_as_uint(t1) << (8 * k + 4);
+        o[k] = f2_to_bf16x2(FAST ? f2_act_fast<ACT>(x) : f2_act_general<ACT>(x));
+      }
+      *(uint4*)(row + j * 16u) = make_uint4(o[0], o[1], o[2], o[3]);
+    } else {
+      const float4 raw = *(const float4*)(row + j * 16u);
+      const float x[4] = {raw.x, raw.y, raw.z, raw.w};
+      float y[4];
+#pragma unroll
+      for (int k = 0; k < 2; ++k) {
+        float t0, t1;
+        f2_unpack(f2_add(f2_scaled(f2_clip(f2_pack(x[2 * k], x[2 * k + 1]), kActClip), min2, inv2), magic2), t0, t1);
+        acc += __float_as_uint(t0) << (8 * k);
+        acc += __float_as_uint(t1) << (8 * k + 4);
+        y[2 * k] = gelu_eval<DT, ACT>(x[2 * k]);
+        y[2 * k + 1] = gelu_eval<DT, ACT>(x[2 * k + 1]);
+      }
+      *(float4*)(row + j * 16u) = make_float4(y[0], y[1], y[2], y[3]);
     }
-    *(typename V::Raw*)(row + j * 16u) = V::narrow(v);
-    V::store_codes(crow, j, pk.acc);
+    V::store_codes(crow, j, acc);
   }
   template <bool FAST>
   static __device__ __forceinline__ void second_pass(unsigned char* row, unsigned char* crow, int ul, uint32_t nv,

@@ -183,6 +183,41 @@ def test_gelu_far_negative_inputs_keep_their_tiny_outputs(rows, L, dt):
     check_gelu(synth.to_io(x.reshape(-1), dt), synth.to_io(g, dt), L, dt)
 
 
+def _double_rounding_tie_rows(L, n_rows, seed):
+    """binary32 rows whose elements sit where Eq. 8's pinned sequence needs BOTH of its roundings:
+    the exact product (x - min) * inv is not a half-integer, but its binary32 rounding is exactly
+    k + 1/2, which the second rounding (to the nearest even code) then resolves.  An evaluation
+    that fuses the multiplication into the rounding step gets the neighbouring code."""
+    rng = np.random.default_rng(seed)
+    rows = []
+    f = np.float32
+    while len(rows) < n_rows:
+        mn, mx = f(-rng.uniform(0.3, 1.9)), f(rng.uniform(0.3, 1.9))
+        inv = f(f(15) / f(mx - mn))
+        found = []
+        for k in range(15):
+            x0 = f(mn + f((k + 0.5) / float(inv)))
+            cand = x0.view(np.uint32).astype(np.int64) + np.arange(-300, 301)
+            x = cand.astype(np.uint32).view(np.float32)
+            t = ((x - mn).astype(np.float32) * inv).astype(np.float32)
+            exact = (x.astype(np.float64) - float(mn))            # exact: few bits, close exponents
+            hit = (t == f(k + 0.5)) & (exact * float(inv) != k + 0.5) & (x > mn) & (x < mx)
+            found.extend(x[hit].tolist())
+        if len(found) < 4:
+            continue
+        row = rng.choice(np.array(found, dtype=np.float32), size=L)
+        row[0], row[1] = mn, mx
+        rows.append(row)
+    return np.stack(rows)
+
+
+@pytest.mark.parametrize("L", [3072, 197, 64])
+def test_gelu_codes_where_the_quantiser_needs_both_of_its_roundings(L):
+    x = _double_rounding_tie_rows(L, 70, seed=L)
+    g = synth.normal(21, ("tie", L), x.size)
+    check_gelu(x.reshape(-1), g, L, F32)
+
+
 def test_gelu_saturated_row_hand_codes():
     # bin edges of a [-2, 2] row; 0 is the exact tie 7.5 and must round to 8
     row = np.array([-3, -2, -1, -0.1333333, 0, 0.1333334, 0.5, 1, 2, 2.5], dtype=np.float32)
