@@ -717,8 +717,9 @@ struct StreamActFwd {
   static __device__ __forceinline__ void init(State&) {}
   static __device__ __forceinline__ uint32_t rows_per_group(uint32_t) { return 1u; }
 
-  // FAST: the short bfloat16 form of the activation, valid on rows with no element below
-  // ActFast::kFastFloor (the caller knows the row minimum before the second pass).
+  // FAST: the short bfloat16 form of the activation (four elements share one reciprocal), valid
+  // on rows with no element below ActQuad::kQuadFloor (the caller knows the row minimum before
+  // the second pass).
   template <bool FAST>
   static __device__ __forceinline__ void vec(unsigned char* row, unsigned char* crow, uint32_t j, const QRange& q) {
     // packed binary32 pairs throughout: one instruction per two elements
@@ -728,14 +729,26 @@ struct StreamActFwd {
       const uint4 raw = *(const uint4*)(row + j * 16u);
       const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
       uint32_t o[4];
+      F2 x[4];
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
-        const F2 x = f2_from_bf16x2(w[k]);
+        x[k] = f2_from_bf16x2(w[k]);
         float t0, t1;
-        f2_unpack(f2_add(f2_scaled(f2_clip(x, kActClip), min2, inv2), magic2), t0, t1);
+        f2_unpack(f2_add(f2_scaled(f2_clip(x[k], kActClip), min2, inv2), magic2), t0, t1);
         acc += __float_as_uint(t0) << (8 * k);
         acc += __float_as_uint(t1) << (8 * k + 4);
-        o[k] = f2_to_bf16x2(FAST ? f2_act_fast<ACT>(x) : f2_act_general<ACT>(x));
+      }
+      if constexpr (FAST) {
+#pragma unroll
+        for (int k = 0; k < 4; k += 2) {
+          F2 ya, yb;
+          ActQuad<ACT>::eval(x[k], x[k + 1], ya, yb);
+          o[k] = f2_to_bf16x2(ya);
+          o[k + 1] = f2_to_bf16x2(yb);
+        }
+      } else {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) o[k] = f2_to_bf16x2(f2_act_general<ACT>(x[k]));
       }
       *(uint4*)(row + j * 16u) = make_uint4(o[0], o[1], o[2], o[3]);
     } else {
@@ -792,7 +805,7 @@ struct StreamActFwd {
     const QRange q = make_qrange(fminf(fmaxf(mn, -kActClip), kActClip), fminf(fmaxf(mx, -kActClip), kActClip));
     if (active && u.ul == 0) { p.meta[2 * r] = q.mn; p.meta[2 * r + 1] = q.s; }
     // mn is the same in every lane of the unit, so the branch does not diverge
-    if (DT == kBF16 && mn >= ActFast<ACT>::kFastFloor) second_pass<true>(row, crow, u.ul, nv, q);
+    if (DT == kBF16 && mn >= ActQuad<ACT>::kQuadFloor) second_pass<true>(row, crow, u.ul, nv, q);
     else second_pass<false>(row, crow, u.ul, nv, q);
   }
 };
@@ -1880,18 +1893,52 @@ struct PairSoftmaxFwd<kBF16, UNIT_, LCT> {
     constexpr int HA = G::kOdd ? 0 : 2, HB = G::kOdd ? 1 : 2;  // the kinds of the pair's two rows
     float mA = load_max<HA>(A, (const uint32_t*)p.data + a0 + ul, ul);
     float mB = load_max<HB>(B, (const uint32_t*)p.data + a1 + ul, ul);
-    mA = u.template reduce<kOpMax>(mA);
-    mB = u.template reduce<kOpMax>(mB);
+    {
+      // both row maxima are bfloat16 values: they travel down ONE shuffle chain as a packed pair
+      __nv_bfloat162 pm = __floats2bfloat162_rn(mA, mB);
+      uint32_t w = *(uint32_t*)&pm;
+#pragma unroll
+      for (int o = UNIT_ / 2; o > 0; o >>= 1) w = max2(w, __shfl_xor_sync(0xffffffffu, w, o));
+      mA = lo(w);
+      mB = hi(w);
+    }
     float zA = exp_sum(A, mA);
     float zB = exp_sum(B, mB);
-    zA = u.template reduce<kOpSum>(zA);
-    zB = u.template reduce<kOpSum>(zB);
+    {
+      F2 z2 = f2_pack(zA, zB);  // the two sums are reduced together, one packed addition per step
+#pragma unroll
+      for (int o = UNIT_ / 2; o > 0; o >>= 1) {
+        float x0, x1;
+        f2_unpack(z2, x0, x1);
+        z2 = f2_add(z2, f2_pack(__shfl_xor_sync(0xffffffffu, x0, o), __shfl_xor_sync(0xffffffffu, x1, o)));
+      }
+      f2_unpack(z2, zA, zB);
+    }
     float mnA, mxA, mnB, mxB;
-    scale_store<HA>(A, __fdiv_rn(1.0f, zA), (uint32_t*)p.data + a0 + ul, ul, active, mnA, mxA);
-    scale_store<HB>(B, __fdiv_rn(1.0f, zB), (uint32_t*)p.data + a1 + ul, ul, active, mnB, mxB);
+    // 1 / z to about an ulp (hardware reciprocal and one correction step): y is rounded to 8 bits
+    const float rA0 = rcp_approx(zA), rB0 = rcp_approx(zB);
+    scale_store<HA>(A, __fmaf_rn(__fmaf_rn(-zA, rA0, 1.0f), rA0, rA0), (uint32_t*)p.data + a0 + ul, ul, active, mnA, mxA);
+    scale_store<HB>(B, __fmaf_rn(__fmaf_rn(-zB, rB0, 1.0f), rB0, rB0), (uint32_t*)p.data + a1 + ul, ul, active, mnB, mxB);
     reduce_minmax_bf16<UNIT_>(mnA, mxA);
     reduce_minmax_bf16<UNIT_>(mnB, mxB);
-    const QRange qA = make_qrange(mnA, mxA), qB = make_qrange(mnB, mxB);
+    // Eq. 8's two correctly rounded quotients per row, 15 / d and d / 15, for both rows with ONE
+    // division: lane 0 of the unit forms 15 / dA, lane 1 dA / 15, lane 2 15 / dB, lane 3 dB / 15
+    // (the other lanes repeat them), and four shuffles hand the results round.
+    QRange qA, qB;
+    {
+      const float dA = __fsub_rn(mxA, mnA), dB = __fsub_rn(mxB, mnB);
+      const float d = (ul & 2) ? dB : dA;
+      const bool odd = (ul & 1) != 0;
+      float quo = __fdiv_rn(odd ? d : kLevels, odd ? kLevels : d);
+      if (d == 0.0f) quo = 0.0f;  // a constant row: inv = s = 0
+      const int base = threadIdx.x & 31 & ~(UNIT_ - 1);
+      qA.mn = mnA;
+      qB.mn = mnB;
+      qA.inv = __shfl_sync(0xffffffffu, quo, base);
+      qA.s = __shfl_sync(0xffffffffu, quo, base + 1);
+      qB.inv = __shfl_sync(0xffffffffu, quo, base + 2);
+      qB.s = __shfl_sync(0xffffffffu, quo, base + 3);
+    }
     if (active && ul == 0) {
       p.meta[2 * r] = qA.mn; p.meta[2 * r + 1] = qA.s;
       p.meta[2 * r + 2] = qB.mn; p.meta[2 * r + 3] = qB.s;
