@@ -160,6 +160,10 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
   } else if (pair_width) {
     variant = kVariantPairFixed;
     unit = L > 257 ? 32u : 8u;
+    // the patch-32 widths: four lanes per row keep seven words each, so that the per-row
+    // reductions and quotients weigh half as much against the per-element work
+    if (L <= 50 && kernel == kSoftmaxFwd) unit = 4;
+    if (env_unit == 4 || env_unit == 8) unit = (uint32_t)env_unit;
     iters = (n_acc + unit - 1) / unit;
   }
   const bool force_any = var && var[0] == 'a';

@@ -1076,69 +1076,157 @@ struct StreamSoftmaxFwd {
   static __device__ __forceinline__ void init(State&) {}
   static __device__ __forceinline__ uint32_t rows_per_group(uint32_t) { return RPU; }
 
+  // All binary32 arithmetic runs on packed pairs (one instruction per two elements).
+  static constexpr int NP = EPA / 2;  // pairs per vector
+  static __device__ __forceinline__ uint32_t hmax2u(uint32_t a, uint32_t b) {
+    __nv_bfloat162 r = __hmax2(*(__nv_bfloat162*)&a, *(__nv_bfloat162*)&b);
+    return *(uint32_t*)&r;
+  }
+  static __device__ __forceinline__ uint32_t hmin2u(uint32_t a, uint32_t b) {
+    __nv_bfloat162 r = __hmin2(*(__nv_bfloat162*)&a, *(__nv_bfloat162*)&b);
+    return *(uint32_t*)&r;
+  }
+
   static __device__ __forceinline__ void group(Unit<UNIT_>& u, State&, const StagePtrs& p, float*, uint32_t grp,
                                                bool active, uint32_t L) {
     const uint32_t nv = active ? L / EPA : 0u;
     const uint32_t r0 = grp * RPU;
-    float e[RPU][NV][EPA];
+    F2 e[RPU][NV][NP];
     float m[RPU], z[RPU], mn[RPU], mx[RPU];
+    const F2 ninf2 = f2_both(-INFINITY);
 #pragma unroll
     for (int rr = 0; rr < RPU; ++rr) {
       const unsigned char* row = p.data + (size_t)(r0 + rr) * L * Io<DT>::kBytes;
       m[rr] = -INFINITY;
+      uint32_t m2 = 0xFF80FF80u;  // bfloat16: packed running maximum
 #pragma unroll
       for (int i = 0; i < NV; ++i) {
         const uint32_t j = u.ul + UNIT_ * i;
         if (j < nv) {
-          V::widen(*(const typename V::Raw*)(row + j * 16u), e[rr][i]);
+          if constexpr (DT == kBF16) {
+            const uint4 raw = *(const uint4*)(row + j * 16u);
+            const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
-          for (int k = 0; k < EPA; ++k) m[rr] = fmaxf(m[rr], e[rr][i][k]);
+            for (int k = 0; k < 4; ++k) {
+              m2 = hmax2u(m2, w[k]);
+              e[rr][i][k] = f2_from_bf16x2(w[k]);
+            }
+          } else {
+            const float4 raw = *(const float4*)(row + j * 16u);
+            m[rr] = fmaxf(fmaxf(m[rr], raw.x), fmaxf(raw.y, fmaxf(raw.z, raw.w)));
+            e[rr][i][0] = f2_pack(raw.x, raw.y);
+            e[rr][i][1] = f2_pack(raw.z, raw.w);
+          }
         } else {
 #pragma unroll
-          for (int k = 0; k < EPA; ++k) e[rr][i][k] = -INFINITY;
+          for (int k = 0; k < NP; ++k) e[rr][i][k] = ninf2;
         }
       }
+      if constexpr (DT == kBF16) m[rr] = fmaxf(__uint_as_float(m2 << 16), __uint_as_float(m2 & 0xffff0000u));
+    }
+    constexpr bool kPackRows = DT == kBF16 && RPU >= 2 && UNIT_ <= 32;  // two rows share a shuffle chain
+    if constexpr (DT == kBF16 && kPackRows) {
+      // the maxima of two rows are bfloat16 values: one shuffle chain for the packed pair
+#pragma unroll
+      for (int rr = 0; rr < RPU; rr += 2) {
+        __nv_bfloat162 pm = __floats2bfloat162_rn(m[rr], m[rr + 1]);
+        uint32_t w = *(uint32_t*)&pm;
+#pragma unroll
+        for (int o = UNIT_ / 2; o > 0; o >>= 1) w = hmax2u(w, __shfl_xor_sync(0xffffffffu, w, o));
+        m[rr] = __uint_as_float(w << 16);
+        m[rr + 1] = __uint_as_float(w & 0xffff0000u);
+      }
+    } else {
+#pragma unroll
+      for (int rr = 0; rr < RPU; ++rr) m[rr] = u.template reduce<kOpMax>(m[rr]);
     }
 #pragma unroll
-    for (int rr = 0; rr < RPU; ++rr) {
-      m[rr] = u.template reduce<kOpMax>(m[rr]);
+    for (int rr = 0; rr < RPU; ++rr)
       if (!active) m[rr] = 0.0f;
-    }
     constexpr float kLog2e = 1.4426950408889634f;
+    const F2 k2 = f2_both(kLog2e);
 #pragma unroll
     for (int rr = 0; rr < RPU; ++rr) {
-      const float nm = -m[rr] * kLog2e;
-      z[rr] = 0.0f;
+      // bfloat16: the exponent's argument is one fused multiply-add (the result is rounded to 8
+      // bits); binary32: the difference, then the product (see exp_eval)
+      const F2 c2 = f2_both(DT == kBF16 ? -m[rr] * kLog2e : m[rr]);
+      F2 z2 = f2_both(0.0f);
 #pragma unroll
       for (int i = 0; i < NV; ++i)
 #pragma unroll
-        for (int k = 0; k < EPA; ++k) {
-          // bfloat16: the exponent's argument is one fused multiply-add (the result is rounded to 8 bits)
-          e[rr][i][k] = DT == kBF16 ? ex2_approx(fmaf(e[rr][i][k], kLog2e, nm)) : exp_eval<DT>(e[rr][i][k] - m[rr]);
-          z[rr] += e[rr][i][k];
+        for (int k = 0; k < NP; ++k) {
+          float a0, a1;
+          f2_unpack(DT == kBF16 ? f2_fma(e[rr][i][k], k2, c2) : f2_mul(k2, f2_sub(e[rr][i][k], c2)), a0, a1);
+          e[rr][i][k] = f2_pack(ex2_approx(a0), ex2_approx(a1));
+          z2 = f2_add(z2, e[rr][i][k]);
         }
+      float z0, z1;
+      f2_unpack(z2, z0, z1);
+      z[rr] = z0 + z1;
     }
+    if constexpr (kPackRows) {
+      // the sums of two rows go down the shuffles together: one packed addition per step
 #pragma unroll
-    for (int rr = 0; rr < RPU; ++rr) z[rr] = u.template reduce<kOpSum>(z[rr]);
+      for (int rr = 0; rr < RPU; rr += 2) {
+        F2 z2 = f2_pack(z[rr], z[rr + 1]);
+#pragma unroll
+        for (int o = UNIT_ / 2; o > 0; o >>= 1) {
+          float x0, x1;
+          f2_unpack(z2, x0, x1);
+          z2 = f2_add(z2, f2_pack(__shfl_xor_sync(0xffffffffu, x0, o), __shfl_xor_sync(0xffffffffu, x1, o)));
+        }
+        f2_unpack(z2, z[rr], z[rr + 1]);
+      }
+    } else {
+#pragma unroll
+      for (int rr = 0; rr < RPU; ++rr) z[rr] = u.template reduce<kOpSum>(z[rr]);
+    }
 #pragma unroll
     for (int rr = 0; rr < RPU; ++rr) {
       unsigned char* row = p.data + (size_t)(r0 + rr) * L * Io<DT>::kBytes;
-      const float rz = __fdiv_rn(1.0f, active ? z[rr] : 1.0f);
-      typename V::MinMax mm;
-      mm.init();
+      const float zz = active ? z[rr] : 1.0f;
+      float rz;
+      if constexpr (DT == kBF16) {
+        const float ra = rcp_approx(zz);  // about an ulp after the correction step; y keeps 8 bits
+        rz = __fmaf_rn(__fmaf_rn(-zz, ra, 1.0f), ra, ra);
+      } else {
+        rz = __fdiv_rn(1.0f, zz);
+      }
+      const F2 rz2 = f2_both(rz);
+      uint32_t mn2 = 0x7F807F80u, mx2 = 0xFF80FF80u;
+      mn[rr] = INFINITY;
+      mx[rr] = -INFINITY;
 #pragma unroll
       for (int i = 0; i < NV; ++i) {
         const uint32_t j = u.ul + UNIT_ * i;
         if (j < nv) {
+          if constexpr (DT == kBF16) {
+            uint32_t w[4];
 #pragma unroll
-          for (int k = 0; k < EPA; ++k) e[rr][i][k] *= rz;
-          const typename V::Raw yw = V::narrow(e[rr][i]);  // e now holds y as written
-          *(typename V::Raw*)(row + j * 16u) = yw;
-          mm.add(yw);
+            for (int k = 0; k < 4; ++k) {
+              w[k] = f2_to_bf16x2(f2_mul(e[rr][i][k], rz2));
+              e[rr][i][k] = f2_from_bf16x2(w[k]);  // y as written
+              mn2 = hmin2u(mn2, w[k]);
+              mx2 = hmax2u(mx2, w[k]);
+            }
+            *(uint4*)(row + j * 16u) = make_uint4(w[0], w[1], w[2], w[3]);
+          } else {
+            float y[4];
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+              e[rr][i][k] = f2_mul(e[rr][i][k], rz2);
+              f2_unpack(e[rr][i][k], y[2 * k], y[2 * k + 1]);
+            }
+            *(float4*)(row + j * 16u) = make_float4(y[0], y[1], y[2], y[3]);
+            mn[rr] = fminf(fminf(mn[rr], y[0]), fminf(y[1], fminf(y[2], y[3])));
+            mx[rr] = fmaxf(fmaxf(mx[rr], y[0]), fmaxf(y[1], fmaxf(y[2], y[3])));
+          }
         }
       }
-      mn[rr] = mm.lo();
-      mx[rr] = mm.hi();
+      if constexpr (DT == kBF16) {
+        mn[rr] = fminf(__uint_as_float(mn2 << 16), __uint_as_float(mn2 & 0xffff0000u));
+        mx[rr] = fmaxf(__uint_as_float(mx2 << 16), __uint_as_float(mx2 & 0xffff0000u));
+      }
     }
 #pragma unroll
     for (int rr = 0; rr < RPU; ++rr) {
@@ -1149,21 +1237,54 @@ struct StreamSoftmaxFwd {
         mx[rr] = u.template reduce<kOpMax>(mx[rr]);
       }
     }
+    const F2 magic2 = f2_both(12582912.0f);
+    // Eq. 8's two correctly rounded quotients per row (15 / d and d / 15).  A unit that walks
+    // several rows forms them for all of its rows together: lane l takes quotient l (row l / 2;
+    // even l: 15 / d, odd l: d / 15), in as many divisions as it takes the unit's lanes to cover
+    // 2 * RPU quotients, and shuffles hand them round.
+    constexpr int NDIV = kPackRows ? (2 * RPU + UNIT_ - 1) / UNIT_ : 1;
+    float quo[NDIV];
+    if constexpr (kPackRows) {
+#pragma unroll
+      for (int dv = 0; dv < NDIV; ++dv) {
+        const int slot = dv * UNIT_ + u.ul;
+        float d = 1.0f;
+#pragma unroll
+        for (int rr = 0; rr < RPU; ++rr)
+          if ((slot >> 1) == rr) d = __fsub_rn(mx[rr], mn[rr]);
+        const bool odd = (slot & 1) != 0;
+        quo[dv] = __fdiv_rn(odd ? d : kLevels, odd ? kLevels : d);
+        if (d == 0.0f) quo[dv] = 0.0f;  // a constant row: inv = s = 0
+      }
+    }
+    const int base = threadIdx.x & 31 & ~((UNIT_ < 32 ? UNIT_ : 32) - 1);
 #pragma unroll
     for (int rr = 0; rr < RPU; ++rr) {
       const uint32_t r = r0 + rr;
       unsigned char* crow = p.codes + (size_t)r * (L / 2);
-      const QRange q = make_qrange(mn[rr], mx[rr]);
+      QRange q;
+      if constexpr (kPackRows) {
+        q.mn = mn[rr];
+        q.inv = __shfl_sync(0xffffffffu, quo[(2 * rr) / UNIT_], base + (2 * rr) % UNIT_);
+        q.s = __shfl_sync(0xffffffffu, quo[(2 * rr + 1) / UNIT_], base + (2 * rr + 1) % UNIT_);
+      } else {
+        q = make_qrange(mn[rr], mx[rr]);
+      }
       if (active && u.ul == 0) { p.meta[2 * r] = q.mn; p.meta[2 * r + 1] = q.s; }
+      const F2 min2 = f2_both(q.mn), inv2 = f2_both(q.inv);
 #pragma unroll
       for (int i = 0; i < NV; ++i) {
         const uint32_t j = u.ul + UNIT_ * i;
         if (j < nv) {
-          CodePacker<EPA> pk;
-          pk.init();
+          uint32_t acc = 0u - kMagicBits * CodePacker<EPA>::kOnes;  // see CodePacker
 #pragma unroll
-          for (int k = 0; k < EPA; ++k) pk.add(k, e[rr][i][k], q);
-          V::store_codes(crow, j, pk.acc);
+          for (int k = 0; k < NP; ++k) {
+            float t0, t1;
+            f2_unpack(f2_add(f2_scaled(e[rr][i][k], min2, inv2), magic2), t0, t1);
+            acc += __float_as_uint(t0) << (8 * k);
+            acc += __float_as_uint(t1) << (8 * k + 4);
+          }
+          V::store_codes(crow, j, acc);
         }
       }
     }
@@ -2348,6 +2469,15 @@ cudaError_t launch_pair_widths(const TilePlan& p, const TileKernelArgs& ka, cuda
     switch (ka.row_len) {
       case 577: return launch_work<WORK<DT, 32, 577>>(p, ka, st);
       case 1025: return launch_work<WORK<DT, 32, 1025>>(p, ka, st);
+    }
+    return cudaErrorInvalidValue;
+  }
+  if (p.unit_lanes == 4) {  // the short widths, forward: four lanes per row
+    if constexpr (WORK<DT, 4, 49>::kKernel == kSoftmaxFwd) {
+      switch (ka.row_len) {
+        case 49: return launch_work<WORK<DT, 4, 49>>(p, ka, st);
+        case 50: return launch_work<WORK<DT, 4, 50>>(p, ka, st);
+      }
     }
     return cudaErrorInvalidValue;
   }
