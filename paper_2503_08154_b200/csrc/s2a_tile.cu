@@ -101,7 +101,7 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
   const bool pair_width = !is_gelu && bits == 4 && !force_generic && !(var && var[0] == 'a') &&
                           (L == 197 || L == 257 || L == 49 || L == 50 || L == 145 || L == 196 || L == 198 || L == 577 ||
                            L == 1025);
-  const bool vec16 = (L % vec) == 0 && !pair_width;
+  const bool vec16 = (L % vec) == 0 && !pair_width && !(bits != 4 && !is_gelu && (L == 197 || L == 257));
   const uint32_t epa = vec16 ? vec : 2u;
   const uint32_t n_acc = vec16 ? L / vec : (L + 1) / 2;  // accesses covering one row
   // rows per tile: the tile's code bytes must be a multiple of 16 (its element count a
@@ -113,7 +113,14 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
 
   uint32_t variant = kVariantGeneric, unit = 0, iters = 0;
   const int env_unit = env_int("S2A_UNIT", 0);
-  if (bits != 4 && (kernel == kSoftmaxFwd || kernel == kSoftmaxBwd)) {
+  const bool pair_bits = bits != 4 && !is_gelu && !force_generic && !(var && var[0] == 'a') && (L == 197 || L == 257);
+  if (pair_bits) {
+    // other code widths at the ViT attention widths: fixed-width kernels of their own (8 bits:
+    // a byte per element, nothing shared; 2 bits: unpacked scratch bytes, packed per tile)
+    variant = kVariantPairFixed;
+    unit = 8;
+    iters = (n_acc + unit - 1) / unit;
+  } else if (bits != 4 && (kernel == kSoftmaxFwd || kernel == kSoftmaxBwd)) {
     // other code widths, softmax: the any-length form (aligned vectors, masked row ends)
     if (L < 16) return p;
     variant = kVariantAny;
@@ -218,6 +225,9 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
   int ctas_per_sm = 2;
   if (variant == kVariantStream && is_gelu) ctas_per_sm = 4;
   if (variant == kVariantPairFixed) ctas_per_sm = 4;
+  // one row at a time per unit; 2 bits: 64-row tiles (whole 16-byte code spans), eight warps, two
+  // CTAs per SM; 8 bits: measured best with the 4-bit kernels' shape (5.2 against 4.9 TB/s)
+  if (pair_bits && bits == 2) { warps = 8; ctas_per_sm = 2; }
   warps = (uint32_t)env_int("S2A_WARPS", (int)warps);
   if (warps < 1 || warps > 16 || (warps * 32) % unit != 0) return p;
   const uint32_t n_units = warps * 32 / unit;
@@ -264,11 +274,15 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
     if (variant == kVariantAny) regs = 80;
     while (ctas_per_sm > 1 && (uint64_t)regs * (warps + 1) * 32 * (uint32_t)ctas_per_sm > 65536) ctas_per_sm /= 2;
   }
+  // beyond the stages: 256-entry derivative tables per unit (8-bit GELU backward), or the CTA's
+  // scratch of one unpacked code byte per element of a tile (2-bit fixed-width softmax forward)
+  const uint32_t extra_bytes = (bits == 8 && is_gelu) ? n_units * 1024u
+                               : ((pair_bits && bits == 2 && kernel == kSoftmaxFwd) ? align_up(rows * L, 128) : 0u);
   const int env_stages = env_int("S2A_STAGES", 0);
   uint32_t stages = 0, smem = 0;
   for (int c = ctas_per_sm; c >= 1 && stages == 0; c /= 2) {
     const uint32_t budget = kMaxSmem / (uint32_t)c - 1024;  // 1 KiB per CTA is the system's
-    const uint32_t fixed = kHeaderBytes + (bits == 8 ? n_units * 1024u : 0u);  // + 256-entry tables
+    const uint32_t fixed = kHeaderBytes + extra_bytes;
     uint32_t fit = budget > fixed ? (budget - fixed) / stage_bytes : 0;
     if (fit > 4) fit = 4;
     if (env_stages > 0 && (uint32_t)env_stages <= fit) fit = (uint32_t)env_stages;
@@ -279,7 +293,7 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
     // and store of a CTA then run one after the other, but the SMs drift out of step and
     // keep the memory system busy between them -- still well ahead of the row-at-a-time path.
     const uint32_t budget = kMaxSmem - 1024;
-    const uint32_t fixed = kHeaderBytes + (bits == 8 ? n_units * 1024u : 0u);
+    const uint32_t fixed = kHeaderBytes + extra_bytes;
     if (budget > fixed && stage_bytes <= budget - fixed) { stages = 1; ctas_per_sm = 1; smem = budget; }
   }
   if (stages == 0) return p;
@@ -306,6 +320,7 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
     const uint32_t upw = unit < 32 ? 32 / unit : 1;
     const uint32_t n_groups = rows / G;
     p.spread_units = (upw > 1 && n_groups % upw == 0 && env_int("S2A_SPREAD", 1) != 0) ? 1u : 0u;
+    if (pair_bits && bits == 2) p.spread_units = 0;  // a warp's units must hold consecutive row pairs
   }
   return p;
 }
@@ -328,7 +343,7 @@ cudaError_t launch_tile(int kernel, int dt, const TilePlan& p, const TileArgs& a
   ka.meta_off = ka.code_off + align_up(ka.code_bytes, 128);
   ka.stage_bytes = ka.meta_off + align_up(ka.meta_bytes, 128);
   ka.stages = p.stages;
-  ka.tab_off = p.bits == 8 ? kHeaderBytes + p.stages * ka.stage_bytes : 0u;
+  ka.tab_off = p.bits != 4 ? kHeaderBytes + p.stages * ka.stage_bytes : 0u;  // the area after the stages
   ka.spread_units = p.spread_units;
   // two tiles per CTA ahead of the dependency wait (measured on the ViT-B/16 step: 0 tiles
   // 5286 GB/s, 1: 5640, 2: 5810, 3: 5700, 4: 5666, 6: 5407 -- more than the first two compete

@@ -2151,6 +2151,227 @@ struct PairSoftmaxBwd {
   }
 };
 
+// ---------------------------------------------------------------- fixed widths at 2 and 8 bits
+// The attention widths 197 and 257 with Eq. 8 at N = 2 or N = 8.  Rows are read as 2-element
+// words like the 4-bit fixed-width kernels, one row at a time per 8-lane unit.  At 8 bits an
+// element owns a whole code byte, so no byte is ever shared.  At 2 bits four elements share a
+// byte and a row of odd length shares bytes with both neighbours -- but EIGHT consecutive rows
+// always own whole bytes (16 L bits).  The four units of a warp take four consecutive row
+// pairs, write one UNPACKED code byte per element into a scratch area of the CTA, and the warp
+// then packs its own eight rows, four scratch bytes to a code byte: nothing is merged
+// atomically and no warp waits for another.
+template <int DT, int UNIT_, int LCT, int NBITS>
+struct PairSoftmaxFwdBits {
+  static_assert(NBITS == 2 || NBITS == 8, "4 bits have kernels of their own");
+  static constexpr int kMaxRegs = 96;
+  static constexpr int kKernel = kSoftmaxFwd;
+  static constexpr int UNIT = UNIT_;
+  static_assert(UNIT_ == 8, "four units per warp: eight consecutive rows per warp and round");
+  static constexpr int kTabFloats = 0;            // `tab` is the CTA's scratch area itself, not a per-unit table
+  using P = P2<DT>;
+  using G = PairGeom<UNIT_, LCT>;
+  struct State {};
+  static __device__ __forceinline__ void init(State&) {}
+  static __device__ __forceinline__ uint32_t rows_per_group(uint32_t) { return 2u; }
+
+  // bytes: where this row's unpacked codes go (element e of the tile at bytes[e]): the code
+  // area itself at 8 bits, the CTA's scratch at 2 bits.
+  template <int HP>
+  static __device__ __forceinline__ void row(Unit<UNIT_>& u, const StagePtrs& p, unsigned char* bytes, uint32_t r,
+                                             bool active) {
+    const uint32_t a0 = (r * (uint32_t)LCT) >> 1;
+    const int ul = u.ul;
+    F2 e[G::ITERS];
+    float m = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < G::ITERS; ++i) {
+      float v0 = -INFINITY, v1 = -INFINITY;
+      if (active && G::has(i, ul)) {
+        const typename P::Raw w = P::load(p.data, a0 + ul + UNIT_ * i);
+        v0 = P::lo(w);
+        v1 = P::hi(w);
+      }
+      if (HP == 1 && i == 0 && ul == 0) v0 = -INFINITY;                        // the previous row's element
+      if (HP == 0 && i == G::LAST_I && ul == G::LAST_UL) v1 = -INFINITY;      // the next row's element
+      e[i] = f2_pack(v0, v1);
+      m = fmaxf(m, fmaxf(v0, v1));
+    }
+    m = u.template reduce<kOpMax>(m);
+    if (!active) m = 0.0f;
+    constexpr float kLog2e = 1.4426950408889634f;
+    const F2 k2 = f2_both(kLog2e), c2 = f2_both(DT == kBF16 ? -m * kLog2e : m);
+    F2 z2 = f2_both(0.0f);
+#pragma unroll
+    for (int i = 0; i < G::ITERS; ++i) {
+      float a, b;
+      f2_unpack(DT == kBF16 ? f2_fma(e[i], k2, c2) : f2_mul(k2, f2_sub(e[i], c2)), a, b);
+      e[i] = f2_pack(ex2_approx(a), ex2_approx(b));  // foreign / absent elements: 2^-inf = 0
+      z2 = f2_add(z2, e[i]);
+    }
+    float z0, z1;
+    f2_unpack(z2, z0, z1);
+    const float z = u.template reduce<kOpSum>(z0 + z1);
+    const float zz = active ? z : 1.0f;
+    float rz;
+    if constexpr (DT == kBF16) {
+      const float ra = rcp_approx(zz);  // about an ulp after the correction step; y keeps 8 bits
+      rz = __fmaf_rn(__fmaf_rn(-zz, ra, 1.0f), ra, ra);
+    } else {
+      rz = __fdiv_rn(1.0f, zz);
+    }
+    const F2 rz2 = f2_both(rz);
+    float mn = INFINITY, mx = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < G::ITERS; ++i) {
+      float y0, y1;
+      f2_unpack(f2_mul(e[i], rz2), y0, y1);
+      const typename P::Raw w = P::pack(y0, y1);
+      y0 = P::lo(w);  // y as written
+      y1 = P::hi(w);
+      e[i] = f2_pack(y0, y1);
+      if (active && G::has(i, ul)) {
+        const bool drop_lo = HP == 1 && i == 0 && ul == 0;
+        const bool drop_hi = HP == 0 && i == G::LAST_I && ul == G::LAST_UL;
+        if (drop_lo) P::store_hi(p.data, a0 + ul + UNIT_ * i, w);
+        else if (drop_hi) P::store_lo(p.data, a0 + ul + UNIT_ * i, w);
+        else P::store(p.data, a0 + ul + UNIT_ * i, w);
+        const float v0 = drop_lo ? y1 : y0, v1 = drop_hi ? y0 : y1;
+        mn = fminf(mn, fminf(v0, v1));
+        mx = fmaxf(mx, fmaxf(v0, v1));
+      }
+    }
+    mn = u.template reduce<kOpMin>(mn);
+    mx = u.template reduce<kOpMax>(mx);
+    const QRange q = make_qrange(mn, mx, (float)((1 << NBITS) - 1));
+    if (active && ul == 0) { p.meta[2 * r] = q.mn; p.meta[2 * r + 1] = q.s; }
+    const F2 min2 = f2_both(q.mn), inv2 = f2_both(q.inv), magic2 = f2_both(12582912.0f);
+    constexpr uint32_t kMask = (1u << NBITS) - 1u;
+#pragma unroll
+    for (int i = 0; i < G::ITERS; ++i) {
+      if (active && G::has(i, ul)) {
+        const bool drop_lo = HP == 1 && i == 0 && ul == 0;
+        const bool drop_hi = HP == 0 && i == G::LAST_I && ul == G::LAST_UL;
+        float t0, t1;
+        f2_unpack(f2_add(f2_scaled(e[i], min2, inv2), magic2), t0, t1);
+        const uint32_t c0 = __float_as_uint(t0) & kMask, c1 = __float_as_uint(t1) & kMask;
+        unsigned char* dst = bytes + 2u * (a0 + ul + UNIT_ * i);
+        if (drop_lo) dst[1] = (unsigned char)c1;
+        else if (drop_hi) dst[0] = (unsigned char)c0;
+        else *(uint16_t*)dst = (uint16_t)(c0 | (c1 << 8));
+      }
+    }
+  }
+
+  static __device__ __forceinline__ void group(Unit<UNIT_>& u, State&, const StagePtrs& p, float* tab, uint32_t grp,
+                                               bool active, uint32_t) {
+    const uint32_t r = active ? 2 * grp : 0;
+    unsigned char* bytes = NBITS == 8 ? p.codes : (unsigned char*)tab;
+    if (G::kOdd) {
+      row<0>(u, p, bytes, r, active);
+      u.sync();  // the odd row reads the word it shares with the even row
+      row<1>(u, p, bytes, r + 1, active);
+    } else {
+      row<2>(u, p, bytes, r, active);
+      row<2>(u, p, bytes, r + 1, active);
+    }
+    u.sync();
+    if (NBITS == 2) {
+      // The warp's four units hold four consecutive pairs (the planner leaves the units unspread
+      // and gives a tile a multiple of four pairs): rows 2 g0 .. 2 g0 + 7, whole code bytes.
+      __syncwarp();
+      const uint32_t e_begin = (grp - (uint32_t)(u.uid & 3)) * 2u * (uint32_t)LCT;
+      if (active) {
+        for (uint32_t b = threadIdx.x & 31u; b < 2u * (uint32_t)LCT; b += 32u) {
+          const uint32_t w = *(const uint32_t*)(bytes + e_begin + 4u * b);
+          p.codes[e_begin / 4u + b] =
+              (unsigned char)((w & 3u) | ((w >> 6) & 0xCu) | ((w >> 12) & 0x30u) | ((w >> 18) & 0xC0u));
+        }
+      }
+      __syncwarp();  // the scratch bytes are free again for the warp's next round
+    }
+  }
+};
+
+template <int DT, int UNIT_, int LCT, int NBITS>
+struct PairSoftmaxBwdBits {
+  static_assert(NBITS == 2 || NBITS == 8, "4 bits have kernels of their own");
+  static constexpr int kMaxRegs = 96;
+  static constexpr int kKernel = kSoftmaxBwd;
+  static constexpr int UNIT = UNIT_;
+  using P = P2<DT>;
+  using G = PairGeom<UNIT_, LCT>;
+  struct State {};
+  static __device__ __forceinline__ void init(State&) {}
+  static __device__ __forceinline__ uint32_t rows_per_group(uint32_t) { return 2u; }
+
+  template <int HP>
+  static __device__ __forceinline__ void row(Unit<UNIT_>& u, const StagePtrs& p, uint32_t r, bool active) {
+    const uint32_t a0 = (r * (uint32_t)LCT) >> 1;
+    const int ul = u.ul;
+    const float mn = p.meta[2 * r];
+    const float s = p.meta[2 * r + 1];
+    const F2 mn2 = f2_both(mn), s2 = f2_both(s);
+    F2 g[G::ITERS], yh[G::ITERS];
+    F2 dot2 = f2_both(0.0f);
+#pragma unroll
+    for (int i = 0; i < G::ITERS; ++i) {
+      float g0 = 0.0f, g1 = 0.0f;
+      uint32_t c0 = 0, c1 = 0;
+      if (G::has(i, ul)) {
+        const uint32_t wd = a0 + ul + UNIT_ * i;           // word of the tile; its elements are 2 wd, 2 wd + 1
+        const typename P::Raw w = P::load(p.data, wd);
+        g0 = P::lo(w);
+        g1 = P::hi(w);
+        if (NBITS == 8) {
+          const uint32_t b = *(const uint16_t*)(p.codes + 2u * wd);
+          c0 = b & 0xFFu;
+          c1 = b >> 8;
+        } else {
+          const uint32_t b = p.codes[wd >> 1] >> (4u * (wd & 1u));   // two words per byte
+          c0 = b & 3u;
+          c1 = (b >> 2) & 3u;
+        }
+      }
+      if (HP == 1 && i == 0 && ul == 0) g0 = 0.0f;
+      if (HP == 0 && i == G::LAST_I && ul == G::LAST_UL) g1 = 0.0f;
+      g[i] = f2_pack(g0, g1);
+      yh[i] = f2_fma(f2_pack((float)c0, (float)c1), s2, mn2);   // Eq. 9, one rounding each (as dequant)
+      dot2 = f2_fma(g[i], yh[i], dot2);
+    }
+    float d0, d1;
+    f2_unpack(dot2, d0, d1);
+    const float dot = u.template reduce<kOpSum>(d0 + d1);
+    const F2 dotv = f2_both(dot);
+#pragma unroll
+    for (int i = 0; i < G::ITERS; ++i) {
+      if (active && G::has(i, ul)) {
+        float o0, o1;
+        f2_unpack(f2_mul(yh[i], f2_sub(g[i], dotv)), o0, o1);
+        const typename P::Raw w = P::pack(o0, o1);
+        const bool drop_lo = HP == 1 && i == 0 && ul == 0;
+        const bool drop_hi = HP == 0 && i == G::LAST_I && ul == G::LAST_UL;
+        if (drop_lo) P::store_hi(p.data, a0 + ul + UNIT_ * i, w);
+        else if (drop_hi) P::store_lo(p.data, a0 + ul + UNIT_ * i, w);
+        else P::store(p.data, a0 + ul + UNIT_ * i, w);
+      }
+    }
+  }
+
+  static __device__ __forceinline__ void group(Unit<UNIT_>& u, State&, const StagePtrs& p, float*, uint32_t grp,
+                                               bool active, uint32_t) {
+    const uint32_t r = active ? 2 * grp : 0;
+    if (G::kOdd) {
+      row<0>(u, p, r, active);
+      u.sync();  // the odd row's first word holds the even row's last result
+      row<1>(u, p, r + 1, active);
+    } else {
+      row<2>(u, p, r, active);
+      row<2>(u, p, r + 1, active);
+    }
+    u.sync();
+  }
+};
+
 // ---------------------------------------------------------------- the kernel
 template <class WORK>
 __global__ void __maxnreg__(WORK::kMaxRegs) tile_kernel(TileKernelArgs a) {
@@ -2554,8 +2775,18 @@ cudaError_t launch_any_bits(const TilePlan& p, const TileKernelArgs& ka, cudaStr
 template <int KERNEL, int DT, int NBITS>
 cudaError_t launch_bits_unit(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
   if constexpr (KERNEL == kSoftmaxFwd) {
+    if (p.variant == kVariantPairFixed) {
+      if (ka.row_len == 197) return launch_work<PairSoftmaxFwdBits<DT, 8, 197, NBITS>>(p, ka, st);
+      if (ka.row_len == 257) return launch_work<PairSoftmaxFwdBits<DT, 8, 257, NBITS>>(p, ka, st);
+      return cudaErrorInvalidValue;
+    }
     return launch_any_bits<AnySoftmaxFwdBits, DT, NBITS>(p, ka, st);
   } else if constexpr (KERNEL == kSoftmaxBwd) {
+    if (p.variant == kVariantPairFixed) {
+      if (ka.row_len == 197) return launch_work<PairSoftmaxBwdBits<DT, 8, 197, NBITS>>(p, ka, st);
+      if (ka.row_len == 257) return launch_work<PairSoftmaxBwdBits<DT, 8, 257, NBITS>>(p, ka, st);
+      return cudaErrorInvalidValue;
+    }
     return launch_any_bits<AnySoftmaxBwdBits, DT, NBITS>(p, ka, st);
   } else if constexpr (KERNEL == kGeluFwd) {
     if (p.unit_lanes == 64) return launch_work<StreamActFwdBits<DT, 64, kActGelu, NBITS>>(p, ka, st);
