@@ -1,8 +1,8 @@
 """Turns an Nsight Compute report into the short text tables kept under profiles/.
 
-    python -m paper_2503_08154_b200.ncu_summary table  <report.ncu-rep> [--title T] [--command C]
+    python -m paper_2503_08154_b200.ncu_summary table  <report.ncu-rep> [more reports] [--title T] [--command C]
     python -m paper_2503_08154_b200.ncu_summary launches <launches.csv> [--title T] [--command C]
-    python -m paper_2503_08154_b200.ncu_summary traffic <report.ncu-rep> --workload NAME [--skip-first N]
+    python -m paper_2503_08154_b200.ncu_summary traffic <report.ncu-rep> [more reports] --workload NAME [--skip-first N]
 
 `table` prints one column per captured launch with the counters the roofline discussion uses
 (duration, DRAM bytes and throughput, issue and pipe utilisation, stalls, registers).
@@ -96,7 +96,9 @@ def fmt(metric, d):
 
 
 def cmd_table(args):
-    launches = read_raw(args.report)
+    launches = []
+    for rep in [args.report] + list(args.more):
+        launches += read_raw(rep)
     if args.title:
         print(args.title)
     if args.command:
@@ -151,9 +153,11 @@ KIND = (("SoftmaxFwd", "softmax_fwd"), ("SoftmaxBwd", "softmax_bwd"), ("ActFwd",
 
 
 def cmd_traffic(args):
-    launches = read_raw(args.report)
+    launches = []
+    for rep in [args.report] + list(args.more):
+        launches += read_raw(rep)[args.skip_first:]
     per = {}
-    for d in launches[args.skip_first:]:
+    for d in launches:
         kind = next((k for pat, k in KIND if pat in d["name"]), None)
         if kind is None or "dram__bytes_read.sum" not in d:
             continue
@@ -174,6 +178,7 @@ def main():
     for name in ("table", "launches", "traffic"):
         p = sub.add_parser(name)
         p.add_argument("report")
+        p.add_argument("more", nargs="*", help="further reports, appended (table and traffic)")
         p.add_argument("--title", default="")
         p.add_argument("--command", default="")
         if name == "traffic":
