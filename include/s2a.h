@@ -254,6 +254,17 @@ int s2a_lrp_fwd(const void* x, const float* A, const float* B, void* y, size_t b
  */
 int s2a_device_error(unsigned int* flags, int clear);
 
+/* Self-test of the bounded waits.  Enqueues one warp that waits, with a 2 ms limit, for a
+ * shared-memory barrier phase that nothing completes: the wait runs out, the kernel records
+ * bit 2 (value 4) in the CURRENT device's error word and returns.  Afterwards
+ * s2a_device_error reports 4 until it is cleared, and the context is as usable as before.
+ * It lets an integrator (and this library's tests) see the give-up path work without any
+ * real fault.  Bits 0 and 1 of the word belong to the pipelined kernels (a consumer gave up
+ * waiting for a tile; the copy lane gave up waiting for the consumers).  Returns S2A_OK or
+ * S2A_ERR_CUDA.  (The paper has no counterpart: this concerns the kernels' plumbing only.)
+ */
+int s2a_selftest_wait_expiry(void* cuda_stream);
+
 /* How a call would be run: writes into `out` (capacity `cap` bytes, always
  * NUL-terminated) a one-line description of the kernel variant and launch shape chosen
  * for (kernel, row_len, dt, n_elems).  kernel: 0 gelu_fwd, 1 gelu_bwd, 2 softmax_fwd,

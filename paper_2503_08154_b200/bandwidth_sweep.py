@@ -203,11 +203,45 @@ def cases(quick: bool):
     return out
 
 
+def table(path: str) -> None:
+    """Prints the compact table kept under profiles/ from the JSON lines of a sweep."""
+    rows = [json.loads(l) for l in open(path) if l.startswith("{")]
+    print("%-24s %-11s %-7s %-5s %9s %9s" % ("kernel pair", "rows", "row_len", "dtype", "fwd GB/s", "bwd GB/s"))
+    for r in rows:
+        if r.get("kernel_pair") in ("gelu", "silu", "softmax"):
+            print("%-24s %-11d %-7d %-5s %9.0f %9.0f" % (r["kernel_pair"], r["rows"], r["row_len"], r["io_dtype"],
+                                                         r["fwd_GBps"], r["bwd_GBps"]))
+    print()
+    for r in rows:
+        if str(r.get("kernel_pair", "")).endswith("_bits"):
+            print("%-24s %-11d %-7d %-5s %9.0f %9.0f   (Eq. 8 at %d bits)" % (r["kernel_pair"], r["rows"], r["row_len"], r["io_dtype"],
+                                                                            r["fwd_GBps"], r["bwd_GBps"], r["bits"]))
+    print()
+    for r in rows:
+        if r.get("kernel_pair") == "relu":
+            print("relu (1-bit mask)        n=%-12d %-5s fwd %6.0f bwd %6.0f" % (r["elems"], r["io_dtype"], r["fwd_GBps"], r["bwd_GBps"]))
+    print()
+    for r in rows:
+        if r.get("kernel") == "gelu_fwd_tensor_range":
+            print("gelu_fwd_tensor_range    n=%-12d %-5s %6.0f GB/s (x read twice: 6.5 / 12.5 B per element)" % (r["elems"], r["io_dtype"], r["GBps"]))
+    print()
+    for r in rows:
+        if r.get("kernel_pair") == "cap":
+            print("cap                      [%d, %d] r=%d %-5s fwd %6.0f bwd %6.0f" % (r["rows"], r["channels"], r["r"], r["io_dtype"],
+                                                                                     r["fwd_GBps"], r["bwd_GBps"]))
+        if r.get("kernel") == "lrp_fwd":
+            print("lrp_fwd                  %s" % json.dumps({k: v for k, v in r.items() if k != "note"}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--quick", action="store_true")
     ap.add_argument("--seeds", type=int, default=5)
+    ap.add_argument("--table", default="", help="print the compact table of a finished sweep's JSON lines and exit")
     args = ap.parse_args()
+    if args.table:
+        table(args.table)
+        return
     for line in _time_side(0):
         print(json.dumps(line), flush=True)
     for line in _time_bits(0):

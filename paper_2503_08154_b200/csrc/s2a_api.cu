@@ -239,6 +239,10 @@ int s2a_device_error(unsigned int* flags, int clear) {
   return read_error_word(flags, clear != 0) == cudaSuccess ? S2A_OK : S2A_ERR_CUDA;
 }
 
+int s2a_selftest_wait_expiry(void* cuda_stream) {
+  return launch_wait_expiry_probe((cudaStream_t)cuda_stream) == cudaSuccess ? S2A_OK : S2A_ERR_CUDA;
+}
+
 int s2a_describe_plan(int kernel, size_t n_elems, size_t row_len, int dt, char* out, size_t cap) {
   if (!out || cap == 0) return S2A_ERR_NULL;
   out[0] = 0;

@@ -20,6 +20,7 @@ constexpr float kLevels = 15.0f;   // 2^N - 1 with N = 4 (Eq. 8)
 // Bits of the per-device error word (see s2a_device_error).
 constexpr unsigned kErrLoadWait = 1u;   // a consumer gave up waiting for a tile to arrive
 constexpr unsigned kErrDrainWait = 2u;  // the producer gave up waiting for the consumers
+constexpr unsigned kErrSelfTest = 4u;   // set by s2a_selftest_wait_expiry only: its wait is meant to run out
 
 // ---------------------------------------------------------------- I/O element types
 template <int DT> struct Io;

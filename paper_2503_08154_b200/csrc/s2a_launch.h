@@ -96,4 +96,7 @@ cudaError_t launch_tile(int kernel, int dt, const TilePlan& p, const TileArgs& a
 // when a bounded wait runs out.  Synchronises the device.
 cudaError_t read_error_word(unsigned int* flags, bool clear);
 
+// Launches the bounded wait's self-test (a wait that is meant to run out after 2 ms).
+cudaError_t launch_wait_expiry_probe(cudaStream_t st);
+
 }  // namespace s2a

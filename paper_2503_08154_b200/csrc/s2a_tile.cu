@@ -366,6 +366,28 @@ cudaError_t launch_tile(int kernel, int dt, const TilePlan& p, const TileArgs& a
   return cudaErrorInvalidValue;
 }
 
+// One warp waits, with a 2 ms limit, for a barrier phase that nothing will ever complete: the
+// give-up path of the bounded wait (record the bit, return) run on purpose, so that a test can
+// see the error word change and the context stay usable.
+namespace {
+__global__ void wait_expiry_probe(unsigned int* error_word) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    fence_barrier_init();
+  }
+  __syncthreads();
+  mbar_wait(&bar, 0, error_word, kErrSelfTest, 2000000ull);
+}
+}  // namespace
+
+cudaError_t launch_wait_expiry_probe(cudaStream_t st) {
+  unsigned int* err = error_word_address();
+  if (!err) return cudaErrorInvalidDevice;
+  wait_expiry_probe<<<1, 32, 0, st>>>(err);
+  return cudaGetLastError();
+}
+
 cudaError_t read_error_word(unsigned int* flags, bool clear) {
   cudaError_t e = cudaMemcpyFromSymbol(flags, g_error_word, sizeof(unsigned int));
   if (e != cudaSuccess) return e;

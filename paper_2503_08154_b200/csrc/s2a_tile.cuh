@@ -110,13 +110,14 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 }
 // Bounded wait for the phase with the given parity to complete: gives up after
 // kWaitLimitNs of wall time or kSpinLimit tries, whichever comes first, and records why.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned int* err, unsigned err_bit) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned int* err, unsigned err_bit,
+                                          uint64_t limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_timer_ns();
 #pragma unroll 1
   for (uint32_t i = 0; i < kSpinLimit; ++i) {
     if (mbar_try_wait_suspend(bar, parity, kSuspendNs)) return true;
-    if (global_timer_ns() - t0 > kWaitLimitNs) break;
+    if (global_timer_ns() - t0 > limit_ns) break;
   }
   atomicOr(err, err_bit);
   return false;

@@ -570,6 +570,27 @@ def test_gelu_tensor_range_in_place_and_argument_errors():
         pu.assert_close(pu.widen(pu.to_host(xd, dt), dt), pu.widen(y_o, dt), dt, "gelu y (tensor range, in place)")
 
 
+def test_a_wait_that_runs_out_sets_the_error_word_and_leaves_the_context_usable():
+    # the self-test's wait has nothing to wait for: it must give up after its 2 ms, record its
+    # bit, and return; the word reads 4 until cleared, and ordinary calls work afterwards
+    import ctypes
+    lib = binding.lib()
+    lib.s2a_selftest_wait_expiry.argtypes = [ctypes.c_void_p]
+    lib.s2a_selftest_wait_expiry.restype = ctypes.c_int
+    flags = ctypes.c_uint(0)
+    assert lib.s2a_device_error(ctypes.byref(flags), 1) == 0
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    assert lib.s2a_selftest_wait_expiry(ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)) == 0
+    t1.record()
+    torch.cuda.synchronize()
+    assert 1.5 < t0.elapsed_time(t1) < 500.0, "the wait should give up after about 2 ms"
+    assert lib.s2a_device_error(ctypes.byref(flags), 0) == 0 and flags.value == 4
+    assert lib.s2a_device_error(ctypes.byref(flags), 1) == 0 and flags.value == 4
+    assert lib.s2a_device_error(ctypes.byref(flags), 0) == 0 and flags.value == 0
+    check_gelu(*_gelu_inputs(70, 3072, BF16, seed=4), 3072, BF16)       # the context is as usable as before
+
+
 def test_device_error_word_reads_zero_and_clears():
     # no kernel of this suite gives up on a wait: the word stays 0, and reading it with
     # clear = 1 leaves it 0 (the expiry path itself is not provoked on a shared GPU)
