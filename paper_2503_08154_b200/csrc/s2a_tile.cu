@@ -224,6 +224,20 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
   }
   int ctas_per_sm = 2;
   if (variant == kVariantStream && is_gelu) ctas_per_sm = 4;
+  // The GELU backward runs with eight warps on four-row tiles, two CTAs per SM: alone it gains
+  // 1-3 % (hidden 4096 / 5120, where two rows leave room for two stages only), and in training
+  // order, alternating with the softmax backward, the step gains 3 % (ViT-B/16 5733 -> 5917 GB/s,
+  // L/16 5392 -> 5559, H/14 5463 -> 5593): most of what that alternation used to cost.  The same
+  // shape for the GELU forward or the softmax kernels measured slower.
+  const int force = env_int("S2A_X2", 1);  // tuning: bit 0 gelu_bwd, 1 gelu_fwd, 2 softmax_bwd, 3 softmax_fwd
+  const bool wide_bwd = variant == kVariantStream && is_gelu && bits == 4 && unit == 64 &&
+                        ((is_act_bwd(kernel) && (force & 1)) || (is_act_fwd(kernel) && (force & 2)));
+  if (variant == kVariantPairFixed && bits == 4 && unit == 8 &&
+      ((kernel == kSoftmaxBwd && (force & 4)) || (kernel == kSoftmaxFwd && (force & 8)))) {
+    warps = 8;
+    ctas_per_sm = 2;
+  }
+  if (wide_bwd) { warps = 8; ctas_per_sm = 2; }
   if (variant == kVariantPairFixed) ctas_per_sm = 4;
   // one row at a time per unit; 2 bits: 64-row tiles (whole 16-byte code spans), eight warps, two
   // CTAs per SM; 8 bits: measured best with the 4-bit kernels' shape (5.2 against 4.9 TB/s)
