@@ -278,8 +278,14 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
   // with programmatic dependent launch the next kernel's CTAs move into the slots that
   // this kernel's CTAs leave, which only works smoothly when the slots have equal sizes
   // (measured: 50.5 KB and 52.5 KB requests in alternation cost 3.7 us per launch).
+  // The fixed-width softmax backward with a tile too large for three stages in a quarter of the
+  // shared memory (width 257: 20.9 KB stages) takes a third of it: three CTAs of three stages
+  // measured 2.5 % faster than four of two (the forward, and width 197, measured slower that way).
+  if (variant == kVariantPairFixed && kernel == kSoftmaxBwd && bits == 4 && ctas_per_sm == 4 &&
+      (kMaxSmem / 4 - 1024 - kHeaderBytes) / stage_bytes < 3 && (kMaxSmem / 3 - 1024 - kHeaderBytes) / stage_bytes >= 3)
+    ctas_per_sm = 3;
   ctas_per_sm = env_int("S2A_CTAS_PER_SM", ctas_per_sm);
-  if (ctas_per_sm != 1 && ctas_per_sm != 2 && ctas_per_sm != 4) ctas_per_sm = 2;
+  if (ctas_per_sm < 1 || ctas_per_sm > 4) ctas_per_sm = 2;
   {
     // registers bound the residency too: the kernels' register caps, by variant
     uint32_t regs = 128;
@@ -294,7 +300,7 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
                                : ((pair_bits && bits == 2 && kernel == kSoftmaxFwd) ? align_up(rows * L, 128) : 0u);
   const int env_stages = env_int("S2A_STAGES", 0);
   uint32_t stages = 0, smem = 0;
-  for (int c = ctas_per_sm; c >= 1 && stages == 0; c /= 2) {
+  for (int c = ctas_per_sm; c >= 1 && stages == 0; c = (c == 3 ? 2 : c / 2)) {
     const uint32_t budget = kMaxSmem / (uint32_t)c - 1024;  // 1 KiB per CTA is the system's
     const uint32_t fixed = kHeaderBytes + extra_bytes;
     uint32_t fit = budget > fixed ? (budget - fixed) / stage_bytes : 0;
