@@ -1446,14 +1446,40 @@ struct AnySoftmaxFwd {
   using V = V16<DT>;
   using R = AnyRow<DT>;
   static constexpr int EPA = V::EPA;
+  static constexpr int NP = EPA / 2;              // packed binary32 pairs per vector
   static constexpr int kVPW = EPA == 8 ? 1 : 2;  // vectors per 32-bit word of codes
   struct State {};
   static __device__ __forceinline__ void init(State&) {}
   static __device__ __forceinline__ uint32_t rows_per_group(uint32_t) { return 1u; }
 
-  static __device__ __forceinline__ float ex(float x, float m, float nm) {
-    constexpr float kLog2e = 1.4426950408889634f;
-    return DT == kBF16 ? ex2_approx(fmaf(x, kLog2e, nm)) : exp_eval<DT>(x - m);
+  // The vector's elements as packed binary32 pairs (exact).
+  static __device__ __forceinline__ void pairs_of(const typename V::Raw& raw, F2* x) {
+    if constexpr (DT == kBF16) {
+      const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+      for (int k = 0; k < 4; ++k) x[k] = f2_from_bf16x2(w[k]);
+    } else {
+      x[0] = f2_pack(raw.x, raw.y);
+      x[1] = f2_pack(raw.z, raw.w);
+    }
+  }
+  // e^(x - m) for the vector's elements: bfloat16 with one fused multiply-add per exponent
+  // argument (c2 = -m log2 e), binary32 with the difference, then the product (c2 = m).
+  static __device__ __forceinline__ void exps_of(const typename V::Raw& raw, F2 c2, F2* e) {
+    const F2 k2 = f2_both(1.4426950408889634f);
+    pairs_of(raw, e);
+#pragma unroll
+    for (int k = 0; k < NP; ++k) {
+      float a, b;
+      f2_unpack(DT == kBF16 ? f2_fma(e[k], k2, c2) : f2_mul(k2, f2_sub(e[k], c2)), a, b);
+      e[k] = f2_pack(ex2_approx(a), ex2_approx(b));
+    }
+  }
+  // Keeps the elements named by msk (bit 2k: low half of pair k, bit 2k + 1: high half), others become `other`.
+  static __device__ __forceinline__ F2 masked(F2 v, uint32_t msk, int k, float other) {
+    float a, b;
+    f2_unpack(v, a, b);
+    return f2_pack((msk >> (2 * k) & 1u) ? a : other, (msk >> (2 * k + 1) & 1u) ? b : other);
   }
 
   static __device__ __forceinline__ void row(Unit<UNIT_>& u, const StagePtrs& p, uint32_t r, bool active, uint32_t L) {
@@ -1477,36 +1503,46 @@ struct AnySoftmaxFwd {
     });
     m = u.template reduce<kOpMax>(fmaxf(m, pm.hi()));
     if (!active) m = 0.0f;
-    const float nm = -m * 1.4426950408889634f;
+    const F2 c2 = f2_both(DT == kBF16 ? -m * 1.4426950408889634f : m);
     // ---- sum of exponentials
-    float z = 0.0f;
+    F2 z2 = f2_both(0.0f);
     any_row_vectors<DT, UNIT_, kVPW>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
-      float v[EPA];
-      V::widen(*(const typename V::Raw*)(p.data + j * 16u), v);
+      F2 e[NP];
+      exps_of(*(const typename V::Raw*)(p.data + j * 16u), c2, e);
 #pragma unroll
-      for (int k = 0; k < EPA; ++k) {
-        const float e = ex(v[k], m, nm);
-        if constexpr (decltype(interior)::value) z += e;
-        else z += (msk >> k & 1u) ? e : 0.0f;
+      for (int k = 0; k < NP; ++k) {
+        if constexpr (decltype(interior)::value) z2 = f2_add(z2, e[k]);
+        else z2 = f2_add(z2, masked(e[k], msk, k, 0.0f));
       }
     });
-    z = u.template reduce<kOpSum>(z);
-    const float rz = __fdiv_rn(1.0f, active ? z : 1.0f);
+    float z0, z1;
+    f2_unpack(z2, z0, z1);
+    const float z = u.template reduce<kOpSum>(z0 + z1);
+    const F2 rz2 = f2_both(__fdiv_rn(1.0f, active ? z : 1.0f));
     // ---- y, written in place, and the range of y as written
     float mn = INFINITY, mx = -INFINITY;
     typename V::MinMax py;
     py.init();
     any_row_vectors<DT, UNIT_, kVPW>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
-      float v[EPA];
-      V::widen(*(const typename V::Raw*)(p.data + j * 16u), v);
-#pragma unroll
-      for (int k = 0; k < EPA; ++k) v[k] = ex(v[k], m, nm) * rz;
-      const typename V::Raw yw = V::narrow(v);  // v now holds y as written
+      F2 e[NP];
+      exps_of(*(const typename V::Raw*)(p.data + j * 16u), c2, e);
+      typename V::Raw yw;
+      if constexpr (DT == kBF16) {
+        yw = make_uint4(f2_to_bf16x2(f2_mul(e[0], rz2)), f2_to_bf16x2(f2_mul(e[1], rz2)), f2_to_bf16x2(f2_mul(e[2], rz2)),
+                        f2_to_bf16x2(f2_mul(e[3], rz2)));
+      } else {
+        float a, b, c, d;
+        f2_unpack(f2_mul(e[0], rz2), a, b);
+        f2_unpack(f2_mul(e[1], rz2), c, d);
+        yw = make_float4(a, b, c, d);
+      }
       if constexpr (decltype(interior)::value) {
         *(typename V::Raw*)(p.data + j * 16u) = yw;
         py.add(yw);
       } else {
         R::store(p.data, j, yw, msk);
+        float v[EPA];
+        V::widen(yw, v);  // y as written
 #pragma unroll
         for (int k = 0; k < EPA; ++k) {
           mn = fminf(mn, (msk >> k & 1u) ? v[k] : INFINITY);
@@ -1518,21 +1554,23 @@ struct AnySoftmaxFwd {
     mx = u.template reduce<kOpMax>(fmaxf(mx, py.hi()));
     const QRange q = make_qrange(mn, mx);
     if (active && ul == 0) { p.meta[2 * r] = q.mn; p.meta[2 * r + 1] = q.s; }
+    const F2 min2 = f2_both(q.mn), inv2 = f2_both(q.inv), magic2 = f2_both(12582912.0f);
     // ---- codes of y as written (each lane reads back the vectors it wrote itself)
     any_row_vectors<DT, UNIT_, kVPW>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
-      float v[EPA];
-      V::widen(*(const typename V::Raw*)(p.data + j * 16u), v);
-      CodePacker<EPA> pk;
-      pk.init();
-      if constexpr (decltype(interior)::value) {
+      F2 y[NP];
+      pairs_of(*(const typename V::Raw*)(p.data + j * 16u), y);
+      uint32_t acc = 0u - kMagicBits * CodePacker<EPA>::kOnes;  // see CodePacker
 #pragma unroll
-        for (int k = 0; k < EPA; ++k) pk.add(k, v[k], q);
-        V::store_codes(p.codes, j, pk.acc);
-      } else {
-#pragma unroll
-        for (int k = 0; k < EPA; ++k) pk.add(k, (msk >> k & 1u) ? v[k] : q.mn, q);  // a neighbour's element codes as 0
-        any_merge_codes<4, EPA>(p.codes, j, &pk.acc, msk);
+      for (int k = 0; k < NP; ++k) {
+        // a neighbour's element codes as 0 (it is replaced by the minimum)
+        const F2 v = decltype(interior)::value ? y[k] : masked(y[k], msk, k, q.mn);
+        float t0, t1;
+        f2_unpack(f2_add(f2_scaled(v, min2, inv2), magic2), t0, t1);
+        acc += __float_as_uint(t0) << (8 * k);
+        acc += __float_as_uint(t1) << (8 * k + 4);
       }
+      if constexpr (decltype(interior)::value) V::store_codes(p.codes, j, acc);
+      else any_merge_codes<4, EPA>(p.codes, j, &acc, msk);
     });
   }
 
@@ -1551,10 +1589,17 @@ struct AnySoftmaxBwd {
   static constexpr int UNIT = UNIT_;
   using V = V16<DT>;
   using R = AnyRow<DT>;
+  using F = AnySoftmaxFwd<DT, UNIT_>;
   static constexpr int EPA = V::EPA;
+  static constexpr int NP = EPA / 2;
   struct State {};
   static __device__ __forceinline__ void init(State&) {}
   static __device__ __forceinline__ uint32_t rows_per_group(uint32_t) { return 1u; }  // codes are only read
+
+  // Eq. 9 for the two codes of pair k of a vector (one rounding each, as dequant).
+  static __device__ __forceinline__ F2 yhat(uint32_t bits, int k, F2 s2, F2 mn2) {
+    return f2_fma(f2_pack((float)((bits >> (8 * k)) & 0xFu), (float)((bits >> (8 * k + 4)) & 0xFu)), s2, mn2);
+  }
 
   static __device__ __forceinline__ void group(Unit<UNIT_>& u, State&, const StagePtrs& p, float*, uint32_t r,
                                                bool active, uint32_t L) {
@@ -1562,28 +1607,36 @@ struct AnySoftmaxBwd {
     R g;
     g.set(active ? r : 0u, L);
     const int ul = u.ul;
-    const float mn = active ? p.meta[2 * r] : 0.0f;
-    const float s = active ? p.meta[2 * r + 1] : 0.0f;
-    float dot = 0.0f;
+    const F2 mn2 = f2_both(active ? p.meta[2 * r] : 0.0f), s2 = f2_both(active ? p.meta[2 * r + 1] : 0.0f);
+    F2 dot2 = f2_both(0.0f);
     any_row_vectors<DT, UNIT_>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
-      float v[EPA];
-      V::widen(*(const typename V::Raw*)(p.data + j * 16u), v);
+      F2 gv[NP];
+      F::pairs_of(*(const typename V::Raw*)(p.data + j * 16u), gv);
       const uint32_t bits = V::load_codes(p.codes, j);
 #pragma unroll
-      for (int k = 0; k < EPA; ++k) {
-        const float yh = dequant((bits >> (4 * k)) & 0xFu, mn, s);
-        if constexpr (decltype(interior)::value) dot = fmaf(v[k], yh, dot);
-        else dot = fmaf((msk >> k & 1u) ? v[k] : 0.0f, yh, dot);
+      for (int k = 0; k < NP; ++k) {
+        const F2 gk = decltype(interior)::value ? gv[k] : F::masked(gv[k], msk, k, 0.0f);
+        dot2 = f2_fma(gk, yhat(bits, k, s2, mn2), dot2);
       }
     });
-    dot = u.template reduce<kOpSum>(dot);
+    float d0, d1;
+    f2_unpack(dot2, d0, d1);
+    const F2 dotv = f2_both(u.template reduce<kOpSum>(d0 + d1));
     any_row_vectors<DT, UNIT_>(g, ul, active, [&](uint32_t j, uint32_t msk, auto interior) {
-      float v[EPA];
-      V::widen(*(const typename V::Raw*)(p.data + j * 16u), v);
+      F2 gv[NP];
+      F::pairs_of(*(const typename V::Raw*)(p.data + j * 16u), gv);
       const uint32_t bits = V::load_codes(p.codes, j);
 #pragma unroll
-      for (int k = 0; k < EPA; ++k) v[k] = dequant((bits >> (4 * k)) & 0xFu, mn, s) * (v[k] - dot);
-      const typename V::Raw ow = V::narrow(v);
+      for (int k = 0; k < NP; ++k) gv[k] = f2_mul(yhat(bits, k, s2, mn2), f2_sub(gv[k], dotv));
+      typename V::Raw ow;
+      if constexpr (DT == kBF16) {
+        ow = make_uint4(f2_to_bf16x2(gv[0]), f2_to_bf16x2(gv[1]), f2_to_bf16x2(gv[2]), f2_to_bf16x2(gv[3]));
+      } else {
+        float a, b, c, d;
+        f2_unpack(gv[0], a, b);
+        f2_unpack(gv[1], c, d);
+        ow = make_float4(a, b, c, d);
+      }
       if constexpr (decltype(interior)::value) *(typename V::Raw*)(p.data + j * 16u) = ow;
       else R::store(p.data, j, ow, msk);
     });
