@@ -2059,12 +2059,13 @@ struct PairSoftmaxFwd<kBF16, UNIT_, LCT> {
     return f2_code_byte(f2_pack(v0, v1), min2, inv2) & 0xFFu;
   }
 
-  static __device__ __forceinline__ void group(Unit<UNIT_>& u, State&, const StagePtrs& p, float*, uint32_t grp,
-                                               bool active, uint32_t) {
-    const uint32_t r = active ? 2 * grp : 0;
+  // Everything up to the quantiser ranges of the pair's two rows (rows r and r + 1): y is
+  // written, A.w / B.w hold y as written, the metadata is stored.  LEVELS = 2^N - 1 of Eq. 8.
+  template <int LEVELS>
+  static __device__ __forceinline__ void front(Unit<UNIT_>& u, const StagePtrs& p, uint32_t r, bool active, Regs& A,
+                                               Regs& B, QRange& qA, QRange& qB) {
     const int ul = u.ul;
     const uint32_t a0 = (r * (uint32_t)LCT) >> 1, a1 = ((r + 1) * (uint32_t)LCT) >> 1;  // odd: a1 = a0 + NACC - 1
-    Regs A, B;
     constexpr int HA = G::kOdd ? 0 : 2, HB = G::kOdd ? 1 : 2;  // the kinds of the pair's two rows
     float mA = load_max<HA>(A, (const uint32_t*)p.data + a0 + ul, ul);
     float mB = load_max<HB>(B, (const uint32_t*)p.data + a1 + ul, ul);
@@ -2096,15 +2097,14 @@ struct PairSoftmaxFwd<kBF16, UNIT_, LCT> {
     scale_store<HB>(B, __fmaf_rn(__fmaf_rn(-zB, rB0, 1.0f), rB0, rB0), (uint32_t*)p.data + a1 + ul, ul, active, mnB, mxB);
     reduce_minmax_bf16<UNIT_>(mnA, mxA);
     reduce_minmax_bf16<UNIT_>(mnB, mxB);
-    // Eq. 8's two correctly rounded quotients per row, 15 / d and d / 15, for both rows with ONE
-    // division: lane 0 of the unit forms 15 / dA, lane 1 dA / 15, lane 2 15 / dB, lane 3 dB / 15
+    // Eq. 8's two correctly rounded quotients per row, LEVELS / d and d / LEVELS, for both rows with ONE
+    // division: lane 0 of the unit forms LEVELS / dA, lane 1 dA / LEVELS, lane 2 LEVELS / dB, lane 3 dB / LEVELS
     // (the other lanes repeat them), and four shuffles hand the results round.
-    QRange qA, qB;
     {
       const float dA = __fsub_rn(mxA, mnA), dB = __fsub_rn(mxB, mnB);
       const float d = (ul & 2) ? dB : dA;
       const bool odd = (ul & 1) != 0;
-      float quo = __fdiv_rn(odd ? d : kLevels, odd ? kLevels : d);
+      float quo = __fdiv_rn(odd ? d : (float)LEVELS, odd ? (float)LEVELS : d);
       if (d == 0.0f) quo = 0.0f;  // a constant row: inv = s = 0
       const int base = threadIdx.x & 31 & ~(UNIT_ - 1);
       qA.mn = mnA;
@@ -2118,6 +2118,17 @@ struct PairSoftmaxFwd<kBF16, UNIT_, LCT> {
       p.meta[2 * r] = qA.mn; p.meta[2 * r + 1] = qA.s;
       p.meta[2 * r + 2] = qB.mn; p.meta[2 * r + 3] = qB.s;
     }
+  }
+
+  static __device__ __forceinline__ void group(Unit<UNIT_>& u, State&, const StagePtrs& p, float*, uint32_t grp,
+                                               bool active, uint32_t) {
+    const uint32_t r = active ? 2 * grp : 0;
+    const int ul = u.ul;
+    const uint32_t a0 = (r * (uint32_t)LCT) >> 1, a1 = ((r + 1) * (uint32_t)LCT) >> 1;
+    Regs A, B;
+    QRange qA, qB;
+    constexpr int HA = G::kOdd ? 0 : 2, HB = G::kOdd ? 1 : 2;  // the kinds of the pair's two rows
+    front<15>(u, p, r, active, A, B, qA, qB);
     // The byte the two rows share: row A's last element is its low nibble, row B's first
     // its high nibble.  A's nibble travels by shuffle to the lane that owns B's first word.
     const F2 minA = f2_both(qA.mn), invA = f2_both(qA.inv), minB = f2_both(qB.mn), invB = f2_both(qB.inv);
@@ -2342,6 +2353,71 @@ struct PairSoftmaxFwdBits {
         }
       }
       __syncwarp();  // the scratch bytes are free again for the warp's next round
+    }
+  }
+};
+
+// bfloat16 form of the forward at 2 and 8 bits: the two rows of a pair are worked on together
+// by the 4-bit kernel's own front part (packed arithmetic, shared shuffle chains, one division);
+// only the code phase differs -- a byte per element into the code area (8 bits) or into the
+// scratch that the warp then packs (2 bits).
+template <int UNIT_, int LCT, int NBITS>
+struct PairSoftmaxFwdBits<kBF16, UNIT_, LCT, NBITS> {
+  static_assert(NBITS == 2 || NBITS == 8, "4 bits have kernels of their own");
+  static_assert(UNIT_ == 8, "four units per warp: eight consecutive rows per warp and round");
+  using B4 = PairSoftmaxFwd<kBF16, UNIT_, LCT>;
+  using G = PairGeom<UNIT_, LCT>;
+  static constexpr int kMaxRegs = 96;
+  static constexpr int kKernel = kSoftmaxFwd;
+  static constexpr int UNIT = UNIT_;
+  static constexpr int kTabFloats = 0;  // `tab` is the CTA's scratch area itself, not a per-unit table
+  struct State {};
+  static __device__ __forceinline__ void init(State&) {}
+  static __device__ __forceinline__ uint32_t rows_per_group(uint32_t) { return 2u; }
+
+  static __device__ __forceinline__ void group(Unit<UNIT_>& u, State&, const StagePtrs& p, float* tab, uint32_t grp,
+                                               bool active, uint32_t) {
+    const uint32_t r = active ? 2 * grp : 0;
+    const int ul = u.ul;
+    const uint32_t a0 = (r * (uint32_t)LCT) >> 1, a1 = ((r + 1) * (uint32_t)LCT) >> 1;
+    typename B4::Regs A, B;
+    QRange qA, qB;
+    constexpr int HA = G::kOdd ? 0 : 2, HB = G::kOdd ? 1 : 2;
+    B4::template front<(1 << NBITS) - 1>(u, p, r, active, A, B, qA, qB);
+    unsigned char* bytes = NBITS == 8 ? p.codes : (unsigned char*)tab;
+    const F2 minA = f2_both(qA.mn), invA = f2_both(qA.inv), minB = f2_both(qB.mn), invB = f2_both(qB.inv);
+    const F2 magic2 = f2_both(12582912.0f);
+    constexpr uint32_t kMask = (1u << NBITS) - 1u;
+#pragma unroll
+    for (int i = 0; i < G::ITERS; ++i) {
+      if (active && G::has(i, ul)) {
+        float t0, t1;
+        f2_unpack(f2_add(f2_scaled(f2_from_bf16x2(A.w[i]), minA, invA), magic2), t0, t1);
+        uint32_t c0 = __float_as_uint(t0) & kMask, c1 = __float_as_uint(t1) & kMask;
+        unsigned char* dst = bytes + 2u * (a0 + ul + UNIT_ * i);
+        if (B4::template drop_hi<HA>(i, ul)) dst[0] = (unsigned char)c0;   // the high half is row B's first element
+        else *(uint16_t*)dst = (uint16_t)(c0 | (c1 << 8));
+        f2_unpack(f2_add(f2_scaled(f2_from_bf16x2(B.w[i]), minB, invB), magic2), t0, t1);
+        c0 = __float_as_uint(t0) & kMask;
+        c1 = __float_as_uint(t1) & kMask;
+        dst = bytes + 2u * (a1 + ul + UNIT_ * i);
+        if (B4::template drop_lo<HB>(i, ul)) dst[1] = (unsigned char)c1;   // the low half is row A's last element
+        else *(uint16_t*)dst = (uint16_t)(c0 | (c1 << 8));
+      }
+    }
+    u.sync();
+    if (NBITS == 2) {
+      // as the general form: the warp packs its own eight consecutive rows
+      __syncwarp();
+      const uint32_t e_begin = (grp - (uint32_t)(u.uid & 3)) * 2u * (uint32_t)LCT;
+      if (active) {
+        for (uint32_t b = threadIdx.x & 31u; b < 2u * (uint32_t)LCT; b += 32u) {
+          const uint32_t w = *(const uint32_t*)(bytes + e_begin + 4u * b);
+          p.codes[e_begin / 4u + b] =
+              (unsigned char)((w & 3u) | ((w >> 6) & 0xCu) | ((w >> 12) & 0x30u) | ((w >> 18) & 0xC0u));
+        }
+      }
+      __syncwarp();
     }
   }
 };
