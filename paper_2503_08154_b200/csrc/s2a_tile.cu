@@ -224,27 +224,22 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
   }
   int ctas_per_sm = 2;
   if (variant == kVariantStream && is_gelu) ctas_per_sm = 4;
+  if (variant == kVariantPairFixed) ctas_per_sm = 4;
   // The GELU backward runs with eight warps on four-row tiles, two CTAs per SM: alone it gains
   // 1-3 % (hidden 4096 / 5120, where two rows leave room for two stages only), and in training
   // order, alternating with the softmax backward, the step gains 3 % (ViT-B/16 5733 -> 5917 GB/s,
-  // L/16 5392 -> 5559, H/14 5463 -> 5593): most of what that alternation used to cost.  The same
-  // shape for the GELU forward or the softmax kernels measured slower.
-  const int force = env_int("S2A_X2", 1);  // tuning: bit 0 gelu_bwd, 1 gelu_fwd, 2 softmax_bwd, 3 softmax_fwd
+  // L/16 5392 -> 5559, H/14 5463 -> 5593): most of what that alternation used to cost.
   // The forward takes the same shape only where two rows leave room for just two stages in a quarter
   // of the shared memory (hidden 4096 / 5120): alone it is then a little slower (5.78 -> 5.53 TB/s at
   // 4096), but alternating with the softmax forward the pair stops losing 4 us per launch (ViT-L/16
-  // step 5598 -> 5727 GB/s; H/14 unchanged); at hidden 3072 (three stages) it measured slower both ways.
+  // step 5598 -> 5727 GB/s; H/14 unchanged); at hidden 3072 (three stages) it measured slower both
+  // ways, and so did this shape for either softmax kernel.
+  const int shape_bits = env_int("S2A_X2", 1);  // tuning: bit 0 backward, bit 1 forward always, bit 4 forward never
   const bool two_stage_rows = (uint64_t)2 * L * esize * 5 / 4 > 17 * 1024;
-  const bool wide_bwd = variant == kVariantStream && is_gelu && bits == 4 && unit == 64 &&
-                        ((is_act_bwd(kernel) && (force & 1)) ||
-                         (is_act_fwd(kernel) && ((force & 2) || (two_stage_rows && (force & 16) == 0))));
-  if (variant == kVariantPairFixed && bits == 4 && unit == 8 &&
-      ((kernel == kSoftmaxBwd && (force & 4)) || (kernel == kSoftmaxFwd && (force & 8)))) {
-    warps = 8;
-    ctas_per_sm = 2;
-  }
-  if (wide_bwd) { warps = 8; ctas_per_sm = 2; }
-  if (variant == kVariantPairFixed) ctas_per_sm = 4;
+  const bool wide_rows = variant == kVariantStream && is_gelu && bits == 4 && unit == 64 &&
+                         ((is_act_bwd(kernel) && (shape_bits & 1)) ||
+                          (is_act_fwd(kernel) && ((shape_bits & 2) || (two_stage_rows && (shape_bits & 16) == 0))));
+  if (wide_rows) { warps = 8; ctas_per_sm = 2; }
   // one row at a time per unit; 2 bits: 64-row tiles (whole 16-byte code spans), eight warps, two
   // CTAs per SM; 8 bits: measured best with the 4-bit kernels' shape (5.2 against 4.9 TB/s)
   if (pair_bits && bits == 2) { warps = 8; ctas_per_sm = 2; }
