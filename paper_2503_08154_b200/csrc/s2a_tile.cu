@@ -221,8 +221,16 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
     // on shuffles; binary32 rows with 32 elements per lane run best with four, except the
     // one-warp units of 1024-element rows (measured at 512, 1024, 2048 and 4096).
     warps = (dt == kBF16 || iters * epa <= 16 || unit == 32) ? 8u : 4u;
+    // The bfloat16 backward is light enough for four warps wherever a row is not exactly a warp's
+    // (measured with the L2 prefetch in place, 4 against 8 warps: 128: 6.0 / 5.5 TB/s, 256: 6.2 / 5.6,
+    // 512: 6.2 / 5.5, 2048: 6.5 / 5.8, 4096: 6.5 / 5.8; 1024, one warp per row: 5.7 / 6.2).
+    if (dt == kBF16 && kernel == kSoftmaxBwd && unit >= 8 && unit != 32) warps = 4;
   }
-  int ctas_per_sm = 2;
+  // bfloat16 rows of 40..64 elements (four lanes per row): four CTAs of four warps on 7-12 KB tiles
+  // (64: forward 4.9 -> 5.1 TB/s, backward 5.8 -> 6.2)
+  const bool short_rows = variant == kVariantStream && !is_gelu && dt == kBF16 && unit == 4 && bits == 4;
+  if (short_rows) warps = 4;
+  int ctas_per_sm = short_rows ? 4 : 2;
   if (variant == kVariantStream && is_gelu) ctas_per_sm = 4;
   if (variant == kVariantPairFixed) ctas_per_sm = 4;
   // The GELU backward runs with eight warps on four-row tiles, two CTAs per SM: alone it gains
@@ -260,9 +268,11 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
   const uint32_t want_rows = n_units * G;
   while (rows % want_rows != 0 && (uint64_t)(rows + r_min) * L * esize <= kMaxStageBytes) rows += r_min;
   while ((uint64_t)rows * L * esize < 16 * 1024 && (uint64_t)rows * 2 * L * esize <= kMaxStageBytes) rows *= 2;
-  if ((variant == kVariantStream && is_gelu) || variant == kVariantPairFixed) {
+  if ((variant == kVariantStream && is_gelu) || variant == kVariantPairFixed || short_rows) {
     rows = r_min;  // small tiles: more CTAs per SM, each with its own pipeline
     while (rows % (n_units * G) != 0 && (uint64_t)(rows + r_min) * L * esize <= kMaxStageBytes) rows += r_min;
+    if (short_rows)
+      while ((uint64_t)rows * L * esize < 7 * 1024) rows *= 2;
   }
   rows = (uint32_t)env_int("S2A_TILE_ROWS", (int)rows);
   if (rows == 0 || rows % r_min != 0 || rows % G != 0 || (uint64_t)rows * L * esize > kHardStageBytes) return p;
