@@ -2346,10 +2346,12 @@ struct PairSoftmaxFwdBits {
       __syncwarp();
       const uint32_t e_begin = (grp - (uint32_t)(u.uid & 3)) * 2u * (uint32_t)LCT;
       if (active) {
-        for (uint32_t b = threadIdx.x & 31u; b < 2u * (uint32_t)LCT; b += 32u) {
-          const uint32_t w = *(const uint32_t*)(bytes + e_begin + 4u * b);
-          p.codes[e_begin / 4u + b] =
-              (unsigned char)((w & 3u) | ((w >> 6) & 0xCu) | ((w >> 12) & 0x30u) | ((w >> 18) & 0xC0u));
+        // eight scratch bytes (8-byte aligned: e_begin is a multiple of 8 L) make two code bytes
+        for (uint32_t b = threadIdx.x & 31u; b < (uint32_t)LCT; b += 32u) {
+          const uint2 w = *(const uint2*)(bytes + e_begin + 8u * b);
+          const uint32_t lo = (w.x & 3u) | ((w.x >> 6) & 0xCu) | ((w.x >> 12) & 0x30u) | ((w.x >> 18) & 0xC0u);
+          const uint32_t hi = (w.y & 3u) | ((w.y >> 6) & 0xCu) | ((w.y >> 12) & 0x30u) | ((w.y >> 18) & 0xC0u);
+          *(uint16_t*)(p.codes + e_begin / 4u + 2u * b) = (uint16_t)(lo | (hi << 8));
         }
       }
       __syncwarp();  // the scratch bytes are free again for the warp's next round
@@ -2411,10 +2413,12 @@ struct PairSoftmaxFwdBits<kBF16, UNIT_, LCT, NBITS> {
       __syncwarp();
       const uint32_t e_begin = (grp - (uint32_t)(u.uid & 3)) * 2u * (uint32_t)LCT;
       if (active) {
-        for (uint32_t b = threadIdx.x & 31u; b < 2u * (uint32_t)LCT; b += 32u) {
-          const uint32_t w = *(const uint32_t*)(bytes + e_begin + 4u * b);
-          p.codes[e_begin / 4u + b] =
-              (unsigned char)((w & 3u) | ((w >> 6) & 0xCu) | ((w >> 12) & 0x30u) | ((w >> 18) & 0xC0u));
+        // eight scratch bytes (8-byte aligned: e_begin is a multiple of 8 L) make two code bytes
+        for (uint32_t b = threadIdx.x & 31u; b < (uint32_t)LCT; b += 32u) {
+          const uint2 w = *(const uint2*)(bytes + e_begin + 8u * b);
+          const uint32_t lo = (w.x & 3u) | ((w.x >> 6) & 0xCu) | ((w.x >> 12) & 0x30u) | ((w.x >> 18) & 0xC0u);
+          const uint32_t hi = (w.y & 3u) | ((w.y >> 6) & 0xCu) | ((w.y >> 12) & 0x30u) | ((w.y >> 18) & 0xC0u);
+          *(uint16_t*)(p.codes + e_begin / 4u + 2u * b) = (uint16_t)(lo | (hi << 8));
         }
       }
       __syncwarp();
