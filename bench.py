@@ -443,6 +443,8 @@ def run_ours(args, shape, blocks, rank, world):
     clocks = sampler.finish(t0, t1)
     total_ms = statistics.median(region_ms)
     spread = (max(region_ms) - min(region_ms)) / total_ms
+    ordered = sorted(region_ms)
+    spread_p10_p90 = (ordered[int(0.9 * (len(ordered) - 1))] - ordered[int(0.1 * (len(ordered) - 1))]) / total_ms
     if binding.s2a_device_error() != 0:
         raise RuntimeError("a kernel gave up on a bounded wait during the timed region")
 
@@ -594,7 +596,7 @@ def run_ours(args, shape, blocks, rank, world):
     line = {
         "metric": "s2a_fwd_bwd_algorithmic_bandwidth", "value": value, "unit": "GB/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
-        "repeats": repeats, "spread": spread, "timing": "median of %d regions of %d steps each" % (repeats, args.steps),
+        "repeats": repeats, "spread": spread, "spread_p10_p90": spread_p10_p90, "timing": "median of %d regions of %d steps each" % (repeats, args.steps),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": shape.name, "blocks": blocks, "io_dtype": "bf16" if shape.dtype else "f32",
