@@ -570,7 +570,7 @@ def run_ours(args, shape, blocks, rank, world):
         # for that block (same inputs) is compared with them: the counts go into the line.
         parity = {"blocks_checked": 0, "gelu_elements": 0, "gelu_code_mismatches": 0, "gelu_meta_mismatches": 0,
                   "softmax_elements": 0, "softmax_code_flips": 0, "softmax_flips_not_at_a_bin_edge": 0,
-                  "softmax_meta_mismatches": 0}
+                  "softmax_rows_whose_range_moved_by_rounding": 0}
 
         def count_parity(i, arrays, fwd):
             B = blks[i]
@@ -585,7 +585,7 @@ def run_ours(args, shape, blocks, rank, world):
                 parity["softmax_elements"] += int(sy.size)
                 parity["softmax_code_flips"] += flips
                 parity["softmax_flips_not_at_a_bin_edge"] += outside
-                parity["softmax_meta_mismatches"] += int(np.count_nonzero(
+                parity["softmax_rows_whose_range_moved_by_rounding"] += int(np.count_nonzero(
                     (B.smeta.cpu().numpy().view(np.uint32) != sm.view(np.uint32)).reshape(-1, 2).any(axis=1)))
 
         gbs, gel, dtc_s, sample = oracle_sample_rate(shape, np_blocks, threads, on_block=count_parity)
