@@ -265,6 +265,20 @@ int s2a_device_error(unsigned int* flags, int clear);
  */
 int s2a_selftest_wait_expiry(void* cuda_stream);
 
+/* Self-test of an assumption of the fixed-width bfloat16 softmax forward (row lengths 49, 50,
+ * 64, 197, 257).  Those kernels do not search y for the range of Eq. 8: they take the row's
+ * smallest and largest INPUT and send both through the same operations as every element.  That
+ * equals min(y) and max(y) as written provided no operation on the way ever decreases when its
+ * argument grows.  The correctly rounded ones cannot; the GPU's approximate 2^x is checked by
+ * this call: it evaluates it at every binary32 argument between -150 and 1 (all the kernels can
+ * produce; below -126 the result is flushed to zero), compares neighbours, and writes the
+ * number of neighbouring pairs found out of order to the HOST word *out_of_order (0 on every
+ * GPU this library is built for; anything else means those kernels must not be trusted there).
+ * About 2.2e9 evaluations, a few milliseconds; synchronises the stream.  Returns S2A_OK,
+ * S2A_ERR_NULL or S2A_ERR_CUDA.
+ */
+int s2a_selftest_exp2_monotone(unsigned long long* out_of_order, void* cuda_stream);
+
 /* How a call would be run: writes into `out` (capacity `cap` bytes, always
  * NUL-terminated) a one-line description of the kernel variant and launch shape chosen
  * for (kernel, row_len, dt, n_elems).  kernel: 0 gelu_fwd, 1 gelu_bwd, 2 softmax_fwd,

@@ -27,6 +27,7 @@ EXPORTS = (
     "s2a_tensor_range_static_max_elems", "s2a_gelu_fwd_tensor_range_static",
     "s2a_silu_fwd", "s2a_silu_bwd", "s2a_cap_fwd", "s2a_cap_bwd", "s2a_lrp_fwd",
     "s2a_selftest_wait_expiry",
+    "s2a_selftest_exp2_monotone",
     "s2a_codes_bytes_bits", "s2a_gelu_fwd_bits", "s2a_gelu_bwd_bits", "s2a_softmax_fwd_bits", "s2a_softmax_bwd_bits",
 )
 
@@ -63,6 +64,8 @@ def lib() -> ctypes.CDLL:
         L.s2a_status_string.restype = c.c_char_p
         L.s2a_selftest_wait_expiry.argtypes = [c.c_void_p]
         L.s2a_selftest_wait_expiry.restype = c.c_int
+        L.s2a_selftest_exp2_monotone.argtypes = [c.POINTER(c.c_ulonglong), c.c_void_p]
+        L.s2a_selftest_exp2_monotone.restype = c.c_int
         for name in ("s2a_gelu_fwd", "s2a_softmax_fwd", "s2a_gelu_bwd", "s2a_softmax_bwd", "s2a_silu_fwd",
                      "s2a_silu_bwd"):
             f = getattr(L, name)

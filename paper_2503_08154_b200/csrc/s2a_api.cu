@@ -243,6 +243,11 @@ int s2a_selftest_wait_expiry(void* cuda_stream) {
   return launch_wait_expiry_probe((cudaStream_t)cuda_stream) == cudaSuccess ? S2A_OK : S2A_ERR_CUDA;
 }
 
+int s2a_selftest_exp2_monotone(unsigned long long* out_of_order, void* cuda_stream) {
+  if (!out_of_order) return S2A_ERR_NULL;
+  return count_exp2_out_of_order(out_of_order, (cudaStream_t)cuda_stream) == cudaSuccess ? S2A_OK : S2A_ERR_CUDA;
+}
+
 int s2a_describe_plan(int kernel, size_t n_elems, size_t row_len, int dt, char* out, size_t cap) {
   if (!out || cap == 0) return S2A_ERR_NULL;
   out[0] = 0;

@@ -98,5 +98,7 @@ cudaError_t read_error_word(unsigned int* flags, bool clear);
 
 // Launches the bounded wait's self-test (a wait that is meant to run out after 2 ms).
 cudaError_t launch_wait_expiry_probe(cudaStream_t st);
+// Counts the neighbouring binary32 arguments in [-150, 1] at which the hardware's approximate 2^x decreases.
+cudaError_t count_exp2_out_of_order(unsigned long long* count, cudaStream_t st);
 
 }  // namespace s2a

@@ -419,6 +419,43 @@ cudaError_t launch_wait_expiry_probe(cudaStream_t st) {
   return cudaGetLastError();
 }
 
+// The fixed-width bfloat16 softmax forward takes a row's smallest and largest y from its smallest
+// and largest x.  That holds when every operation between x and y never decreases as its input
+// grows: the correctly rounded ones (fused multiply-add, product, rounding to bfloat16) cannot;
+// the hardware's approximate 2^x is CHECKED here, over every binary32 argument the kernel can hand
+// it (-150 .. 1; below -126 the result is flushed to zero): neighbouring arguments are compared
+// and the pairs out of order are counted.
+namespace {
+__device__ unsigned long long g_exp2_out_of_order;
+constexpr uint32_t kBitsMinus150 = 0xC3160000u, kBitsMinusZero = 0x80000000u, kBitsOne = 0x3F800000u;
+__global__ void exp2_monotone_probe() {
+  const uint64_t n_neg = kBitsMinus150 - kBitsMinusZero, n_pos = kBitsOne;
+  unsigned long long bad = 0;
+  for (uint64_t k = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; k < n_neg + n_pos; k += (uint64_t)gridDim.x * blockDim.x) {
+    if (k < n_neg) {  // negative arguments: the larger bit pattern is the smaller number
+      const uint32_t b = kBitsMinusZero + (uint32_t)k;
+      bad += ex2_approx(__uint_as_float(b + 1)) > ex2_approx(__uint_as_float(b));
+    } else {
+      const uint32_t b = (uint32_t)(k - n_neg);
+      bad += ex2_approx(__uint_as_float(b + 1)) < ex2_approx(__uint_as_float(b));
+    }
+  }
+  if (bad) atomicAdd(&g_exp2_out_of_order, bad);
+}
+}  // namespace
+
+cudaError_t count_exp2_out_of_order(unsigned long long* count, cudaStream_t st) {
+  const unsigned long long zero = 0;
+  cudaError_t e = cudaMemcpyToSymbolAsync(g_exp2_out_of_order, &zero, sizeof(zero), 0, cudaMemcpyHostToDevice, st);
+  if (e != cudaSuccess) return e;
+  exp2_monotone_probe<<<sm_count() * 8, 256, 0, st>>>();
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  e = cudaMemcpyFromSymbolAsync(count, g_exp2_out_of_order, sizeof(*count), 0, cudaMemcpyDeviceToHost, st);
+  if (e != cudaSuccess) return e;
+  return cudaStreamSynchronize(st);
+}
+
 cudaError_t read_error_word(unsigned int* flags, bool clear) {
   cudaError_t e = cudaMemcpyFromSymbol(flags, g_error_word, sizeof(unsigned int));
   if (e != cudaSuccess) return e;

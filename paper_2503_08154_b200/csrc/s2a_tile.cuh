@@ -1991,26 +1991,41 @@ struct PairSoftmaxFwd<kBF16, UNIT_, LCT> {
   template <int HP>
   static __device__ __forceinline__ bool drop_hi(int i, int ul) { return HP == 0 && i == G::LAST_I && ul == G::LAST_UL; }
 
+  // Loads the row's words (foreign and absent halves become -inf, so that they vanish from the
+  // exponentials) and returns the row's largest AND smallest input: softmax is monotone, so the
+  // extreme outputs sit at the extreme inputs and the range of y needs no reduction of its own
+  // (see front()).
   template <int HP>
-  static __device__ __forceinline__ float load_max(Regs& R, const uint32_t* words, int ul) {
-    constexpr uint32_t kNegInf2 = 0xFF80FF80u;
-    uint32_t mx2 = kNegInf2;
+  static __device__ __forceinline__ void load_minmax(Regs& R, const uint32_t* words, int ul, float& mx, float& mn) {
+    constexpr uint32_t kNegInf2 = 0xFF80FF80u, kPosInf2 = 0x7F807F80u;
+    uint32_t mx2 = kNegInf2, mn2 = kPosInf2;
 #pragma unroll
     for (int i = 0; i < G::ITERS; ++i) {
-      uint32_t w = kNegInf2;
-      if (G::has(i, ul)) w = words[UNIT_ * i];
-      if (drop_lo<HP>(i, ul)) w = (w & 0xffff0000u) | 0xFF80u;      // foreign low half
-      if (drop_hi<HP>(i, ul)) w = (w & 0x0000ffffu) | 0xFF800000u;  // foreign high half
+      uint32_t w = kNegInf2, wn = kPosInf2;
+      if (G::has(i, ul)) {
+        w = words[UNIT_ * i];
+        wn = w;
+      }
+      if (drop_lo<HP>(i, ul)) {  // foreign low half
+        w = (w & 0xffff0000u) | 0xFF80u;
+        wn = (wn & 0xffff0000u) | 0x7F80u;
+      }
+      if (drop_hi<HP>(i, ul)) {  // foreign high half
+        w = (w & 0x0000ffffu) | 0xFF800000u;
+        wn = (wn & 0x0000ffffu) | 0x7F800000u;
+      }
       R.w[i] = w;
       mx2 = max2(mx2, w);
+      mn2 = min2(mn2, wn);
     }
-    return fmaxf(lo(mx2), hi(mx2));
+    mx = fmaxf(lo(mx2), hi(mx2));
+    mn = fminf(lo(mn2), hi(mn2));
   }
 
   // All binary32 arithmetic below runs on packed pairs (one instruction per word).
-  static __device__ __forceinline__ float exp_sum(Regs& R, float m) {
+  static __device__ __forceinline__ float exp_sum(Regs& R, float nm) {  // nm = -(row maximum) * log2 e
     constexpr float kLog2e = 1.4426950408889634f;
-    const F2 k2 = f2_both(kLog2e), nm2 = f2_both(-m * kLog2e);
+    const F2 k2 = f2_both(kLog2e), nm2 = f2_both(nm);
     F2 z2 = f2_both(0.0f);
 #pragma unroll
     for (int i = 0; i < G::ITERS; ++i) {
@@ -2025,29 +2040,29 @@ struct PairSoftmaxFwd<kBF16, UNIT_, LCT> {
   }
 
   template <int HP>
-  static __device__ __forceinline__ void scale_store(Regs& R, float rz, uint32_t* out, int ul, bool active,
-                                                     float& mn, float& mx) {
-    uint32_t mn2 = 0x7F807F80u, mx2 = 0xFF80FF80u;
+  static __device__ __forceinline__ void scale_store(Regs& R, float rz, uint32_t* out, int ul, bool active) {
     const F2 rz2 = f2_both(rz);
 #pragma unroll
     for (int i = 0; i < G::ITERS; ++i) {
       const uint32_t w = f2_to_bf16x2(f2_mul(R.e[i], rz2));  // y as written
       R.w[i] = w;
-      if (G::has(i, ul)) {
-        uint32_t wm = w;  // for min/max a foreign half is replaced by its neighbour
-        if (drop_lo<HP>(i, ul)) wm = (w & 0xffff0000u) | (w >> 16);
-        if (drop_hi<HP>(i, ul)) wm = (w & 0x0000ffffu) | (w << 16);
-        mn2 = min2(mn2, wm);
-        mx2 = max2(mx2, wm);
-        if (active) {
-          if (drop_lo<HP>(i, ul)) *((uint16_t*)(out + UNIT_ * i) + 1) = (uint16_t)(w >> 16);
-          else if (drop_hi<HP>(i, ul)) *(uint16_t*)(out + UNIT_ * i) = (uint16_t)w;
-          else out[UNIT_ * i] = w;
-        }
+      if (active && G::has(i, ul)) {
+        if (drop_lo<HP>(i, ul)) *((uint16_t*)(out + UNIT_ * i) + 1) = (uint16_t)(w >> 16);
+        else if (drop_hi<HP>(i, ul)) *(uint16_t*)(out + UNIT_ * i) = (uint16_t)w;
+        else out[UNIT_ * i] = w;
       }
     }
-    mn = fminf(lo(mn2), hi(mn2));
-    mx = fmaxf(lo(mx2), hi(mx2));
+  }
+
+  // y as written at the row's smallest and largest input -- the very operations every element
+  // goes through (one fused multiply-add, 2^x, the scaling, the rounding to bfloat16), each of
+  // them monotone, so these ARE the minimum and the maximum of the row's y as written.
+  static __device__ __forceinline__ void range_of_y(float x_min, float x_max, float nm, float rz, float& mn, float& mx) {
+    float a0, a1;
+    f2_unpack(f2_fma(f2_pack(x_min, x_max), f2_both(1.4426950408889634f), f2_both(nm)), a0, a1);
+    const uint32_t w = f2_to_bf16x2(f2_mul(f2_pack(ex2_approx(a0), ex2_approx(a1)), f2_both(rz)));
+    mn = lo(w);
+    mx = hi(w);
   }
 
   // Code byte of word i of a row (a foreign half codes as 0: it is replaced by the minimum).
@@ -2067,19 +2082,28 @@ struct PairSoftmaxFwd<kBF16, UNIT_, LCT> {
     const int ul = u.ul;
     const uint32_t a0 = (r * (uint32_t)LCT) >> 1, a1 = ((r + 1) * (uint32_t)LCT) >> 1;  // odd: a1 = a0 + NACC - 1
     constexpr int HA = G::kOdd ? 0 : 2, HB = G::kOdd ? 1 : 2;  // the kinds of the pair's two rows
-    float mA = load_max<HA>(A, (const uint32_t*)p.data + a0 + ul, ul);
-    float mB = load_max<HB>(B, (const uint32_t*)p.data + a1 + ul, ul);
+    float mA, mB, nA, nB;  // the rows' largest and smallest inputs
+    load_minmax<HA>(A, (const uint32_t*)p.data + a0 + ul, ul, mA, nA);
+    load_minmax<HB>(B, (const uint32_t*)p.data + a1 + ul, ul, mB, nB);
     {
-      // both row maxima are bfloat16 values: they travel down ONE shuffle chain as a packed pair
-      __nv_bfloat162 pm = __floats2bfloat162_rn(mA, mB);
-      uint32_t w = *(uint32_t*)&pm;
+      // all four are bfloat16 values: the maxima travel down one shuffle chain as a packed pair,
+      // the minima down another
+      __nv_bfloat162 pm = __floats2bfloat162_rn(mA, mB), pn = __floats2bfloat162_rn(nA, nB);
+      uint32_t w = *(uint32_t*)&pm, v = *(uint32_t*)&pn;
 #pragma unroll
-      for (int o = UNIT_ / 2; o > 0; o >>= 1) w = max2(w, __shfl_xor_sync(0xffffffffu, w, o));
+      for (int o = UNIT_ / 2; o > 0; o >>= 1) {
+        w = max2(w, __shfl_xor_sync(0xffffffffu, w, o));
+        v = min2(v, __shfl_xor_sync(0xffffffffu, v, o));
+      }
       mA = lo(w);
       mB = hi(w);
+      nA = lo(v);
+      nB = hi(v);
     }
-    float zA = exp_sum(A, mA);
-    float zB = exp_sum(B, mB);
+    constexpr float kLog2e = 1.4426950408889634f;
+    const float nmA = -mA * kLog2e, nmB = -mB * kLog2e;
+    float zA = exp_sum(A, nmA);
+    float zB = exp_sum(B, nmB);
     {
       F2 z2 = f2_pack(zA, zB);  // the two sums are reduced together, one packed addition per step
 #pragma unroll
@@ -2090,13 +2114,14 @@ struct PairSoftmaxFwd<kBF16, UNIT_, LCT> {
       }
       f2_unpack(z2, zA, zB);
     }
-    float mnA, mxA, mnB, mxB;
     // 1 / z to about an ulp (hardware reciprocal and one correction step): y is rounded to 8 bits
     const float rA0 = rcp_approx(zA), rB0 = rcp_approx(zB);
-    scale_store<HA>(A, __fmaf_rn(__fmaf_rn(-zA, rA0, 1.0f), rA0, rA0), (uint32_t*)p.data + a0 + ul, ul, active, mnA, mxA);
-    scale_store<HB>(B, __fmaf_rn(__fmaf_rn(-zB, rB0, 1.0f), rB0, rB0), (uint32_t*)p.data + a1 + ul, ul, active, mnB, mxB);
-    reduce_minmax_bf16<UNIT_>(mnA, mxA);
-    reduce_minmax_bf16<UNIT_>(mnB, mxB);
+    const float rzA = __fmaf_rn(__fmaf_rn(-zA, rA0, 1.0f), rA0, rA0), rzB = __fmaf_rn(__fmaf_rn(-zB, rB0, 1.0f), rB0, rB0);
+    scale_store<HA>(A, rzA, (uint32_t*)p.data + a0 + ul, ul, active);
+    scale_store<HB>(B, rzB, (uint32_t*)p.data + a1 + ul, ul, active);
+    float mnA, mxA, mnB, mxB;
+    range_of_y(nA, mA, nmA, rzA, mnA, mxA);
+    range_of_y(nB, mB, nmB, rzB, mnB, mxB);
     // Eq. 8's two correctly rounded quotients per row, LEVELS / d and d / LEVELS, for both rows with ONE
     // division: lane 0 of the unit forms LEVELS / dA, lane 1 dA / LEVELS, lane 2 LEVELS / dB, lane 3 dB / LEVELS
     // (the other lanes repeat them), and four shuffles hand the results round.

@@ -153,6 +153,40 @@ def test_degenerate_rows(dt, L):
     check_softmax(synth.to_io(xs.reshape(-1), dt), synth.to_io(g, dt), L, dt)
 
 
+@pytest.mark.parametrize("L", [49, 50, 64, 197, 257])
+@pytest.mark.parametrize("dt", [F32, BF16])
+def test_softmax_extremes_at_every_position(dt, L):
+    # The fixed-width bfloat16 kernels find the range of y from the row's smallest and largest
+    # input.  Every position of a row takes a turn at holding the maximum and the minimum (the
+    # first and last elements share a 4-byte word with the neighbouring row when L is odd), some
+    # rows hold several equal extremes, some a masked (hugely negative) entry: check_softmax
+    # compares (min, s) and every code with Q(y as written), without tolerance.
+    rows = 3 * L + 5
+    x = synth.normal(9, ("ext", L, dt), rows * L).reshape(rows, L) * np.float32(1.5)
+    r = np.arange(rows)
+    hi_at, lo_at = r % L, (3 * r + 1) % L
+    x[r, lo_at] = -9.0
+    x[r, hi_at] = 6.0                       # where both fall on one element the maximum wins
+    x[5, :] = np.where(np.arange(L) % 2 == 0, 1.25, -1.25)   # many equal extremes
+    x[6, 0], x[6, L - 1] = 6.5, -9.5        # extremes in the two halves shared with neighbours
+    x[7, 0], x[7, L - 1] = -9.5, 6.5
+    x[8, L // 2] = -1.0e4                   # a masked entry: y underflows to exactly 0
+    x[9, 0] = -1.0e4
+    x[10, L - 1] = -1.0e4
+    g = synth.normal(9, ("extg", L, dt), rows * L)
+    check_softmax(synth.to_io(x.reshape(-1).astype(np.float32), dt), synth.to_io(g, dt), L, dt, max_flip_frac=5e-3)
+
+
+def test_hardware_exp2_never_decreases_over_the_arguments_softmax_uses():
+    # exhaustive: every binary32 argument in [-150, 1], neighbours compared on the device
+    import ctypes
+    lib = binding.lib()
+    bad = ctypes.c_ulonglong(12345)
+    assert lib.s2a_selftest_exp2_monotone(ctypes.byref(bad), ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)) == 0
+    assert bad.value == 0, "2^x approximate decreases at %d neighbouring arguments" % bad.value
+    assert lib.s2a_selftest_exp2_monotone(None, None) == 1   # S2A_ERR_NULL
+
+
 @pytest.mark.parametrize("L", [197, 64, 145, 1024])
 @pytest.mark.parametrize("dt", [F32, BF16])
 def test_softmax_large_common_offset(dt, L):
