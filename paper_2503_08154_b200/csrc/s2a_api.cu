@@ -261,10 +261,10 @@ int s2a_describe_plan(int kernel, size_t n_elems, size_t row_len, int dt, char* 
   } else {
     snprintf(out, cap,
              "tile variant=%s rows/tile=%u unit=%u vec=%u iters=%u warps=%u stages=%u smem=%u grid=%u "
-             "group=%u spread=%u tiles=%llu tail_rows=%llu",
+             "group=%u spread=%u ragged_codes=%u tiles=%llu tail_rows=%llu",
              p.variant == kVariantStream ? "stream" : (p.variant == kVariantPairFixed ? "pair-fixed" : (p.variant == kVariantAny ? "any-length" : "generic")),
              p.tile_rows, p.unit_lanes, p.vec_elems, p.iters, p.warps, p.stages, p.smem_bytes,
-             p.grid, p.rows_per_group, p.spread_units, (unsigned long long)p.n_tiles,
+             p.grid, p.rows_per_group, p.spread_units, p.ragged_codes, (unsigned long long)p.n_tiles,
              (unsigned long long)(n_rows - p.n_tiles * p.tile_rows));
   }
   return S2A_OK;

@@ -77,6 +77,7 @@ struct TilePlan {
   uint32_t bits;        // code width of Eq. 8: 4, or 2 / 8 (GELU rows of whole 16-byte vectors)
   uint32_t rows_per_group;  // rows a unit takes together (the kernel's WORK::rows_per_group); divides tile_rows
   uint32_t spread_units;    // 1: the sub-warp units of a warp take groups tile_groups / (units per warp) apart
+  uint32_t ragged_codes;    // 1: a tile's code bytes need not start on a 16-byte boundary of the code tensor
 };
 
 struct TileArgs {

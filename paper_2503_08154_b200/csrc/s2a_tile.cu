@@ -109,6 +109,21 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
   const uint32_t epc = 128u / (uint32_t)bits;  // elements per 16 code bytes
   uint32_t r_min = epc / gcd_u32(L, epc);
   if (r_min < 2) r_min = 2;
+  // Widths 577 and 1025: only every 32nd row starts on a 16-byte boundary of the code tensor, and
+  // 32 rows are 37-131 KB of data: two stages at best, a single one for binary32 rows of 1025.
+  // Their kernels can take tiles whose codes start anywhere (see tile_kernel's RAGGED): the row
+  // count only has to make the DATA a multiple of 16 bytes (and be even), so a tile is 8 or 16
+  // rows.  Measured on [97536, 1025] and [173280, 577], forward / backward TB/s, aligned 32-row
+  // tiles -> ragged ones: 1025 binary32 3.27 / 5.24 -> 5.62 / 6.25, 1025 bfloat16 5.54 / 6.15 ->
+  // 6.00 / 5.6, 577 binary32 5.78 / 5.87 -> 6.09 / 6.72, 577 bfloat16 5.81 / 5.59 -> 5.7 / 5.91:
+  // taken wherever it won.
+  const bool sm_fwd = kernel == kSoftmaxFwd, sm_bwd = kernel == kSoftmaxBwd;
+  const bool ragged = pair_width && env_int("S2A_RAGGED", 1) != 0 &&
+                      ((L == 1025 && !(dt == kBF16 && sm_bwd)) || (L == 577 && !(dt == kBF16 && sm_fwd)));
+  if (ragged) {
+    r_min = 16u / gcd_u32(L * esize, 16u);
+    if (r_min < 2) r_min = 2;
+  }
   if ((uint64_t)r_min * L * esize > kHardStageBytes) return p;
 
   uint32_t variant = kVariantGeneric, unit = 0, iters = 0;
@@ -210,6 +225,10 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
 
   uint32_t warps = unit == 128 ? 8u : 4u;
   if (variant == kVariantPairFixed && unit == 32) warps = 8;  // four row pairs in flight are too few (measured)
+  // ragged tiles: 16 rows for eight warps, except (measured) binary32 1025 forward -- 8 rows, four
+  // warps, two CTAs of two stages -- and binary32 577 backward -- 8 rows, four warps, one CTA of four stages
+  const bool ragged_small = ragged && dt == kF32 && ((L == 1025 && sm_fwd) || (L == 577 && sm_bwd));
+  if (ragged_small) warps = 4;
   if (variant == kVariantAny) {
     // eight consumer warps, four when that many sub-warp units would need a tile beyond 40 KB
     const uint32_t want = 256u / unit;  // rows that keep eight warps busy
@@ -233,6 +252,7 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
   int ctas_per_sm = short_rows ? 4 : 2;
   if (variant == kVariantStream && is_gelu) ctas_per_sm = 4;
   if (variant == kVariantPairFixed) ctas_per_sm = 4;
+  if (ragged_small && L == 577) ctas_per_sm = 1;
   // The GELU backward runs with eight warps on four-row tiles, two CTAs per SM: alone it gains
   // 1-3 % (hidden 4096 / 5120, where two rows leave room for two stages only), and in training
   // order, alternating with the softmax backward, the step gains 3 % (ViT-B/16 5733 -> 5917 GB/s,
@@ -273,6 +293,7 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
     while (rows % (n_units * G) != 0 && (uint64_t)(rows + r_min) * L * esize <= kMaxStageBytes) rows += r_min;
     if (short_rows)
       while ((uint64_t)rows * L * esize < 7 * 1024) rows *= 2;
+    if (ragged) rows = n_units * G;  // one row pair per unit and round: 8 or 16 rows, multiples of r_min
   }
   rows = (uint32_t)env_int("S2A_TILE_ROWS", (int)rows);
   if (rows == 0 || rows % r_min != 0 || rows % G != 0 || (uint64_t)rows * L * esize > kHardStageBytes) return p;
@@ -281,7 +302,7 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
   const uint32_t code_bytes = (uint32_t)((uint64_t)rows * L * (uint32_t)bits / 8);
   const uint32_t meta_bytes = rows * 8;
   const uint32_t code_off = align_up(data_bytes, 128);
-  const uint32_t meta_off = code_off + align_up(code_bytes, 128);
+  const uint32_t meta_off = code_off + align_up(code_bytes + (ragged ? 32u : 0u), 128);
   const uint32_t stage_bytes = meta_off + align_up(meta_bytes, 128);
 
   // CTAs per SM and stages per CTA.  Every tile kernel asks for a power-of-two fraction
@@ -330,6 +351,10 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
   if (stages == 0) return p;
 
   p.n_tiles = n_rows / rows;
+  // the backward loads the aligned span that covers a tile's codes: where that span of the very
+  // last tile would reach beyond the code tensor, that tile is left to the row-at-a-time path
+  if (ragged && p.n_tiles != 0 && n_rows % rows == 0 && (p.n_tiles * code_bytes) % 16 != 0) p.n_tiles -= 1;
+  p.ragged_codes = ragged ? 1u : 0u;
   if (p.n_tiles == 0) return TilePlan{};
   p.tile_rows = rows;
   p.variant = variant;
@@ -371,7 +396,7 @@ cudaError_t launch_tile(int kernel, int dt, const TilePlan& p, const TileArgs& a
   ka.code_bytes = (uint32_t)((uint64_t)p.tile_rows * a.row_len * p.bits / 8);
   ka.meta_bytes = p.tile_rows * 8;
   ka.code_off = align_up(ka.data_bytes, 128);
-  ka.meta_off = ka.code_off + align_up(ka.code_bytes, 128);
+  ka.meta_off = ka.code_off + align_up(ka.code_bytes + (p.ragged_codes ? 32u : 0u), 128);  // as plan_tile
   ka.stage_bytes = ka.meta_off + align_up(ka.meta_bytes, 128);
   ka.stages = p.stages;
   ka.tab_off = p.bits != 4 ? kHeaderBytes + p.stages * ka.stage_bytes : 0u;  // the area after the stages
@@ -381,6 +406,7 @@ cudaError_t launch_tile(int kernel, int dt, const TilePlan& p, const TileArgs& a
   // with the predecessor's last stores)
   ka.prefetch_tiles = p.overlap_launch ? (uint32_t)env_int("S2A_PREFETCH", p.stages < 2 ? (int)p.stages : 2) : 0u;
   ka.prefetch_ahead = (uint32_t)env_int("S2A_X1", 0);
+  ka.ragged_codes = p.ragged_codes;
   ka.error_word = error_word_address();
   if (!ka.error_word) return cudaErrorInvalidDevice;
   if (p.bits != 4) return launch_tile_bits(kernel, dt, p, &ka, st);

@@ -60,6 +60,7 @@ struct TileKernelArgs {
   uint32_t tab_off;          // byte offset of the wide derivative tables (8-bit codes), else 0
   uint32_t prefetch_tiles;   // tiles whose inputs the copy lane asks into the L2 before the dependency wait
   uint32_t prefetch_ahead;   // steady state: with the load of tile i, tile i + this many is asked into the L2 (0: off)
+  uint32_t ragged_codes;     // 1: a tile's code bytes start anywhere (tile_kernel<WORK, true> only), see there
   unsigned int* error_word;  // device address of the per-device error word
 };
 
@@ -2532,7 +2533,28 @@ struct PairSoftmaxBwdBits {
 };
 
 // ---------------------------------------------------------------- the kernel
-template <class WORK>
+// RAGGED: the code bytes of a tile need not start on a 16-byte boundary of the code tensor (a
+// bulk copy must).  Rows of 1025 elements own 512.5 code bytes each, so only every 32nd row
+// starts on such a boundary, and 32 rows of binary32 data are too large a tile to
+// double-buffer.  With RAGGED a tile is any even number of rows whose DATA is a multiple of 16
+// bytes.  Its codes sit in the stage at the same offset modulo 16 as in global memory
+// (code_shift below): the backward loads the 16-byte-aligned span that covers them, the forward
+// writes the aligned middle with one bulk store and the up to 15 bytes before and after it
+// with plain byte stores of the copy lane.  The kernels that use it access codes bytewise.
+struct CodeSpan {
+  uint64_t start;    // byte offset of the tile's codes in the code tensor
+  uint32_t shift;    // start % 16: where they begin inside the stage's code area
+  uint32_t cover;    // bytes of the aligned span covering them (loads)
+};
+__device__ __forceinline__ CodeSpan code_span(uint64_t tile, uint32_t code_bytes) {
+  CodeSpan c;
+  c.start = tile * code_bytes;
+  c.shift = (uint32_t)c.start & 15u;
+  c.cover = (c.shift + code_bytes + 15u) & ~15u;
+  return c;
+}
+
+template <class WORK, bool RAGGED = false>
 __global__ void __maxnreg__(WORK::kMaxRegs) tile_kernel(TileKernelArgs a) {
   extern __shared__ __align__(1024) unsigned char smem[];
   constexpr int KERNEL = WORK::kKernel;
@@ -2570,7 +2592,12 @@ __global__ void __maxnreg__(WORK::kMaxRegs) tile_kernel(TileKernelArgs a) {
       const uint64_t t = blockIdx.x + (uint64_t)i * gridDim.x;
       bulk_prefetch_l2(a.in + t * a.data_bytes, a.data_bytes);
       if (!kFwd) {
-        bulk_prefetch_l2(a.codes + t * a.code_bytes, a.code_bytes);
+        if (RAGGED) {
+          const CodeSpan c = code_span(t, a.code_bytes);
+          bulk_prefetch_l2(a.codes + (c.start - c.shift), c.cover);
+        } else {
+          bulk_prefetch_l2(a.codes + t * a.code_bytes, a.code_bytes);
+        }
         bulk_prefetch_l2(a.meta + t * a.meta_bytes, a.meta_bytes);
       }
     }
@@ -2588,11 +2615,13 @@ __global__ void __maxnreg__(WORK::kMaxRegs) tile_kernel(TileKernelArgs a) {
       const uint64_t t = blockIdx.x + it * gridDim.x;
       unsigned char* st = smem + kHeaderBytes + (size_t)s * a.stage_bytes;
       uint64_t* bar = &full[s];
-      const uint32_t bytes = kFwd ? a.data_bytes : a.data_bytes + a.code_bytes + a.meta_bytes;
+      const CodeSpan c = code_span(t, a.code_bytes);
+      const uint32_t code_load = RAGGED ? c.cover : a.code_bytes;
+      const uint32_t bytes = kFwd ? a.data_bytes : a.data_bytes + code_load + a.meta_bytes;
       mbar_arrive_expect_tx(bar, bytes);
       bulk_load(st, a.in + t * a.data_bytes, a.data_bytes, bar);
       if (!kFwd) {
-        bulk_load(st + a.code_off, a.codes + t * a.code_bytes, a.code_bytes, bar);
+        bulk_load(st + a.code_off, a.codes + (RAGGED ? c.start - c.shift : c.start), code_load, bar);
         bulk_load(st + a.meta_off, a.meta + t * a.meta_bytes, a.meta_bytes, bar);
       }
     };
@@ -2600,7 +2629,8 @@ __global__ void __maxnreg__(WORK::kMaxRegs) tile_kernel(TileKernelArgs a) {
       const uint64_t t = blockIdx.x + it * gridDim.x;
       bulk_prefetch_l2(a.in + t * a.data_bytes, a.data_bytes);
       if (!kFwd) {
-        bulk_prefetch_l2(a.codes + t * a.code_bytes, a.code_bytes);
+        const CodeSpan c = code_span(t, a.code_bytes);
+        bulk_prefetch_l2(a.codes + (RAGGED ? c.start - c.shift : c.start), RAGGED ? c.cover : a.code_bytes);
         bulk_prefetch_l2(a.meta + t * a.meta_bytes, a.meta_bytes);
       }
     };
@@ -2618,7 +2648,20 @@ __global__ void __maxnreg__(WORK::kMaxRegs) tile_kernel(TileKernelArgs a) {
       unsigned char* st = smem + kHeaderBytes + (size_t)s * a.stage_bytes;
       bulk_store(a.out + t * a.data_bytes, st, a.data_bytes);
       if (kFwd) {
-        bulk_store(a.codes + t * a.code_bytes, st + a.code_off, a.code_bytes);
+        if (RAGGED) {
+          const CodeSpan c = code_span(t, a.code_bytes);
+          const unsigned char* src = st + a.code_off + c.shift;
+          unsigned char* dst = a.codes + c.start;
+          const uint32_t head = (16u - c.shift) & 15u;             // bytes before the first boundary
+          const uint32_t mid = (a.code_bytes - head) & ~15u;       // whole 16-byte pieces (code_bytes >= 32)
+          bulk_store(dst + head, src + head, mid);
+#pragma unroll 1
+          for (uint32_t k = 0; k < head; ++k) dst[k] = src[k];
+#pragma unroll 1
+          for (uint32_t k = head + mid; k < a.code_bytes; ++k) dst[k] = src[k];
+        } else {
+          bulk_store(a.codes + t * a.code_bytes, st + a.code_off, a.code_bytes);
+        }
         bulk_store(a.meta + t * a.meta_bytes, st + a.meta_off, a.meta_bytes);
       }
       bulk_commit();
@@ -2672,7 +2715,8 @@ __global__ void __maxnreg__(WORK::kMaxRegs) tile_kernel(TileKernelArgs a) {
     }
     if (!ok) break;
     unsigned char* st = smem + kHeaderBytes + (size_t)s * a.stage_bytes;
-    StagePtrs sp{st, st + a.code_off, (float*)(st + a.meta_off)};
+    const uint32_t code_shift = RAGGED ? code_span(blockIdx.x + it * gridDim.x, a.code_bytes).shift : 0u;
+    StagePtrs sp{st, st + a.code_off + code_shift, (float*)(st + a.meta_off)};
     for (uint32_t rd = 0; rd < rounds; ++rd) {
       uint32_t grp = rd * n_units + u.uid;
       bool active = grp < n_groups;
@@ -2697,9 +2741,10 @@ __global__ void __maxnreg__(WORK::kMaxRegs) tile_kernel(TileKernelArgs a) {
 // ---------------------------------------------------------------- launching
 constexpr uint32_t kMaxSmem = 227 * 1024;
 
-template <class WORK>
+template <class WORK, bool RAGGED = false>
 cudaError_t launch_work(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
-  auto kfn = tile_kernel<WORK>;
+  if (RAGGED != (ka.ragged_codes != 0)) return cudaErrorInvalidValue;
+  auto kfn = tile_kernel<WORK, RAGGED>;
   // The attributes belong to a device's context: one bit per device and instantiation.  Two
   // threads making the first launch on a device may both set them (the same values).
   static std::atomic<uint64_t> configured{0};
@@ -2847,8 +2892,10 @@ template <template <int, int, int> class WORK, int DT>
 cudaError_t launch_pair_widths(const TilePlan& p, const TileKernelArgs& ka, cudaStream_t st) {
   if (p.unit_lanes == 32) {  // the long widths: a warp per row pair
     switch (ka.row_len) {
-      case 577: return launch_work<WORK<DT, 32, 577>>(p, ka, st);
-      case 1025: return launch_work<WORK<DT, 32, 1025>>(p, ka, st);
+      case 577:
+        return ka.ragged_codes ? launch_work<WORK<DT, 32, 577>, true>(p, ka, st) : launch_work<WORK<DT, 32, 577>>(p, ka, st);
+      case 1025:
+        return ka.ragged_codes ? launch_work<WORK<DT, 32, 1025>, true>(p, ka, st) : launch_work<WORK<DT, 32, 1025>>(p, ka, st);
     }
     return cudaErrorInvalidValue;
   }
