@@ -327,9 +327,11 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
     while (ctas_per_sm > 1 && (uint64_t)regs * (warps + 1) * 32 * (uint32_t)ctas_per_sm > 65536) ctas_per_sm /= 2;
   }
   // beyond the stages: 256-entry derivative tables per unit (8-bit GELU backward), or the CTA's
-  // scratch of one unpacked code byte per element of a tile (2-bit fixed-width softmax forward)
+  // scratch of the 2-bit fixed-width softmax forward: one unpacked code byte per element of a tile
+  // (binary32), one byte per 2-element word (bfloat16)
   const uint32_t extra_bytes = (bits == 8 && is_gelu) ? n_units * 1024u
-                               : ((pair_bits && bits == 2 && kernel == kSoftmaxFwd) ? align_up(rows * L, 128) : 0u);
+                               : ((pair_bits && bits == 2 && kernel == kSoftmaxFwd)
+                                      ? align_up(dt == kBF16 ? rows * L / 2 : rows * L, 128) : 0u);
   const int env_stages = env_int("S2A_STAGES", 0);
   uint32_t stages = 0, smem = 0;
   for (int c = ctas_per_sm; c >= 1 && stages == 0; c = (c == 3 ? 2 : c / 2)) {

@@ -2387,8 +2387,8 @@ struct PairSoftmaxFwdBits {
 
 // bfloat16 form of the forward at 2 and 8 bits: the two rows of a pair are worked on together
 // by the 4-bit kernel's own front part (packed arithmetic, shared shuffle chains, one division);
-// only the code phase differs -- a byte per element into the code area (8 bits) or into the
-// scratch that the warp then packs (2 bits).
+// only the code phase differs -- a byte per element into the code area (8 bits), or a nibble per
+// 2-element word into the scratch that the warp then packs (2 bits).
 template <int UNIT_, int LCT, int NBITS>
 struct PairSoftmaxFwdBits<kBF16, UNIT_, LCT, NBITS> {
   static_assert(NBITS == 2 || NBITS == 8, "4 bits have kernels of their own");
@@ -2412,39 +2412,65 @@ struct PairSoftmaxFwdBits<kBF16, UNIT_, LCT, NBITS> {
     QRange qA, qB;
     constexpr int HA = G::kOdd ? 0 : 2, HB = G::kOdd ? 1 : 2;
     B4::template front<(1 << NBITS) - 1>(u, p, r, active, A, B, qA, qB);
-    unsigned char* bytes = NBITS == 8 ? p.codes : (unsigned char*)tab;
     const F2 minA = f2_both(qA.mn), invA = f2_both(qA.inv), minB = f2_both(qB.mn), invB = f2_both(qB.inv);
     const F2 magic2 = f2_both(12582912.0f);
-    constexpr uint32_t kMask = (1u << NBITS) - 1u;
+    if constexpr (NBITS == 8) {
 #pragma unroll
-    for (int i = 0; i < G::ITERS; ++i) {
-      if (active && G::has(i, ul)) {
-        float t0, t1;
-        f2_unpack(f2_add(f2_scaled(f2_from_bf16x2(A.w[i]), minA, invA), magic2), t0, t1);
-        uint32_t c0 = __float_as_uint(t0) & kMask, c1 = __float_as_uint(t1) & kMask;
-        unsigned char* dst = bytes + 2u * (a0 + ul + UNIT_ * i);
-        if (B4::template drop_hi<HA>(i, ul)) dst[0] = (unsigned char)c0;   // the high half is row B's first element
-        else *(uint16_t*)dst = (uint16_t)(c0 | (c1 << 8));
-        f2_unpack(f2_add(f2_scaled(f2_from_bf16x2(B.w[i]), minB, invB), magic2), t0, t1);
-        c0 = __float_as_uint(t0) & kMask;
-        c1 = __float_as_uint(t1) & kMask;
-        dst = bytes + 2u * (a1 + ul + UNIT_ * i);
-        if (B4::template drop_lo<HB>(i, ul)) dst[1] = (unsigned char)c1;   // the low half is row A's last element
-        else *(uint16_t*)dst = (uint16_t)(c0 | (c1 << 8));
+      for (int i = 0; i < G::ITERS; ++i) {
+        if (active && G::has(i, ul)) {
+          float t0, t1;
+          f2_unpack(f2_add(f2_scaled(f2_from_bf16x2(A.w[i]), minA, invA), magic2), t0, t1);
+          uint32_t c0 = __float_as_uint(t0) & 0xFFu, c1 = __float_as_uint(t1) & 0xFFu;
+          unsigned char* dst = p.codes + 2u * (a0 + ul + UNIT_ * i);
+          if (B4::template drop_hi<HA>(i, ul)) dst[0] = (unsigned char)c0;   // the high half is row B's first element
+          else *(uint16_t*)dst = (uint16_t)(c0 | (c1 << 8));
+          f2_unpack(f2_add(f2_scaled(f2_from_bf16x2(B.w[i]), minB, invB), magic2), t0, t1);
+          c0 = __float_as_uint(t0) & 0xFFu;
+          c1 = __float_as_uint(t1) & 0xFFu;
+          dst = p.codes + 2u * (a1 + ul + UNIT_ * i);
+          if (B4::template drop_lo<HB>(i, ul)) dst[1] = (unsigned char)c1;   // the low half is row A's last element
+          else *(uint16_t*)dst = (uint16_t)(c0 | (c1 << 8));
+        }
       }
-    }
-    u.sync();
-    if (NBITS == 2) {
-      // as the general form: the warp packs its own eight consecutive rows
+      u.sync();
+    } else {
+      // 2 bits: a word's two codes make a nibble (a foreign half codes as 0), one scratch byte per
+      // WORD of the tile; the word the two rows share is written by row B with row A's code merged
+      // in (as the 4-bit kernel does with its shared byte).  The warp then packs the scratch of its
+      // eight rows, two nibbles to a code byte.
+      unsigned char* nibbles = (unsigned char*)tab;
+      auto nibble = [&](uint32_t w, bool no_lo, bool no_hi, const QRange& q, F2 min2, F2 inv2) -> uint32_t {
+        float v0 = B4::lo(w), v1 = B4::hi(w);
+        if (no_lo) v0 = q.mn;
+        if (no_hi) v1 = q.mn;
+        float t0, t1;
+        f2_unpack(f2_add(f2_scaled(f2_pack(v0, v1), min2, inv2), magic2), t0, t1);
+        return (__float_as_uint(t0) + (__float_as_uint(t1) << 2)) & 0xFu;  // 0x4B400000 has no bits there
+      };
+      const uint32_t a_last = nibble(A.w[G::LAST_I], B4::template drop_lo<HA>(G::LAST_I, ul),
+                                     B4::template drop_hi<HA>(G::LAST_I, ul), qA, minA, invA);
+      const uint32_t shared_lo = __shfl_sync(0xffffffffu, a_last, (threadIdx.x & 31 & ~(UNIT_ - 1)) | G::LAST_UL);
+#pragma unroll
+      for (int i = 0; i < G::ITERS; ++i) {
+        if (active && G::has(i, ul)) {
+          if (!G::kOdd || !(i == G::LAST_I && ul == G::LAST_UL))
+            nibbles[a0 + ul + UNIT_ * i] = (unsigned char)nibble(A.w[i], B4::template drop_lo<HA>(i, ul),
+                                                                 B4::template drop_hi<HA>(i, ul), qA, minA, invA);
+          uint32_t b = nibble(B.w[i], B4::template drop_lo<HB>(i, ul), B4::template drop_hi<HB>(i, ul), qB, minB, invB);
+          if (G::kOdd && i == 0 && ul == 0) b |= shared_lo & 0x3u;
+          nibbles[a1 + ul + UNIT_ * i] = (unsigned char)b;
+        }
+      }
+      u.sync();
       __syncwarp();
-      const uint32_t e_begin = (grp - (uint32_t)(u.uid & 3)) * 2u * (uint32_t)LCT;
+      // the warp's eight rows are 4 L words, starting at a multiple of 4 L: four scratch bytes
+      // (4-byte aligned) make two code bytes
+      const uint32_t w_begin = (grp - (uint32_t)(u.uid & 3)) * (uint32_t)LCT;
       if (active) {
-        // eight scratch bytes (8-byte aligned: e_begin is a multiple of 8 L) make two code bytes
         for (uint32_t b = threadIdx.x & 31u; b < (uint32_t)LCT; b += 32u) {
-          const uint2 w = *(const uint2*)(bytes + e_begin + 8u * b);
-          const uint32_t lo = (w.x & 3u) | ((w.x >> 6) & 0xCu) | ((w.x >> 12) & 0x30u) | ((w.x >> 18) & 0xC0u);
-          const uint32_t hi = (w.y & 3u) | ((w.y >> 6) & 0xCu) | ((w.y >> 12) & 0x30u) | ((w.y >> 18) & 0xC0u);
-          *(uint16_t*)(p.codes + e_begin / 4u + 2u * b) = (uint16_t)(lo | (hi << 8));
+          const uint32_t w = *(const uint32_t*)(nibbles + w_begin + 4u * b);
+          const uint32_t t = (w & 0x000F000Fu) | ((w >> 4) & 0x00F000F0u);   // bytes 0 and 2: the two code bytes
+          *(uint16_t*)(p.codes + w_begin / 2u + 2u * b) = (uint16_t)__byte_perm(t, 0u, 0x4420u);
         }
       }
       __syncwarp();
