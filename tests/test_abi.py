@@ -134,3 +134,32 @@ def test_every_plan_gives_each_unit_whole_row_groups(lib):
                 n_units = f["warps"] * 32 // unit
                 assert n_units >= 1 and (f["warps"] * 32) % unit == 0, text
     assert seen_spread > 0
+
+
+def test_tiles_whose_codes_start_off_the_16_byte_grid_stay_inside_the_code_tensor(lib):
+    """Widths 577 / 1025 may take tiles of 8 or 16 rows, whose code bytes begin anywhere.  The
+    data of such a tile must still be whole 16-byte pieces, its rows even (no byte shared with
+    another tile), and the aligned span the backward loads for the LAST tile must end inside the
+    code tensor: either rows are left for the row path, or the tiles end on the grid."""
+    seen = 0
+    for L in (577, 1025):
+        for dt, esize in ((0, 4), (1, 2)):
+            for kernel in (2, 3):
+                for n_rows in (16, 40, 48, 72, 163, 1000, 2000, 9000, 97536, 173280):
+                    text = binding.s2a_describe_plan(kernel, n_rows * L, L, dt)
+                    if not text.startswith("tile"):
+                        continue
+                    f = {k: int(v) for k, v in _plan_fields(text).items() if v.isdigit()}
+                    rows, tiles, tail = f["rows/tile"], f["tiles"], f["tail_rows"]
+                    assert tiles * rows + tail == n_rows, text
+                    assert rows % 2 == 0 and (rows * L * esize) % 16 == 0, text
+                    if f["ragged_codes"]:
+                        seen += 1
+                        code_bytes = rows * L // 2
+                        assert (rows * L) % 2 == 0 and code_bytes >= 32, text
+                        end = tiles * code_bytes
+                        total = (n_rows * L + 1) // 2
+                        assert (end + 15) // 16 * 16 <= total or end % 16 == 0, text
+                    else:
+                        assert (rows * L // 2) % 16 == 0, text
+    assert seen > 0
