@@ -2,6 +2,7 @@
 // per-device error word.
 #include "s2a_tile.cuh"
 
+#include <stdio.h>
 #include <stdlib.h>
 
 #include <atomic>
@@ -29,8 +30,14 @@ constexpr uint32_t kHardStageBytes = 176 * 1024;  // the smallest legal tile may
 // (build.py --tuning writes it to a file of its own).  The library proper reads no
 // environment variable: a plan is a pure function of its arguments and the device.
 #ifdef S2A_TUNING
+// An override may be given for one kernel only: K<kernel id>_<name> (K3_S2A_CTAS_PER_SM=3) is
+// looked up before <name>.
+thread_local int tuning_kernel = -1;
 int env_int(const char* name, int dflt) {
-  const char* v = getenv(name);
+  char scoped[96];
+  snprintf(scoped, sizeof scoped, "K%d_%s", tuning_kernel, name);
+  const char* v = getenv(scoped);
+  if (!(v && *v)) v = getenv(name);
   return (v && *v) ? atoi(v) : dflt;
 }
 const char* env_str(const char* name) { return getenv(name); }
@@ -86,6 +93,9 @@ unsigned int* error_word_address() {
 TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
   TilePlan p{};
   p.bits = (uint32_t)bits;
+#ifdef S2A_TUNING
+  tuning_kernel = kernel;
+#endif
   if (bits != 4 && bits != 2 && bits != 8) return p;
   const char* path = env_str("S2A_PATH");
   if (path && path[0] == 'r') return p;
