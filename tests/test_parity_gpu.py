@@ -180,6 +180,43 @@ def test_softmax_extremes_at_every_position(dt, L):
     check_softmax(synth.to_io(x.reshape(-1).astype(np.float32), dt), synth.to_io(g, dt), L, dt, max_flip_frac=5e-3)
 
 
+def _random_shapes(seed, count):
+    """Seeded (rows, L) pairs: lengths near the widths that have kernels of their own, powers of
+    two and their neighbours, and arbitrary ones; row counts that leave ragged tails or none."""
+    rng = np.random.RandomState(seed)
+    special = [49, 50, 64, 145, 196, 197, 198, 257, 577, 1025, 3072, 4096]
+    out = []
+    for i in range(count):
+        kind = i % 3
+        if kind == 0:
+            L = int(special[rng.randint(len(special))] + rng.randint(-1, 2))
+        elif kind == 1:
+            L = int(2 ** rng.randint(3, 12) + rng.randint(-1, 2))
+        else:
+            L = int(rng.randint(1, 2200))
+        rows = int(rng.randint(1, max(2, min(3000, 600000 // max(L, 1)))))
+        if rng.randint(2):
+            rows = max(32, rows // 32 * 32)      # whole tiles, no tail
+        out.append((rows, max(L, 1)))
+    return out
+
+
+@pytest.mark.parametrize("dt", [F32, BF16])
+def test_seeded_random_shapes(dt):
+    # the planner picks a kernel form and a tile per (kernel, length, type): a seeded walk over
+    # shapes nobody chose by hand, every one compared with the oracle like the listed shapes
+    for rows, L in _random_shapes(20250308, 36):
+        check_gelu(*_gelu_inputs(rows, L, dt, seed=rows + L), L, dt)
+        check_softmax(*_softmax_inputs(rows, L, dt, seed=rows + L), L, dt, max_flip_frac=8e-3)
+
+
+@pytest.mark.parametrize("rows,L,dt", [(97536, 1025, F32), (173280, 577, BF16)])
+def test_sweep_size_tensors_of_the_wide_odd_widths(rows, L, dt):
+    # the bandwidth sweep's tensors at 577 / 1025 (1e8 elements): thousands of tiles whose code
+    # bytes start at every offset of the 16-byte grid, all ranks of the persistent grid busy
+    check_softmax(*_softmax_inputs(rows, L, dt, seed=3), L, dt, report="[%d, %d]" % (rows, L))
+
+
 def test_hardware_exp2_never_decreases_over_the_arguments_softmax_uses():
     # exhaustive: every binary32 argument in [-150, 1], neighbours compared on the device
     import ctypes
