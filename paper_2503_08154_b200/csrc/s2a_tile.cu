@@ -333,6 +333,11 @@ TilePlan plan_tile(int kernel, int dt, uint64_t n_rows, uint32_t L, int bits) {
     uint32_t regs = 128;
     if (variant == kVariantStream) regs = is_gelu ? 64u : (uint32_t)softmax_stream_regs(dt, (int)(iters * epa));
     if (variant == kVariantPairFixed) regs = 96;
+    // the bfloat16 kernels at width 257 are built for 128 registers: three CTAs per SM
+    if (variant == kVariantPairFixed && bits == 4 && dt == kBF16 && L == 257) {
+      regs = 128;
+      if (ctas_per_sm > 3) ctas_per_sm = 3;
+    }
     if (variant == kVariantAny) regs = 80;
     while (ctas_per_sm > 1 && (uint64_t)regs * (warps + 1) * 32 * (uint32_t)ctas_per_sm > 65536) ctas_per_sm /= 2;
   }

@@ -1958,7 +1958,9 @@ struct PairSoftmaxFwd {
 // and the exponent's argument is one fused multiply-add.
 template <int UNIT_, int LCT>
 struct PairSoftmaxFwd<kBF16, UNIT_, LCT> {
-  static constexpr int kMaxRegs = 96;  // 4 CTAs of 160 threads per SM
+  // 4 CTAs of 160 threads per SM; width 257 (17 words per lane and row) runs with 3 CTAs of three stages
+  // and 128 registers: 28.6 -> 28.0 us (with 96 registers three CTAs had measured slower than four)
+  static constexpr int kMaxRegs = LCT == 257 ? 128 : 96;
   static constexpr int kKernel = kSoftmaxFwd;
   static constexpr int UNIT = UNIT_;
   using G = PairGeom<UNIT_, LCT>;
@@ -2178,7 +2180,9 @@ struct PairSoftmaxFwd<kBF16, UNIT_, LCT> {
 
 template <int DT, int UNIT_, int LCT>
 struct PairSoftmaxBwd {
-  static constexpr int kMaxRegs = 96;  // 4 CTAs of 160 threads per SM
+  // 4 CTAs of 160 threads per SM; the bfloat16 kernel at width 257 runs with 3 CTAs per SM (its stages
+  // fit a quarter of the shared memory only twice) and may use the registers that frees: 25.5 -> 24.9 us
+  static constexpr int kMaxRegs = (LCT == 257 && DT == kBF16) ? 128 : 96;
   static constexpr int kKernel = kSoftmaxBwd;
   static constexpr int UNIT = UNIT_;
   using P = P2<DT>;
