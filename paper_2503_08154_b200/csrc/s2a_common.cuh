@@ -238,11 +238,13 @@ __device__ __forceinline__ F2 f2_act_fast(F2 x) {
   f2_unpack(f2_add(f2_pack(ex2_approx(k0), ex2_approx(k1)), f2_both(1.0f)), d0, d1);
   return f2_mul(x, f2_pack(rcp_approx(d0), rcp_approx(d1)));
 }
-// Four elements with ONE reciprocal: 1 / (d0 d1 d2 d3) and seven multiplications give the
-// four 1 / d_i (the special-function unit, at a quarter of the rate of the other pipes, is what
-// the forward kernel's row work waits for; this takes its load from 8 to 5 operations per four
-// elements).  Each d_i = 1 + 2^k_i must stay below 2^31 for the product to stay finite:
-// callers use it on rows whose minimum is at or above kQuadFloor (k <= 30).
+// Four elements per call, two elements per reciprocal: 1 / (d0 d1) and two multiplications give
+// 1 / d0 and 1 / d1.  The forward kernel's row work is bound by instruction issue first and by the
+// special-function unit (a quarter of the other pipes' rate) second; measured on the ViT-B/16
+// GELU launch at sustained clocks: a reciprocal per element (8 special-function operations per four
+// elements) 31.3 us, one per four elements (5 operations, seven multiplications) 30.6 us, one per
+// pair (6 operations, four multiplications) 30.3 us.  Each d_i = 1 + 2^k_i: callers use this on
+// rows whose minimum is at or above kQuadFloor (k <= 30), so that a product stays far from overflow.
 template <int ACT>
 struct ActQuad {
   static constexpr float kQuadFloor = -30.0f / (Act<ACT>::kSlopeOf * 1.4426950408889634f);
@@ -253,9 +255,7 @@ struct ActQuad {
     f2_unpack(f2_mul(xb, c2), k2, k3);
     f2_unpack(f2_add(f2_pack(ex2_approx(k0), ex2_approx(k1)), one2), d0, d1);
     f2_unpack(f2_add(f2_pack(ex2_approx(k2), ex2_approx(k3)), one2), d2, d3);
-    const float pa = d0 * d1, pb = d2 * d3;
-    const float r = rcp_approx(pa * pb);
-    const float ra = r * pb, rb = r * pa;                    // 1 / (d0 d1), 1 / (d2 d3)
+    const float ra = rcp_approx(d0 * d1), rb = rcp_approx(d2 * d3);
     ya = f2_mul(xa, f2_mul(f2_pack(d1, d0), f2_both(ra)));   // x0 / d0, x1 / d1
     yb = f2_mul(xb, f2_mul(f2_pack(d3, d2), f2_both(rb)));
   }

@@ -719,7 +719,7 @@ struct StreamActFwd {
   static __device__ __forceinline__ void init(State&) {}
   static __device__ __forceinline__ uint32_t rows_per_group(uint32_t) { return 1u; }
 
-  // FAST: the short bfloat16 form of the activation (four elements share one reciprocal), valid
+  // FAST: the short bfloat16 form of the activation (two elements share one reciprocal), valid
   // on rows with no element below ActQuad::kQuadFloor (the caller knows the row minimum before
   // the second pass).
   template <bool FAST>
