@@ -315,6 +315,32 @@ struct Unit {
     }
     return v;
   }
+  // Minimum of a packed bfloat16x2 over the unit, both halves at once (a row's minimum and the
+  // negative of its maximum travel together: one shuffle sequence, one exchange between warps).
+  __device__ __forceinline__ uint32_t reduce_min_bf16x2(uint32_t w) {
+    constexpr int W = UNIT < 32 ? UNIT : 32;
+#pragma unroll
+    for (int o = W / 2; o > 0; o >>= 1) {
+      const uint32_t other = __shfl_xor_sync(0xffffffffu, w, o);
+      const __nv_bfloat162 r = __hmin2(*(const __nv_bfloat162*)&w, *(const __nv_bfloat162*)&other);
+      w = *(const uint32_t*)&r;
+    }
+    if (UNIT > 32) {
+      constexpr int NW = UNIT / 32;
+      uint32_t* slot = (uint32_t*)red + (phase & 1) * 64;
+      if ((ul & 31) == 0) slot[ul >> 5] = w;
+      named_bar_sync(1 + uid, UNIT);
+      w = slot[0];
+#pragma unroll
+      for (int k = 1; k < NW; ++k) {
+        const uint32_t other = slot[k];
+        const __nv_bfloat162 r = __hmin2(*(const __nv_bfloat162*)&w, *(const __nv_bfloat162*)&other);
+        w = *(const uint32_t*)&r;
+      }
+      ++phase;
+    }
+    return w;
+  }
   // Orders shared-memory accesses of the unit's lanes (and keeps them in step).
   __device__ __forceinline__ void sync() {
     if (UNIT > 32) named_bar_sync(1 + uid, UNIT);
@@ -792,19 +818,87 @@ struct StreamActFwd {
     const uint32_t nv = active ? L / V::EPA : 0u;
     unsigned char* row = p.data + (size_t)r * L * Io<DT>::kBytes;
     unsigned char* crow = p.codes + (size_t)r * (L / 2);
-    typename V::MinMax mm;
-    mm.init();
-    if (NVL > 0) {
+    float mn, mx;
+    if constexpr (DT == kBF16) {
+      // The range of Eq. 8 is that of the CLIPPED row, so of the maximum only "at least the clip
+      // value, or else its exact value" matters: it is taken over each lane's first vector, and
+      // the whole row is searched only if that sample stays below the clip (a hidden vector of
+      // thousands of activations practically never does).  The minimum is needed exactly -- it
+      // also decides which form of the activation the second pass may use.  Packed bfloat16 pairs
+      // throughout; (min, -max) are reduced together.
+      auto min4 = [](uint32_t m, const uint4& v) {
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-      for (int i = 0; i < NVL; ++i) mm.add(*(const typename V::Raw*)(row + (u.ul + UNIT_ * i) * 16u));
-    } else {
+        for (int k = 0; k < 4; ++k) {
+          const __nv_bfloat162 a = __hmin2(*(const __nv_bfloat162*)&m, *(const __nv_bfloat162*)&w[k]);
+          m = *(const uint32_t*)&a;
+        }
+        return m;
+      };
+      auto max4 = [](uint32_t m, const uint4& v) {
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const __nv_bfloat162 a = __hmax2(*(const __nv_bfloat162*)&m, *(const __nv_bfloat162*)&w[k]);
+          m = *(const uint32_t*)&a;
+        }
+        return m;
+      };
+      auto lo = [](uint32_t w) { return __uint_as_float(w << 16); };
+      auto hi = [](uint32_t w) { return __uint_as_float(w & 0xffff0000u); };
+      uint32_t mn2 = 0x7F807F80u, mx2 = 0xFF80FF80u;
+      if (NVL > 0) {
+#pragma unroll
+        for (int i = 0; i < NVL; ++i) {
+          const uint4 v = *(const uint4*)(row + (u.ul + UNIT_ * i) * 16u);
+          mn2 = min4(mn2, v);
+          if (i == 0) mx2 = max4(mx2, v);
+        }
+      } else {
+        if ((uint32_t)u.ul < nv) mx2 = max4(mx2, *(const uint4*)(row + u.ul * 16u));
 #pragma unroll 4
-      for (uint32_t j = u.ul; j < nv; j += UNIT_) mm.add(*(const typename V::Raw*)(row + j * 16u));
+        for (uint32_t j = u.ul; j < nv; j += UNIT_) mn2 = min4(mn2, *(const uint4*)(row + j * 16u));
+      }
+      const __nv_bfloat162 both = __floats2bfloat162_rn(fminf(lo(mn2), hi(mn2)), -fmaxf(lo(mx2), hi(mx2)));  // exact
+      const uint32_t w = u.reduce_min_bf16x2(*(const uint32_t*)&both);
+      mn = lo(w);
+      mx = -hi(w);
+      // The decision is the same in every lane of a unit; sub-warp units share their warp's
+      // shuffles, so there the whole warp searches as soon as one of its units has to (a unit that
+      // did not need it finds its exact maximum, which clips to the same value).
+      bool search = mx < kActClip;
+      if (UNIT_ < 32) search = __any_sync(0xffffffffu, search);
+      if (search) {
+        mx2 = 0xFF80FF80u;
+        for (uint32_t j = u.ul; j < nv; j += UNIT_) mx2 = max4(mx2, *(const uint4*)(row + j * 16u));
+        mx = u.template reduce<kOpMax>(fmaxf(lo(mx2), hi(mx2)));
+      }
+    } else {
+      typename V::MinMax mm;
+      mm.init();
+      if (NVL > 0) {
+#pragma unroll
+        for (int i = 0; i < NVL; ++i) mm.add(*(const typename V::Raw*)(row + (u.ul + UNIT_ * i) * 16u));
+      } else {
+#pragma unroll 4
+        for (uint32_t j = u.ul; j < nv; j += UNIT_) mm.add(*(const typename V::Raw*)(row + j * 16u));
+      }
+      mn = u.template reduce<kOpMin>(mm.lo());
+      mx = u.template reduce<kOpMax>(mm.hi());
     }
-    const float mn = u.template reduce<kOpMin>(mm.lo());
-    const float mx = u.template reduce<kOpMax>(mm.hi());
-    // min / max of the clipped row = clipped min / max of the row (the clip is monotone)
-    const QRange q = make_qrange(fminf(fmaxf(mn, -kActClip), kActClip), fminf(fmaxf(mx, -kActClip), kActClip));
+    // min / max of the clipped row = clipped min / max of the row (the clip is monotone).  A row
+    // that reaches both clip values has the same range as every other such row: its two
+    // quotients are constants, correctly rounded at compile time.
+    const float cmn = fminf(fmaxf(mn, -kActClip), kActClip), cmx = fminf(fmaxf(mx, -kActClip), kActClip);
+    QRange q;
+    if (cmn == -kActClip && cmx == kActClip) {
+      constexpr float kFullInv = kLevels / (2.0f * kActClip), kFullS = (2.0f * kActClip) / kLevels;
+      q.mn = -kActClip;
+      q.inv = kFullInv;
+      q.s = kFullS;
+    } else {
+      q = make_qrange(cmn, cmx);
+    }
     if (active && u.ul == 0) { p.meta[2 * r] = q.mn; p.meta[2 * r + 1] = q.s; }
     // mn is the same in every lane of the unit, so the branch does not diverge
     if (DT == kBF16 && mn >= ActQuad<ACT>::kQuadFloor) second_pass<true>(row, crow, u.ul, nv, q);
