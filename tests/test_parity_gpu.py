@@ -257,6 +257,26 @@ def test_gelu_far_negative_inputs_keep_their_tiny_outputs(rows, L, dt):
     check_gelu(synth.to_io(x.reshape(-1), dt), synth.to_io(g, dt), L, dt)
 
 
+@pytest.mark.parametrize("L", [64, 128, 256, 1024, 3072])
+def test_gelu_rows_whose_maximum_hides_at_the_end(L):
+    # The bfloat16 forward takes a row's maximum from the first 16-byte vector of every lane and
+    # searches the whole row only when that sample stays below the clip.  Neighbouring rows here
+    # take different turns: saturated within the sample, saturated only by the row's last
+    # element, not saturated at all, constant -- in one warp where several rows share a warp.
+    rows = 96
+    x = synth.normal(11, ("hide", L), rows * L).reshape(rows, L) * np.float32(0.3)
+    x = np.clip(x, -1.5, 1.5)
+    kind = np.arange(rows) % 6
+    x[kind == 0, 0] = 5.0
+    x[kind == 0, 1] = -5.0
+    x[kind == 1, L - 1] = 2.5           # only the last element reaches the clip
+    x[kind == 2, L - 1] = 1.75          # the maximum sits at the end and stays below the clip
+    x[kind == 3, L - 1] = -7.0          # the minimum sits at the end
+    x[kind == 4, :] = 0.625             # constant
+    g = synth.normal(11, ("hideg", L), rows * L)
+    check_gelu(synth.to_io(x.reshape(-1).astype(np.float32), BF16), synth.to_io(g, BF16), L, BF16)
+
+
 def _double_rounding_tie_rows(L, n_rows, seed):
     """binary32 rows whose elements sit where Eq. 8's pinned sequence needs BOTH of its roundings:
     the exact product (x - min) * inv is not a half-integer, but its binary32 rounding is exactly
