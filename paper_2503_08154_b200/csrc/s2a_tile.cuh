@@ -732,6 +732,101 @@ struct CodePacker {
   }
 };
 
+// First pass of the activation forward over one row in shared memory: the row's exact minimum
+// and its maximum "up to the clip" (exact when below `clip`, otherwise some value >= clip).
+template <int DT, int UNIT_, int NVL>
+__device__ __forceinline__ void act_row_extremes(Unit<UNIT_>& u, const unsigned char* row, uint32_t nv, float clip,
+                                                 float& mn, float& mx) {
+  using V = V16<DT>;
+  if constexpr (DT == kBF16) {
+    // The range of Eq. 8 is that of the CLIPPED row, so of the maximum only "at least the clip
+    // value, or else its exact value" matters: it is taken over each lane's first vector, and
+    // the whole row is searched only if that sample stays below the clip (a hidden vector of
+    // thousands of activations practically never does).  The minimum is needed exactly -- it
+    // also decides which form of the activation the second pass may use.  Packed bfloat16 pairs
+    // throughout; (min, -max) are reduced together.
+    auto min4 = [](uint32_t m, const uint4& v) {
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const __nv_bfloat162 a = __hmin2(*(const __nv_bfloat162*)&m, *(const __nv_bfloat162*)&w[k]);
+        m = *(const uint32_t*)&a;
+      }
+      return m;
+    };
+    auto max4 = [](uint32_t m, const uint4& v) {
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const __nv_bfloat162 a = __hmax2(*(const __nv_bfloat162*)&m, *(const __nv_bfloat162*)&w[k]);
+        m = *(const uint32_t*)&a;
+      }
+      return m;
+    };
+    auto lo = [](uint32_t w) { return __uint_as_float(w << 16); };
+    auto hi = [](uint32_t w) { return __uint_as_float(w & 0xffff0000u); };
+    uint32_t mn2 = 0x7F807F80u, mx2 = 0xFF80FF80u;
+    if (NVL > 0) {
+#pragma unroll
+      for (int i = 0; i < NVL; ++i) {
+        const uint4 v = *(const uint4*)(row + (u.ul + UNIT_ * i) * 16u);
+        mn2 = min4(mn2, v);
+        if (i == 0) mx2 = max4(mx2, v);
+      }
+    } else {
+      if ((uint32_t)u.ul < nv) mx2 = max4(mx2, *(const uint4*)(row + u.ul * 16u));
+#pragma unroll 4
+      for (uint32_t j = u.ul; j < nv; j += UNIT_) mn2 = min4(mn2, *(const uint4*)(row + j * 16u));
+    }
+    const __nv_bfloat162 both = __floats2bfloat162_rn(fminf(lo(mn2), hi(mn2)), -fmaxf(lo(mx2), hi(mx2)));  // exact
+    const uint32_t w = u.reduce_min_bf16x2(*(const uint32_t*)&both);
+    mn = lo(w);
+    mx = -hi(w);
+    // The decision is the same in every lane of a unit; sub-warp units share their warp's
+    // shuffles, so there the whole warp searches as soon as one of its units has to (a unit that
+    // did not need it finds its exact maximum, which clips to the same value).
+    bool search = mx < clip;
+    if (UNIT_ < 32) search = __any_sync(0xffffffffu, search);
+    if (search) {
+      mx2 = 0xFF80FF80u;
+      for (uint32_t j = u.ul; j < nv; j += UNIT_) mx2 = max4(mx2, *(const uint4*)(row + j * 16u));
+      mx = u.template reduce<kOpMax>(fmaxf(lo(mx2), hi(mx2)));
+    }
+  } else {
+    typename V::MinMax mm;
+    mm.init();
+    if (NVL > 0) {
+#pragma unroll
+      for (int i = 0; i < NVL; ++i) mm.add(*(const typename V::Raw*)(row + (u.ul + UNIT_ * i) * 16u));
+    } else {
+#pragma unroll 4
+      for (uint32_t j = u.ul; j < nv; j += UNIT_) mm.add(*(const typename V::Raw*)(row + j * 16u));
+    }
+    mn = u.template reduce<kOpMin>(mm.lo());
+    mx = u.template reduce<kOpMax>(mm.hi());
+  }
+}
+
+// Eq. 8's range of a row clipped to +-clip, from the row's extremes: min / max of the clipped row
+// = clipped min / max of the row (the clip is monotone).  A row that reaches both clip values has
+// the same range as every other such row: its two quotients are constants, correctly rounded at
+// compile time.
+template <int ACT, int LEVELS>
+__device__ __forceinline__ QRange clipped_qrange(float mn, float mx) {
+  constexpr float kClip = Act<ACT>::kClipOf;
+  const float cmn = fminf(fmaxf(mn, -kClip), kClip), cmx = fminf(fmaxf(mx, -kClip), kClip);
+  QRange q;
+  if (cmn == -kClip && cmx == kClip) {
+    constexpr float kFullInv = (float)LEVELS / (2.0f * kClip), kFullS = (2.0f * kClip) / (float)LEVELS;
+    q.mn = -kClip;
+    q.inv = kFullInv;
+    q.s = kFullS;
+  } else {
+    q = make_qrange(cmn, cmx, (float)LEVELS);
+  }
+  return q;
+}
+
 // NVL > 0 fixes the number of vectors per lane (row_len == NVL * UNIT * EPA), which lets
 // the compiler drop every loop counter and bound check; NVL == 0 is the general loop.
 template <int DT, int UNIT_, int NVL, int ACT>
@@ -819,86 +914,8 @@ struct StreamActFwd {
     unsigned char* row = p.data + (size_t)r * L * Io<DT>::kBytes;
     unsigned char* crow = p.codes + (size_t)r * (L / 2);
     float mn, mx;
-    if constexpr (DT == kBF16) {
-      // The range of Eq. 8 is that of the CLIPPED row, so of the maximum only "at least the clip
-      // value, or else its exact value" matters: it is taken over each lane's first vector, and
-      // the whole row is searched only if that sample stays below the clip (a hidden vector of
-      // thousands of activations practically never does).  The minimum is needed exactly -- it
-      // also decides which form of the activation the second pass may use.  Packed bfloat16 pairs
-      // throughout; (min, -max) are reduced together.
-      auto min4 = [](uint32_t m, const uint4& v) {
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const __nv_bfloat162 a = __hmin2(*(const __nv_bfloat162*)&m, *(const __nv_bfloat162*)&w[k]);
-          m = *(const uint32_t*)&a;
-        }
-        return m;
-      };
-      auto max4 = [](uint32_t m, const uint4& v) {
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const __nv_bfloat162 a = __hmax2(*(const __nv_bfloat162*)&m, *(const __nv_bfloat162*)&w[k]);
-          m = *(const uint32_t*)&a;
-        }
-        return m;
-      };
-      auto lo = [](uint32_t w) { return __uint_as_float(w << 16); };
-      auto hi = [](uint32_t w) { return __uint_as_float(w & 0xffff0000u); };
-      uint32_t mn2 = 0x7F807F80u, mx2 = 0xFF80FF80u;
-      if (NVL > 0) {
-#pragma unroll
-        for (int i = 0; i < NVL; ++i) {
-          const uint4 v = *(const uint4*)(row + (u.ul + UNIT_ * i) * 16u);
-          mn2 = min4(mn2, v);
-          if (i == 0) mx2 = max4(mx2, v);
-        }
-      } else {
-        if ((uint32_t)u.ul < nv) mx2 = max4(mx2, *(const uint4*)(row + u.ul * 16u));
-#pragma unroll 4
-        for (uint32_t j = u.ul; j < nv; j += UNIT_) mn2 = min4(mn2, *(const uint4*)(row + j * 16u));
-      }
-      const __nv_bfloat162 both = __floats2bfloat162_rn(fminf(lo(mn2), hi(mn2)), -fmaxf(lo(mx2), hi(mx2)));  // exact
-      const uint32_t w = u.reduce_min_bf16x2(*(const uint32_t*)&both);
-      mn = lo(w);
-      mx = -hi(w);
-      // The decision is the same in every lane of a unit; sub-warp units share their warp's
-      // shuffles, so there the whole warp searches as soon as one of its units has to (a unit that
-      // did not need it finds its exact maximum, which clips to the same value).
-      bool search = mx < kActClip;
-      if (UNIT_ < 32) search = __any_sync(0xffffffffu, search);
-      if (search) {
-        mx2 = 0xFF80FF80u;
-        for (uint32_t j = u.ul; j < nv; j += UNIT_) mx2 = max4(mx2, *(const uint4*)(row + j * 16u));
-        mx = u.template reduce<kOpMax>(fmaxf(lo(mx2), hi(mx2)));
-      }
-    } else {
-      typename V::MinMax mm;
-      mm.init();
-      if (NVL > 0) {
-#pragma unroll
-        for (int i = 0; i < NVL; ++i) mm.add(*(const typename V::Raw*)(row + (u.ul + UNIT_ * i) * 16u));
-      } else {
-#pragma unroll 4
-        for (uint32_t j = u.ul; j < nv; j += UNIT_) mm.add(*(const typename V::Raw*)(row + j * 16u));
-      }
-      mn = u.template reduce<kOpMin>(mm.lo());
-      mx = u.template reduce<kOpMax>(mm.hi());
-    }
-    // min / max of the clipped row = clipped min / max of the row (the clip is monotone).  A row
-    // that reaches both clip values has the same range as every other such row: its two
-    // quotients are constants, correctly rounded at compile time.
-    const float cmn = fminf(fmaxf(mn, -kActClip), kActClip), cmx = fminf(fmaxf(mx, -kActClip), kActClip);
-    QRange q;
-    if (cmn == -kActClip && cmx == kActClip) {
-      constexpr float kFullInv = kLevels / (2.0f * kActClip), kFullS = (2.0f * kActClip) / kLevels;
-      q.mn = -kActClip;
-      q.inv = kFullInv;
-      q.s = kFullS;
-    } else {
-      q = make_qrange(cmn, cmx);
-    }
+    act_row_extremes<DT, UNIT_, NVL>(u, row, nv, kActClip, mn, mx);
+    const QRange q = clipped_qrange<ACT, 15>(mn, mx);
     if (active && u.ul == 0) { p.meta[2 * r] = q.mn; p.meta[2 * r + 1] = q.s; }
     // mn is the same in every lane of the unit, so the branch does not diverge
     if (DT == kBF16 && mn >= ActQuad<ACT>::kQuadFloor) second_pass<true>(row, crow, u.ul, nv, q);
@@ -1053,14 +1070,9 @@ struct StreamActFwdBits {
     const uint32_t nv = L / V::EPA;
     unsigned char* row = p.data + (size_t)r * L * Io<DT>::kBytes;
     unsigned char* crow = p.codes + (size_t)r * (L / V::EPA) * C::BYTES;
-    typename V::MinMax mm;
-    mm.init();
-#pragma unroll 4
-    for (uint32_t j = u.ul; j < nv; j += UNIT_) mm.add(*(const typename V::Raw*)(row + j * 16u));
-    const float mn = u.template reduce<kOpMin>(mm.lo());
-    const float mx = u.template reduce<kOpMax>(mm.hi());
-    const QRange q = make_qrange(fminf(fmaxf(mn, -kActClip), kActClip), fminf(fmaxf(mx, -kActClip), kActClip),
-                                 (float)((1 << NBITS) - 1));
+    float mn, mx;
+    act_row_extremes<DT, UNIT_, 0>(u, row, nv, kActClip, mn, mx);
+    const QRange q = clipped_qrange<ACT, (1 << NBITS) - 1>(mn, mx);
     if (u.ul == 0) { p.meta[2 * r] = q.mn; p.meta[2 * r + 1] = q.s; }
 #pragma unroll 2
     for (uint32_t j = u.ul; j < nv; j += UNIT_) {
